@@ -1,0 +1,11 @@
+"""CPU oracle for the Trivance AllReduce path.  TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package.  It never imports the CUDA package and the CUDA package never
+imports it.
+"""
+from .oracle import (  # noqa: F401
+    ALGO_BRUCK, ALGO_RECDOUB, ALGO_TRIVANCE, VARIANT_BANDWIDTH, VARIANT_LATENCY,
+    OracleError, allreduce, block_bounds, block_propagation, build, link_loads,
+    naive_sum_f32, num_steps, peers, send_set, step_list,
+)

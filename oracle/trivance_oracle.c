@@ -1,0 +1,496 @@
+/*
+ * Trivance AllReduce -- plain CPU oracle.  TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is the slow, literal restatement of what the Trivance paper's
+ * AllReduce computes, used to check the CUDA library.  Only tests, the smoke
+ * check and the benchmark's CPU-baseline leg may call it; the product never
+ * does.  It shares no code, header, table or constant with the CUDA path.
+ *
+ * What it follows (paper sections):
+ *   - problem statement: every rank ends with the element-wise reduction of
+ *     all n input vectors (Sec. 2.2);
+ *   - peers pi(r,k,n) = (r - 3^k, r + 3^k) mod n (Sec. 4.1);
+ *   - latency-optimal form: log3 n steps, whole vector to both peers, joint
+ *     reduction of the two received vectors with the local partial (Sec. 4.2);
+ *   - bandwidth-optimal form: Reduce-Scatter over n blocks, block sets from
+ *     the recursive BlockPropagation procedure (Algorithm 1, Sec. 4.3), then
+ *     AllGather in reverse order (Sec. 4.1);
+ *   - D-dimensional tori: D collectives on 1/D of the vector each, every
+ *     collective on a different dimension in every step (Sec. 5);
+ *   - congestion c_k = number of messages sharing a link in a step under
+ *     deterministic shortest-path routing inside one dimension (Sec. 2.1,
+ *     Fig. 1, App. E); Bruck-style and Recursive-Doubling schedules only as
+ *     link-load comparators (Sec. 2.4, Fig. 1).
+ *
+ * Readings where the paper is silent (each also listed in the design notes):
+ *   - a joint reduction adds as (from_left + own) + from_right, where "left"
+ *     is the peer r - 3^k.  PARITY UNPINNED by the paper: any fixed order
+ *     satisfies every published fact; the tests pin it to this reading with an
+ *     independent ternary-tree evaluator.
+ *   - slice c of a D-dim torus is elements [floor(cE/D), floor((c+1)E/D));
+ *     block j of a slice [lo,hi) is [lo+floor(j*L/n), lo+floor((j+1)*L/n)),
+ *     L = hi-lo; ranks are linearised r = x0 + a0*x1 + a0*a1*x2 ...; block j
+ *     is owned by linear rank j; collective c uses, at step t, the next
+ *     dimension in round-robin order starting at c that still has steps left,
+ *     with distance 3^(earlier visits of that dimension).  PARITY UNPINNED by
+ *     the paper beyond "collective 0 starts horizontal, collective 1 vertical
+ *     and they swap every step" (Sec. 5).
+ *   - int32 addition wraps modulo 2^32.
+ *
+ * Floating point: binary32 (or binary64 for the error-bound checks), one add
+ * at a time, no contraction, no reassociation.  Compile with
+ *   gcc -O2 -ffp-contract=off -fno-fast-math -std=c99
+ *
+ * All functions work on an element WINDOW [e0,e1) of a global per-rank vector
+ * of E elements: columns are independent, so a window gives exactly the values
+ * the full run would give for those columns.  Arrays are [n][w], w = e1-e0.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_MAX_DIMS 8
+
+enum { ORC_OK = 0, ORC_BAD_ARG = 1, ORC_UNDEFINED = 2, ORC_NOMEM = 3, ORC_INTERNAL = 4 };
+enum { ORC_TRIVANCE = 0, ORC_BRUCK = 1, ORC_RECDOUB = 2 };
+enum { ORC_LATENCY = 0, ORC_BANDWIDTH = 1 };
+enum { ORC_I32 = 0, ORC_F32 = 1, ORC_F64 = 2 };
+
+typedef struct {
+    int algo, ndims, n, S;          /* S = steps per phase, summed over dimensions */
+    int base;                       /* 3 (Trivance, Bruck) or 2 (Recursive Doubling) */
+    int dims[ORC_MAX_DIMS];
+    int stride[ORC_MAX_DIMS];       /* rank = sum x_d * stride_d */
+    int sdim[ORC_MAX_DIMS];         /* steps spent in dimension d = log_base a_d */
+} orc_topo;
+
+static int ilog_exact(int a, int base) {       /* log_base a, or -1 if a is no power */
+    int s = 0;
+    if (a < 1) return -1;
+    while (a > 1) { if (a % base) return -1; a /= base; ++s; }
+    return s;
+}
+
+static int topo_init(orc_topo *tp, const int32_t *dims, int ndims, int algo) {
+    if (!dims || ndims < 1 || ndims > ORC_MAX_DIMS) return ORC_BAD_ARG;
+    if (algo != ORC_TRIVANCE && algo != ORC_BRUCK && algo != ORC_RECDOUB) return ORC_BAD_ARG;
+    tp->algo = algo; tp->ndims = ndims; tp->base = (algo == ORC_RECDOUB) ? 2 : 3;
+    if (algo == ORC_RECDOUB && ndims != 1) return ORC_UNDEFINED;
+    long long n = 1; tp->S = 0;
+    for (int d = 0; d < ndims; ++d) {
+        int s = ilog_exact(dims[d], tp->base);
+        if (s < 1) return (dims[d] >= 2) ? ORC_UNDEFINED : ORC_BAD_ARG;
+        tp->dims[d] = dims[d]; tp->sdim[d] = s; tp->stride[d] = (int)n;
+        n *= dims[d]; tp->S += s;
+        if (n > (1 << 20)) return ORC_BAD_ARG;
+    }
+    tp->n = (int)n;
+    return ORC_OK;
+}
+
+static int ipow(int b, int e) { int r = 1; while (e-- > 0) r *= b; return r; }
+
+/* Step list of collective (slice) c (Sec. 5): round-robin over dimensions,
+ * starting at dimension c, skipping dimensions whose steps are used up; the
+ * distance in a dimension grows by the base each time it is revisited. */
+static void step_list(const orc_topo *tp, int c, int *sdim_out, int *sdist_out) {
+    int visits[ORC_MAX_DIMS] = {0};
+    int cur = c % tp->ndims;
+    for (int t = 0; t < tp->S; ++t) {
+        int d = cur;
+        while (visits[d] >= tp->sdim[d]) d = (d + 1) % tp->ndims;
+        sdim_out[t] = d;
+        sdist_out[t] = ipow(tp->base, visits[d]);
+        visits[d]++;
+        cur = (d + 1) % tp->ndims;
+    }
+}
+
+/* rank reached from r by moving delta positions along dimension d (wraps). */
+static int shift_rank(const orc_topo *tp, int r, int d, int delta) {
+    int a = tp->dims[d], st = tp->stride[d];
+    int x = (r / st) % a;
+    int y = ((x + delta) % a + a) % a;
+    return r + (y - x) * st;
+}
+
+/* Peers a rank SENDS to in a step of (dim, dist).  Returns their number;
+ * dir = +1/-1 ring direction of travel, hops = links crossed.
+ *   Trivance: left = r - dist (travels -), right = r + dist (travels +)  (Sec. 4.1)
+ *   Bruck (as drawn in Fig. 1): r + dist and r + 2*dist, both travelling +  (Sec. 2.4)
+ *   Recursive Doubling: coordinate XOR dist; the lower rank of a pair sends +. */
+static int send_peers(const orc_topo *tp, int r, int d, int dist, int *peer, int *dir, int *hops) {
+    if (tp->algo == ORC_TRIVANCE) {
+        peer[0] = shift_rank(tp, r, d, -dist); dir[0] = -1; hops[0] = dist;
+        peer[1] = shift_rank(tp, r, d, +dist); dir[1] = +1; hops[1] = dist;
+        return 2;
+    }
+    if (tp->algo == ORC_BRUCK) {
+        peer[0] = shift_rank(tp, r, d, dist);     dir[0] = +1; hops[0] = dist;
+        peer[1] = shift_rank(tp, r, d, 2 * dist); dir[1] = +1; hops[1] = 2 * dist;
+        return 2;
+    }
+    {
+        int st = tp->stride[d], x = (r / st) % tp->dims[d];
+        int y = x ^ dist;
+        peer[0] = r + (y - x) * st; dir[0] = (y > x) ? +1 : -1; hops[0] = dist;
+        return 1;
+    }
+}
+
+/* Algorithm 1 (BlockPropagation), generalised from the ring's pi(r,k,n) to the
+ * step list of one collective: marks every rank reachable from r through the
+ * steps step..S-1. */
+static void block_propagation(const orc_topo *tp, const int *sdim, const int *sdist,
+                              int r, int step, uint8_t *blocks) {
+    if (step >= tp->S) return;
+    for (int k = step; k < tp->S; ++k) {
+        int peer[2], dir[2], hops[2];
+        int np = send_peers(tp, r, sdim[k], sdist[k], peer, dir, hops);
+        for (int i = 0; i < np; ++i) blocks[peer[i]] = 1;
+        for (int i = 0; i < np; ++i) block_propagation(tp, sdim, sdist, peer[i], k + 1, blocks);
+    }
+}
+
+/* Blocks a rank sends to peer p in Reduce-Scatter step k: p's own block plus
+ * everything p still has to forward in later steps (Sec. 4.1 / 4.3). */
+static void send_set(const orc_topo *tp, const int *sdim, const int *sdist, int p, int k, uint8_t *set) {
+    memset(set, 0, (size_t)tp->n);
+    set[p] = 1;
+    block_propagation(tp, sdim, sdist, p, k + 1, set);
+}
+
+static void slice_bounds(int64_t E, int D, int c, int64_t *lo, int64_t *hi) {
+    *lo = (int64_t)(((__int128)c * E) / D);
+    *hi = (int64_t)(((__int128)(c + 1) * E) / D);
+}
+static int64_t block_bound(int64_t lo, int64_t hi, int n, int j) {
+    return lo + (int64_t)(((__int128)j * (hi - lo)) / n);
+}
+static int64_t clampi(int64_t v, int64_t a, int64_t b) { return v < a ? a : (v > b ? b : v); }
+
+/* ------------------------------------------------------------------ exported helpers */
+
+int orc_num_steps(const int32_t *dims, int ndims, int algo, int *n_out, int *S_out) {
+    orc_topo tp; int rc = topo_init(&tp, dims, ndims, algo);
+    if (rc) return rc;
+    if (n_out) *n_out = tp.n;
+    if (S_out) *S_out = tp.S;
+    return ORC_OK;
+}
+
+int orc_step_list(const int32_t *dims, int ndims, int algo, int c, int32_t *dim_out, int32_t *dist_out) {
+    orc_topo tp; int rc = topo_init(&tp, dims, ndims, algo);
+    if (rc) return rc;
+    if (c < 0 || c >= ndims) return ORC_BAD_ARG;
+    int sd[64], sx[64];
+    step_list(&tp, c, sd, sx);
+    for (int t = 0; t < tp.S; ++t) { dim_out[t] = sd[t]; dist_out[t] = sx[t]; }
+    return ORC_OK;
+}
+
+/* peers_out[2*r+0] = first peer (Trivance: left), [2*r+1] = second (Trivance: right;
+ * Recursive Doubling: -1). */
+int orc_peers(const int32_t *dims, int ndims, int algo, int c, int step, int32_t *peers_out) {
+    orc_topo tp; int rc = topo_init(&tp, dims, ndims, algo);
+    if (rc) return rc;
+    if (c < 0 || c >= ndims || step < 0 || step >= tp.S) return ORC_BAD_ARG;
+    int sd[64], sx[64];
+    step_list(&tp, c, sd, sx);
+    for (int r = 0; r < tp.n; ++r) {
+        int peer[2] = {-1, -1}, dir[2], hops[2];
+        send_peers(&tp, r, sd[step], sx[step], peer, dir, hops);
+        peers_out[2 * r] = peer[0]; peers_out[2 * r + 1] = peer[1];
+    }
+    return ORC_OK;
+}
+
+/* Raw Algorithm 1: marks[] (n bytes, caller-zeroed or not: it is cleared here). */
+int orc_block_propagation(const int32_t *dims, int ndims, int algo, int c, int r, int step, uint8_t *marks) {
+    orc_topo tp; int rc = topo_init(&tp, dims, ndims, algo);
+    if (rc) return rc;
+    if (c < 0 || c >= ndims || r < 0 || r >= tp.n || step < 0) return ORC_BAD_ARG;
+    int sd[64], sx[64];
+    step_list(&tp, c, sd, sx);
+    memset(marks, 0, (size_t)tp.n);
+    block_propagation(&tp, sd, sx, r, step, marks);
+    return ORC_OK;
+}
+
+/* Blocks sent to peer p in Reduce-Scatter step k of collective c. */
+int orc_send_set(const int32_t *dims, int ndims, int algo, int c, int p, int k, uint8_t *set) {
+    orc_topo tp; int rc = topo_init(&tp, dims, ndims, algo);
+    if (rc) return rc;
+    if (c < 0 || c >= ndims || p < 0 || p >= tp.n || k < 0 || k >= tp.S) return ORC_BAD_ARG;
+    int sd[64], sx[64];
+    step_list(&tp, c, sd, sx);
+    send_set(&tp, sd, sx, p, k, set);
+    return ORC_OK;
+}
+
+/* bounds_out[0..n]: element index where block j of slice c starts (global indices). */
+int orc_block_bounds(int64_t E, int D, int n, int c, int64_t *bounds_out) {
+    if (E < 0 || D < 1 || n < 1 || c < 0 || c >= D) return ORC_BAD_ARG;
+    int64_t lo, hi; slice_bounds(E, D, c, &lo, &hi);
+    for (int j = 0; j <= n; ++j) bounds_out[j] = block_bound(lo, hi, n, j);
+    return ORC_OK;
+}
+
+/* Naive sequential binary32 sum over ranks u = 0..n-1, per column. */
+void orc_naive_sum_f32(int n, int64_t w, const float *in, float *out) {
+    for (int64_t e = 0; e < w; ++e) {
+        float acc = in[e];
+        for (int u = 1; u < n; ++u) acc = acc + in[(int64_t)u * w + e];
+        out[e] = acc;
+    }
+}
+
+/* ------------------------------------------------------------------ data path (Trivance) */
+
+typedef struct {
+    /* all optional (NULL allowed); each is an array of n int64, bytes per rank */
+    int64_t *sent_rs;       /* bytes sent in the Reduce-Scatter phase (or the single latency phase) */
+    int64_t *sent_ag;       /* bytes sent in the AllGather phase */
+    int64_t *reduced;       /* bytes entering the reducer (both messages + local partial) */
+} orc_counters;
+
+#define DEFINE_PATH(T, SUFFIX, ADD)                                                                        \
+/* Latency-optimal form (Sec. 4.2): each step every rank copies its whole current partial into a          \
+ * message for both peers; when both messages are in, it reduces (left + own) + right. */                 \
+static int latency_slice_##SUFFIX(const orc_topo *tp, const int *sdim, const int *sdist,                   \
+                                  int64_t w, int64_t c0, int64_t c1, const T *in, T *out,                  \
+                                  int max_steps, orc_counters *ctr) {                                      \
+    int n = tp->n; int64_t wc = c1 - c0;                                                                   \
+    if (wc <= 0) return ORC_OK;                                                                            \
+    T *partial = (T *)malloc(sizeof(T) * (size_t)n * (size_t)wc);                                          \
+    T *message = (T *)malloc(sizeof(T) * (size_t)n * (size_t)wc);                                          \
+    if (!partial || !message) { free(partial); free(message); return ORC_NOMEM; }                          \
+    for (int r = 0; r < n; ++r) memcpy(partial + (size_t)r * wc, in + (size_t)r * w + c0, sizeof(T) * wc); \
+    int steps = (max_steps >= 0 && max_steps < tp->S) ? max_steps : tp->S;                                 \
+    for (int t = 0; t < steps; ++t) {                                                                      \
+        /* every rank builds its outgoing message first ... */                                            \
+        memcpy(message, partial, sizeof(T) * (size_t)n * (size_t)wc);                                      \
+        /* ... then every rank, having received both, reduces */                                          \
+        for (int p = 0; p < n; ++p) {                                                                      \
+            const T *from_left  = message + (size_t)shift_rank(tp, p, sdim[t], -sdist[t]) * wc;            \
+            const T *from_right = message + (size_t)shift_rank(tp, p, sdim[t], +sdist[t]) * wc;            \
+            T *own = partial + (size_t)p * wc;                                                             \
+            for (int64_t e = 0; e < wc; ++e) own[e] = ADD(ADD(from_left[e], own[e]), from_right[e]);       \
+            if (ctr && ctr->sent_rs) ctr->sent_rs[p] += 2 * (int64_t)sizeof(T) * wc;                       \
+            if (ctr && ctr->reduced) ctr->reduced[p] += 3 * (int64_t)sizeof(T) * wc;                       \
+        }                                                                                                  \
+    }                                                                                                      \
+    for (int r = 0; r < n; ++r) memcpy(out + (size_t)r * w + c0, partial + (size_t)r * wc, sizeof(T) * wc);\
+    free(partial); free(message);                                                                          \
+    return ORC_OK;                                                                                         \
+}                                                                                                          \
+                                                                                                           \
+/* Bandwidth-optimal form (Sec. 4.1, 4.3): Reduce-Scatter with Algorithm-1 block sets and literal         \
+ * messages, then AllGather with the steps in reverse order. */                                           \
+static int bandwidth_slice_##SUFFIX(const orc_topo *tp, const int *sdim, const int *sdist,                 \
+                                    int64_t slo, int64_t shi, int64_t e0, int64_t e1, int64_t w,           \
+                                    const T *in, T *out, orc_counters *ctr) {                              \
+    int n = tp->n, S = tp->S, rc = ORC_OK;                                                                 \
+    int64_t c0 = clampi(slo, e0, e1) - e0, c1 = clampi(shi, e0, e1) - e0, wc = c1 - c0;                    \
+    if (wc <= 0) return ORC_OK;                                                                            \
+    /* block j restricted to the window, as columns of the slice-local arrays */                          \
+    int64_t *bs = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n + 1));                                    \
+    T *partial = (T *)malloc(sizeof(T) * (size_t)n * (size_t)wc);                                          \
+    T *msg = (T *)malloc(sizeof(T) * (size_t)n * 2 * (size_t)wc);   /* [rank][side][<=wc] */               \
+    int64_t *mlen = (int64_t *)malloc(sizeof(int64_t) * (size_t)n * 2);                                    \
+    uint8_t *mset = (uint8_t *)malloc((size_t)n * 2 * (size_t)n);   /* block set of each message */        \
+    uint8_t *have = (uint8_t *)calloc((size_t)n, (size_t)n);        /* finished blocks held */             \
+    uint8_t *snap = (uint8_t *)malloc((size_t)n * (size_t)n);                                              \
+    if (!bs || !partial || !msg || !mlen || !mset || !have || !snap) { rc = ORC_NOMEM; goto done; }        \
+    for (int j = 0; j <= n; ++j) bs[j] = clampi(block_bound(slo, shi, n, j), e0, e1) - e0 - c0;            \
+    for (int r = 0; r < n; ++r) memcpy(partial + (size_t)r * wc, in + (size_t)r * w + c0, sizeof(T) * wc); \
+    /* ---- Reduce-Scatter */                                                                             \
+    for (int t = 0; t < S; ++t) {                                                                          \
+        for (int r = 0; r < n; ++r) {                                                                      \
+            int peer[2], dir[2], hops[2];                                                                  \
+            send_peers(tp, r, sdim[t], sdist[t], peer, dir, hops);                                         \
+            for (int side = 0; side < 2; ++side) {                                                         \
+                uint8_t *set = mset + ((size_t)r * 2 + side) * n;                                          \
+                T *m = msg + ((size_t)r * 2 + side) * wc; int64_t len = 0;                                 \
+                send_set(tp, sdim, sdist, peer[side], t, set);                                             \
+                for (int j = 0; j < n; ++j) if (set[j]) {                                                  \
+                    memcpy(m + len, partial + (size_t)r * wc + bs[j], sizeof(T) * (size_t)(bs[j+1]-bs[j]));\
+                    len += bs[j + 1] - bs[j];                                                              \
+                }                                                                                          \
+                mlen[(size_t)r * 2 + side] = len;                                                          \
+                if (ctr && ctr->sent_rs) ctr->sent_rs[r] += (int64_t)sizeof(T) * len;                      \
+            }                                                                                              \
+        }                                                                                                  \
+        for (int p = 0; p < n; ++p) {                                                                      \
+            int ql = shift_rank(tp, p, sdim[t], -sdist[t]);   /* left peer: its message to ITS right */   \
+            int qr = shift_rank(tp, p, sdim[t], +sdist[t]);   /* right peer: its message to ITS left */   \
+            const uint8_t *setl = mset + ((size_t)ql * 2 + 1) * n, *setr = mset + ((size_t)qr * 2 + 0) * n;\
+            const T *ml = msg + ((size_t)ql * 2 + 1) * wc, *mr = msg + ((size_t)qr * 2 + 0) * wc;          \
+            int64_t off = 0;                                                                               \
+            if (memcmp(setl, setr, (size_t)n)) { rc = ORC_INTERNAL; goto done; }                           \
+            for (int j = 0; j < n; ++j) if (setl[j]) {                                                     \
+                T *own = partial + (size_t)p * wc + bs[j]; int64_t bl = bs[j + 1] - bs[j];                 \
+                for (int64_t e = 0; e < bl; ++e) own[e] = ADD(ADD(ml[off + e], own[e]), mr[off + e]);      \
+                off += bl;                                                                                 \
+            }                                                                                              \
+            if (off != mlen[(size_t)ql * 2 + 1] || off != mlen[(size_t)qr * 2]) { rc = ORC_INTERNAL; goto done; } \
+            if (ctr && ctr->reduced) ctr->reduced[p] += 3 * (int64_t)sizeof(T) * off;                      \
+        }                                                                                                  \
+    }                                                                                                      \
+    /* ---- AllGather: reverse step order, every rank forwards all finished blocks it holds */            \
+    for (int r = 0; r < n; ++r) have[(size_t)r * n + r] = 1;                                               \
+    for (int t = S - 1; t >= 0; --t) {                                                                     \
+        memcpy(snap, have, (size_t)n * (size_t)n);                                                         \
+        for (int r = 0; r < n; ++r) {                                                                      \
+            T *m = msg + (size_t)r * 2 * wc; int64_t len = 0;       /* same message to both peers */       \
+            for (int j = 0; j < n; ++j) if (snap[(size_t)r * n + j]) {                                     \
+                memcpy(m + len, partial + (size_t)r * wc + bs[j], sizeof(T) * (size_t)(bs[j+1]-bs[j]));    \
+                len += bs[j + 1] - bs[j];                                                                  \
+            }                                                                                              \
+            if (ctr && ctr->sent_ag) ctr->sent_ag[r] += 2 * (int64_t)sizeof(T) * len;                      \
+        }                                                                                                  \
+        for (int p = 0; p < n; ++p) {                                                                      \
+            for (int side = 0; side < 2; ++side) {                                                         \
+                int q = shift_rank(tp, p, sdim[t], side ? +sdist[t] : -sdist[t]);                          \
+                const T *m = msg + (size_t)q * 2 * wc; int64_t off = 0;                                    \
+                for (int j = 0; j < n; ++j) if (snap[(size_t)q * n + j]) {                                 \
+                    int64_t bl = bs[j + 1] - bs[j];                                                        \
+                    if (have[(size_t)p * n + j]) { rc = ORC_INTERNAL; goto done; }  /* never twice */      \
+                    memcpy(partial + (size_t)p * wc + bs[j], m + off, sizeof(T) * (size_t)bl);             \
+                    have[(size_t)p * n + j] = 1; off += bl;                                                \
+                }                                                                                          \
+            }                                                                                              \
+        }                                                                                                  \
+    }                                                                                                      \
+    for (size_t i = 0; i < (size_t)n * (size_t)n; ++i) if (!have[i]) { rc = ORC_INTERNAL; goto done; }     \
+    for (int r = 0; r < n; ++r) memcpy(out + (size_t)r * w + c0, partial + (size_t)r * wc, sizeof(T) * wc);\
+done:                                                                                                      \
+    free(bs); free(partial); free(msg); free(mlen); free(mset); free(have); free(snap);                    \
+    return rc;                                                                                             \
+}
+
+#define ADD_WRAP(a, b) ((uint32_t)((a) + (b)))
+#define ADD_FP(a, b) ((a) + (b))
+DEFINE_PATH(uint32_t, i32, ADD_WRAP)
+DEFINE_PATH(float, f32, ADD_FP)
+DEFINE_PATH(double, f64, ADD_FP)
+
+/*
+ * Trivance AllReduce over the window [e0,e1) of per-rank vectors of E elements.
+ *   in, out : [n][w] row-major, w = e1-e0 (out may not alias in)
+ *   variant : ORC_LATENCY or ORC_BANDWIDTH
+ *   max_steps: latency form only: stop after this many steps (<0 = run all); lets
+ *              tests look at the partials after step k.
+ *   sent_rs/sent_ag/reduced: optional [n] int64 byte counters (accumulated into).
+ */
+int orc_allreduce(const int32_t *dims, int ndims, int variant, int dtype,
+                  int64_t E, int64_t e0, int64_t e1, const void *in, void *out, int max_steps,
+                  int64_t *sent_rs, int64_t *sent_ag, int64_t *reduced) {
+    orc_topo tp; int rc = topo_init(&tp, dims, ndims, ORC_TRIVANCE);
+    if (rc) return rc;
+    if (E < 0 || e0 < 0 || e1 < e0 || e1 > E || !in || !out) return ORC_BAD_ARG;
+    if (variant != ORC_LATENCY && variant != ORC_BANDWIDTH) return ORC_BAD_ARG;
+    if (dtype != ORC_I32 && dtype != ORC_F32 && dtype != ORC_F64) return ORC_BAD_ARG;
+    orc_counters ctr = { sent_rs, sent_ag, reduced };
+    int64_t w = e1 - e0;
+    for (int c = 0; c < tp.ndims; ++c) {
+        int sd[64], sx[64];
+        int64_t slo, shi;
+        step_list(&tp, c, sd, sx);
+        slice_bounds(E, tp.ndims, c, &slo, &shi);
+        int64_t c0 = clampi(slo, e0, e1) - e0, c1 = clampi(shi, e0, e1) - e0;
+        if (variant == ORC_LATENCY) {
+            if (dtype == ORC_I32) rc = latency_slice_i32(&tp, sd, sx, w, c0, c1, (const uint32_t *)in, (uint32_t *)out, max_steps, &ctr);
+            else if (dtype == ORC_F32) rc = latency_slice_f32(&tp, sd, sx, w, c0, c1, (const float *)in, (float *)out, max_steps, &ctr);
+            else rc = latency_slice_f64(&tp, sd, sx, w, c0, c1, (const double *)in, (double *)out, max_steps, &ctr);
+        } else {
+            if (dtype == ORC_I32) rc = bandwidth_slice_i32(&tp, sd, sx, slo, shi, e0, e1, w, (const uint32_t *)in, (uint32_t *)out, &ctr);
+            else if (dtype == ORC_F32) rc = bandwidth_slice_f32(&tp, sd, sx, slo, shi, e0, e1, w, (const float *)in, (float *)out, &ctr);
+            else rc = bandwidth_slice_f64(&tp, sd, sx, slo, shi, e0, e1, w, (const double *)in, (double *)out, &ctr);
+        }
+        if (rc) return rc;
+    }
+    return ORC_OK;
+}
+
+/* ------------------------------------------------------------------ link loads */
+
+/*
+ * Per-step, per-directed-link load (Sec. 2.1: c_k; Fig. 1; App. E routing).
+ * Rows: T = S (latency form) or 2S (bandwidth form: Reduce-Scatter steps 0..S-1,
+ * then the AllGather steps, which mirror S-1..0).
+ * msgs/bytes are [T][n][D][2]: link leaving `node` along dimension `dim`,
+ * direction index 0 = towards +, 1 = towards -.  Every message walks hop by hop
+ * from its source in its direction of travel.  A message's bytes are the real
+ * (possibly uneven) lengths of the blocks it carries times elem_size.
+ * All four outputs are optional.
+ */
+int orc_link_loads(const int32_t *dims, int ndims, int variant, int algo, int64_t E, int64_t elem_size,
+                   int32_t *msgs, int64_t *bytes, int32_t *max_msgs, int64_t *max_bytes) {
+    orc_topo tp; int rc = topo_init(&tp, dims, ndims, algo);
+    if (rc) return rc;
+    if (E < 0 || elem_size < 1) return ORC_BAD_ARG;
+    if (variant != ORC_LATENCY && variant != ORC_BANDWIDTH) return ORC_BAD_ARG;
+    int n = tp.n, D = tp.ndims, S = tp.S, T = (variant == ORC_BANDWIDTH) ? 2 * S : S;
+    size_t links = (size_t)n * D * 2;
+    int32_t *lm = (int32_t *)calloc((size_t)T * links, sizeof(int32_t));
+    int64_t *lb = (int64_t *)calloc((size_t)T * links, sizeof(int64_t));
+    uint8_t *set = (uint8_t *)malloc((size_t)n);
+    uint8_t *have = (uint8_t *)malloc((size_t)n * n), *snap = (uint8_t *)malloc((size_t)n * n);
+    int64_t *blen = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);
+    if (!lm || !lb || !set || !have || !snap || !blen) { rc = ORC_NOMEM; goto done; }
+
+    for (int c = 0; c < D; ++c) {
+        int sd[64], sx[64];
+        int64_t slo, shi;
+        step_list(&tp, c, sd, sx);
+        slice_bounds(E, D, c, &slo, &shi);
+        for (int j = 0; j < n; ++j) blen[j] = block_bound(slo, shi, n, j + 1) - block_bound(slo, shi, n, j);
+        memset(have, 0, (size_t)n * n);
+        for (int r = 0; r < n; ++r) have[(size_t)r * n + r] = 1;
+        for (int row = 0; row < T; ++row) {
+            int t = (row < S) ? row : (2 * S - 1 - row);      /* AllGather mirrors */
+            int d = sd[t], dist = sx[t];
+            if (row >= S) memcpy(snap, have, (size_t)n * n);
+            for (int r = 0; r < n; ++r) {
+                int peer[2], dir[2], hops[2];
+                int np = send_peers(&tp, r, d, dist, peer, dir, hops);
+                for (int i = 0; i < np; ++i) {
+                    int64_t mbytes = 0;
+                    if (variant == ORC_LATENCY) {
+                        mbytes = (shi - slo) * elem_size;
+                    } else if (row < S) {
+                        send_set(&tp, sd, sx, peer[i], t, set);
+                        for (int j = 0; j < n; ++j) if (set[j]) mbytes += blen[j] * elem_size;
+                    } else {
+                        for (int j = 0; j < n; ++j) if (snap[(size_t)r * n + j]) {
+                            mbytes += blen[j] * elem_size;
+                            have[(size_t)peer[i] * n + j] = 1;
+                        }
+                    }
+                    int cur = r;
+                    for (int h = 0; h < hops[i]; ++h) {
+                        size_t li = (((size_t)row * n + cur) * D + d) * 2 + (dir[i] > 0 ? 0 : 1);
+                        lm[li] += 1; lb[li] += mbytes;
+                        cur = shift_rank(&tp, cur, d, dir[i]);
+                    }
+                    if (cur != peer[i]) { rc = ORC_INTERNAL; goto done; }
+                }
+            }
+        }
+    }
+    for (int row = 0; row < T; ++row) {
+        int32_t mm = 0; int64_t mb = 0;
+        for (size_t l = 0; l < links; ++l) {
+            if (lm[(size_t)row * links + l] > mm) mm = lm[(size_t)row * links + l];
+            if (lb[(size_t)row * links + l] > mb) mb = lb[(size_t)row * links + l];
+        }
+        if (max_msgs) max_msgs[row] = mm;
+        if (max_bytes) max_bytes[row] = mb;
+    }
+    if (msgs) memcpy(msgs, lm, sizeof(int32_t) * (size_t)T * links);
+    if (bytes) memcpy(bytes, lb, sizeof(int64_t) * (size_t)T * links);
+done:
+    free(lm); free(lb); free(set); free(have); free(snap); free(blen);
+    return rc;
+}
