@@ -1,0 +1,193 @@
+/*
+ * trivance.h -- C ABI of the B200 Trivance AllReduce engine.
+ *
+ * The engine executes the Trivance AllReduce schedule (Juerss, Addanki, Schmid:
+ * "Trivance: Latency-Optimal AllReduce by Shortcutting Multiport Networks") over n
+ * SIMULATED ranks whose buffers all live in one GPU's memory.  Nothing moves between
+ * GPUs.  All entry points are plain C: pointers (each documented as HOST or DEVICE)
+ * and sizes.  No entry point throws, aborts or synchronises the device unless it says
+ * so.  Every function returns a trv_status_t; argument errors are found on the host
+ * before anything is launched.
+ *
+ * Notation (paper): n ranks on a D-dimensional torus with sides a_0..a_{D-1}, every side
+ * a power of three; rank r = x_0 + a_0 x_1 + a_0 a_1 x_2 + ...; S = sum_d log3 a_d steps
+ * per phase; every rank owns a vector of `count` 4-byte elements.
+ */
+#ifndef TRIVANCE_H_
+#define TRIVANCE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct trv_plan_s *trv_plan_t;          /* opaque; owned by the library */
+
+typedef enum {
+    TRV_OK = 0,
+    TRV_ERR_INVALID_ARG = 1,        /* NULL pointer, bad enum, misaligned or aliasing buffers ... */
+    TRV_ERR_UNSUPPORTED = 2,        /* a side that is not a power of three, too many ranks, op != sum */
+    TRV_ERR_UNDEFINED_SCHEDULE = 3, /* the schedule does not exist for this n (Recursive Doubling, n != 2^q) */
+    TRV_ERR_ALLOC = 4,
+    TRV_ERR_CUDA = 5,               /* a CUDA runtime call failed; cudaGetLastError has the reason */
+    TRV_ERR_SCRATCH = 6             /* caller-provided scratch/workspace too small or misaligned */
+} trv_status_t;
+
+typedef enum { TRV_LATENCY_OPTIMAL = 0, TRV_BANDWIDTH_OPTIMAL = 1 } trv_variant_t;
+typedef enum { TRV_ALGO_TRIVANCE = 0, TRV_ALGO_BRUCK = 1, TRV_ALGO_RECDOUB = 2 } trv_algo_t;
+typedef enum { TRV_INT32 = 0, TRV_FLOAT32 = 1 } trv_dtype_t;
+typedef enum { TRV_SUM = 0 } trv_op_t;
+
+/* Which kernel family executes the schedule.
+ *   STEP : one launch per schedule step, exactly as the paper states the steps (latency form:
+ *          ping-pong through scratch; bandwidth form: block-indexed three-input Reduce-Scatter
+ *          steps and AllGather copy steps, in place).
+ *   FUSED: all steps of a column of elements on chip; one read and one write per element.
+ *          Exists for the shapes trv_kernel_supported() reports.
+ *   AUTO : FUSED where it exists, else STEP.
+ * Both families give bit-identical results. */
+typedef enum { TRV_KERNEL_AUTO = 0, TRV_KERNEL_STEP = 1, TRV_KERNEL_FUSED = 2 } trv_kernel_t;
+
+#define TRV_MAX_DIMS 8
+#define TRV_MAX_RANKS 1024
+
+/* ---------------------------------------------------------------- plan (schedule builder)
+ *
+ * trv_plan_create builds the Trivance schedule for a torus with the given sides:
+ * peers pi(r,k,n) = (r - 3^k, r + 3^k) mod n (Sec. 4.1); for D > 1 one collective per
+ * dimension on 1/D of the vector, collective c using in step t the next dimension, in
+ * round-robin order starting at c, that still has steps left (Sec. 5).
+ *   dims  : HOST array of ndims sides (1 <= ndims <= TRV_MAX_DIMS), each 3^k, k >= 1
+ *   out   : receives the plan; release with trv_plan_destroy
+ * Host-only integer work; makes no CUDA call.  A plan is immutable: it may be used from
+ * several threads and streams at once.
+ * Errors: INVALID_ARG (NULL, ndims out of range, side < 2), UNSUPPORTED (side not a power
+ * of three, more than TRV_MAX_RANKS ranks). */
+trv_status_t trv_plan_create(const int32_t *dims, int32_t ndims, trv_variant_t variant, trv_plan_t *out);
+
+/* Same, for a comparator schedule (Sec. 2.4, Fig. 1).  TRV_ALGO_BRUCK: peers r + 3^k and
+ * r + 2*3^k, both sent in the + direction.  TRV_ALGO_RECDOUB: peer r XOR 2^k on a ring of
+ * 2^q ranks (ndims must be 1), the lower rank of a pair sending in the + direction;
+ * UNDEFINED_SCHEDULE for other ring sizes.  Comparator plans serve trv_link_loads and the
+ * schedule queries only; trv_allreduce returns UNSUPPORTED for them. */
+trv_status_t trv_plan_create_algo(const int32_t *dims, int32_t ndims, trv_variant_t variant, trv_algo_t algo,
+                                  trv_plan_t *out);
+
+trv_status_t trv_plan_destroy(trv_plan_t plan);
+
+/* n = number of ranks; rows = schedule rows = S for the latency form (Sec. 4.2), 2S for the
+ * bandwidth form (Reduce-Scatter steps 0..S-1, then the AllGather steps, which mirror
+ * S-1..0, Sec. 4.1).  Any output may be NULL. */
+trv_status_t trv_plan_info(trv_plan_t plan, int32_t *n, int32_t *ndims, int32_t *rows);
+
+/* Row `row` of collective (slice) c: the dimension it runs along and the ring distance. */
+trv_status_t trv_plan_step(trv_plan_t plan, int32_t c, int32_t row, int32_t *dim, int32_t *dist);
+
+/* peers: HOST array [n][2]; the ranks each rank sends to in that row (Trivance: left = minus
+ * distance, right = plus distance; Recursive Doubling: second entry -1). */
+trv_status_t trv_plan_peers(trv_plan_t plan, int32_t c, int32_t row, int32_t *peers);
+
+/* set: HOST array of n bytes; set[j] = 1 iff block j is part of the message sent to rank
+ * `dst` in Reduce-Scatter step `step` of collective c (closed form Pi of Sec. 4.3: the
+ * blocks that agree with dst modulo 3^(visits so far) in every dimension). */
+trv_status_t trv_plan_send_set(trv_plan_t plan, int32_t c, int32_t step, int32_t dst, uint8_t *set);
+
+/* bounds: HOST array of n+1 global element indices: block j of collective c covers
+ * [bounds[j], bounds[j+1]).  Slice c = [floor(c*count/D), floor((c+1)*count/D)), block j of a
+ * slice [lo,hi) = [lo + floor(j*(hi-lo)/n), lo + floor((j+1)*(hi-lo)/n)) (Sec. 4.1, Sec. 5). */
+trv_status_t trv_plan_block_bounds(trv_plan_t plan, size_t count, int32_t c, int64_t *bounds);
+
+/* ---------------------------------------------------------------- AllReduce
+ *
+ * In-place AllReduce (Sec. 2.2): on return of the work queued on `cuda_stream`, every
+ * rank_buffers[r] holds, element-wise, the sum of all n input vectors, associated in the
+ * order the schedule defines: each joint reduction is (from_left + own) + from_right
+ * (Sec. 3.1, 4.2).  In the latency form the n results differ in rounding for float32
+ * (each rank has its own reduction tree); in the bandwidth form all n are identical.
+ *   rank_buffers: HOST array of n DEVICE pointers, each >= count*4 bytes, 16-byte aligned,
+ *                 pairwise disjoint; caller-owned, never freed here
+ *   count       : elements per rank (0 is allowed: nothing happens)
+ *   dtype       : TRV_INT32 adds modulo 2^32; TRV_FLOAT32 is IEEE binary32, round to
+ *                 nearest even, no flush to zero
+ *   op          : TRV_SUM only
+ *   cuda_stream : a cudaStream_t (NULL = the legacy default stream)
+ * Asynchronous; never synchronises.  If the chosen kernel family needs scratch memory (the
+ * STEP family of the latency form does), the plan allocates it with cudaMalloc on first
+ * need, keeps it, and frees it in trv_plan_destroy; such calls on ONE plan must then not
+ * overlap on the device.  Use trv_allreduce_ex to pass your own scratch instead. */
+trv_status_t trv_allreduce(trv_plan_t plan, void *const *rank_buffers, size_t count, trv_dtype_t dtype, trv_op_t op,
+                           void *cuda_stream);
+
+/* Bytes of scratch trv_allreduce_ex needs for this call shape (0 if none). */
+trv_status_t trv_scratch_bytes(trv_plan_t plan, size_t count, trv_kernel_t kernel, int32_t in_place, size_t *bytes);
+
+/* 1 if the FUSED family exists for this plan, else 0. */
+int32_t trv_kernel_supported(trv_plan_t plan, trv_kernel_t kernel);
+
+/* General form.
+ *   in_buffers / out_buffers: HOST arrays of n DEVICE pointers (rules as above).  They may be
+ *                 the same array (in place); otherwise no input may overlap any output.
+ *   count       : elements per rank held in these buffers
+ *   global_count, global_offset: the buffers hold elements [global_offset, global_offset +
+ *                 count) of per-rank vectors of global_count elements; slice and block
+ *                 membership follow the GLOBAL element index.  This is how a vector is
+ *                 sharded by element range over several GPUs without any exchange
+ *                 (columns are independent).  Pass count and 0 for an unsharded call.
+ *   kernel      : kernel family (see trv_kernel_t)
+ *   scratch     : DEVICE pointer, 256-byte aligned, scratch_bytes >= trv_scratch_bytes(...);
+ *                 may be NULL when 0 bytes are needed.  Contents are undefined afterwards.
+ * Errors: as trv_allreduce, plus SCRATCH. */
+trv_status_t trv_allreduce_ex(trv_plan_t plan, const void *const *in_buffers, void *const *out_buffers, size_t count,
+                              size_t global_count, size_t global_offset, trv_dtype_t dtype, trv_op_t op,
+                              trv_kernel_t kernel, void *scratch, size_t scratch_bytes, void *cuda_stream);
+
+/* AllReduce of HOST vectors: copies the n host vectors into `workspace`, runs the AllReduce
+ * there and copies the n results back, all queued on `cuda_stream`; returns without
+ * synchronising (the host buffers must stay valid, and should be pinned, until the stream
+ * reaches the end of this work).
+ *   host_in / host_out: HOST arrays of n HOST pointers to count*4 bytes each (may be equal)
+ *   workspace   : DEVICE pointer, 256-byte aligned, >= trv_host_workspace_bytes(...) bytes */
+trv_status_t trv_allreduce_host(trv_plan_t plan, const void *const *host_in, void *const *host_out, size_t count,
+                                trv_dtype_t dtype, trv_op_t op, void *workspace, size_t workspace_bytes,
+                                void *cuda_stream);
+trv_status_t trv_host_workspace_bytes(trv_plan_t plan, size_t count, size_t *bytes);
+
+/* ---------------------------------------------------------------- link loads
+ *
+ * Per-step, per-directed-link load of the plan's schedule (Sec. 2.1: c_k = number of
+ * messages sharing a link in step k; Fig. 1; App. E: deterministic shortest-path routing
+ * inside one dimension).  Tallied on the GPU; synchronous (uses the legacy default stream,
+ * allocates and frees a few small device buffers).
+ *   count, elem_size: per-rank vector length and bytes per element (message bytes use the
+ *                 real, possibly uneven, block lengths)
+ *   msgs      : HOST int32 [rows][n][D][2]; link leaving `node` along `dim`, index 0 = towards
+ *               +, 1 = towards -; number of messages crossing it in that row
+ *   bytes     : HOST int64, same shape; bytes crossing it
+ *   max_msgs  : HOST int32 [rows]; max over links    max_bytes: HOST int64 [rows]
+ * Any output may be NULL. */
+trv_status_t trv_link_loads(trv_plan_t plan, size_t count, size_t elem_size, int32_t *msgs, int64_t *bytes,
+                            int32_t *max_msgs, int64_t *max_bytes);
+
+/* bytes: HOST int64 [n].  Row < S (Reduce-Scatter or latency form): bytes of the message a
+ * rank RECEIVES from each sender in that row, indexed by destination.  Row >= S (AllGather):
+ * bytes of the message a rank SENDS to each of its peers, indexed by source.  Host-only. */
+trv_status_t trv_plan_message_bytes(trv_plan_t plan, size_t count, size_t elem_size, int32_t c, int32_t row,
+                                    int64_t *bytes);
+
+/* ---------------------------------------------------------------- misc */
+
+const char *trv_strerror(trv_status_t status);
+
+/* Number of kernels this library has launched in this process so far. */
+uint64_t trv_launch_count(void);
+
+/* Name of the kernel family member the last trv_allreduce* call of this thread used
+ * (static string, e.g. "lat_reg<27>", "step"); for reports. */
+const char *trv_last_kernel_name(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TRIVANCE_H_ */

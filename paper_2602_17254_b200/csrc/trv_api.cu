@@ -1,0 +1,269 @@
+// C ABI of the Trivance engine: argument checks, kernel-family choice, host-buffer variant.
+#include <algorithm>
+#include <cstring>
+#include <vector>
+
+#include "trv_dev.cuh"
+
+namespace trv {
+std::atomic<uint64_t> g_launches{0};
+thread_local const char* g_last_kernel = "none";
+
+static bool fused_supported(const Plan& p) {
+    return p.variant == TRV_LATENCY_OPTIMAL ? fused_latency_supported(p) : fused_bandwidth_supported(p);
+}
+
+static trv_status_t check_buffers(const Plan& p, const void* const* in, void* const* out, size_t count, bool* in_place) {
+    if (!in || !out) return TRV_ERR_INVALID_ARG;
+    const int n = p.n;
+    bool same = true;
+    for (int r = 0; r < n; ++r) {
+        if (!in[r] || !out[r]) return TRV_ERR_INVALID_ARG;
+        if (((uintptr_t)in[r] | (uintptr_t)out[r]) & 15) return TRV_ERR_INVALID_ARG;
+        if (in[r] != out[r]) same = false;
+    }
+    // pairwise disjoint outputs; inputs either identical to the outputs or disjoint from all of them
+    const size_t bytes = count * 4;
+    std::vector<std::pair<uintptr_t, int>> iv;
+    iv.reserve(2 * (size_t)n);
+    for (int r = 0; r < n; ++r) iv.emplace_back((uintptr_t)out[r], 1);
+    if (!same)
+        for (int r = 0; r < n; ++r) iv.emplace_back((uintptr_t)in[r], 0);
+    std::sort(iv.begin(), iv.end());
+    for (size_t i = 1; i < iv.size(); ++i) {
+        if (iv[i - 1].first + bytes > iv[i].first) {
+            // two inputs may coincide or overlap each other (reading is harmless); anything
+            // touching an output may not
+            if (iv[i - 1].second == 0 && iv[i].second == 0) continue;
+            return TRV_ERR_INVALID_ARG;
+        }
+    }
+    *in_place = same;
+    return TRV_OK;
+}
+
+static trv_status_t dispatch(Call& c, trv_kernel_t kernel) {
+    const Plan& p = *c.plan;
+    bool fused = false;
+    if (kernel == TRV_KERNEL_FUSED) {
+        if (!fused_supported(p)) return TRV_ERR_UNSUPPORTED;
+        fused = true;
+    } else if (kernel == TRV_KERNEL_AUTO) {
+        fused = fused_supported(p);
+    }
+    if (p.variant == TRV_LATENCY_OPTIMAL) return fused ? run_fused_latency(c) : run_step_latency(c);
+    return fused ? run_fused_bandwidth(c) : run_step_bandwidth(c);
+}
+}  // namespace trv
+
+using namespace trv;
+
+extern "C" {
+
+trv_status_t trv_plan_create(const int32_t* dims, int32_t ndims, trv_variant_t variant, trv_plan_t* out) {
+    return trv_plan_create_algo(dims, ndims, variant, TRV_ALGO_TRIVANCE, out);
+}
+
+trv_status_t trv_plan_create_algo(const int32_t* dims, int32_t ndims, trv_variant_t variant, trv_algo_t algo,
+                                  trv_plan_t* out) {
+    if (!out) return TRV_ERR_INVALID_ARG;
+    *out = nullptr;
+    return build_plan(dims, ndims, (int)variant, (int)algo, out);
+}
+
+trv_status_t trv_plan_destroy(trv_plan_t plan) {
+    if (!plan) return TRV_ERR_INVALID_ARG;
+    trv_status_t st = TRV_OK;
+    if (plan->plan.scratch && cudaFree(plan->plan.scratch) != cudaSuccess) st = TRV_ERR_CUDA;
+    delete plan;
+    return st;
+}
+
+trv_status_t trv_plan_info(trv_plan_t plan, int32_t* n, int32_t* ndims, int32_t* rows) {
+    if (!plan) return TRV_ERR_INVALID_ARG;
+    if (n) *n = plan->plan.n;
+    if (ndims) *ndims = plan->plan.ndims;
+    if (rows) *rows = plan->plan.rows();
+    return TRV_OK;
+}
+
+trv_status_t trv_plan_step(trv_plan_t plan, int32_t c, int32_t row, int32_t* dim, int32_t* dist) {
+    if (!plan) return TRV_ERR_INVALID_ARG;
+    const Plan& p = plan->plan;
+    if (c < 0 || c >= p.ndims || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
+    const Step& s = p.steps[c][p.step_of_row(row)];
+    if (dim) *dim = s.dim;
+    if (dist) *dist = s.dist;
+    return TRV_OK;
+}
+
+trv_status_t trv_plan_peers(trv_plan_t plan, int32_t c, int32_t row, int32_t* peers) {
+    if (!plan || !peers) return TRV_ERR_INVALID_ARG;
+    const Plan& p = plan->plan;
+    if (c < 0 || c >= p.ndims || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
+    const Step& s = p.steps[c][p.step_of_row(row)];
+    for (int r = 0; r < p.n; ++r) {
+        int peer[2], dir[2], hops[2];
+        send_peers(p, r, s.dim, s.dist, peer, dir, hops);
+        peers[2 * r] = peer[0];
+        peers[2 * r + 1] = peer[1];
+    }
+    return TRV_OK;
+}
+
+trv_status_t trv_plan_send_set(trv_plan_t plan, int32_t c, int32_t step, int32_t dst, uint8_t* set) {
+    if (!plan || !set) return TRV_ERR_INVALID_ARG;
+    const Plan& p = plan->plan;
+    if (c < 0 || c >= p.ndims || step < 0 || step >= p.S || dst < 0 || dst >= p.n) return TRV_ERR_INVALID_ARG;
+    for (int j = 0; j < p.n; ++j) set[j] = in_send_set(p, c, step, dst, j) ? 1 : 0;
+    return TRV_OK;
+}
+
+trv_status_t trv_plan_block_bounds(trv_plan_t plan, size_t count, int32_t c, int64_t* bounds) {
+    if (!plan || !bounds) return TRV_ERR_INVALID_ARG;
+    const Plan& p = plan->plan;
+    if (c < 0 || c >= p.ndims) return TRV_ERR_INVALID_ARG;
+    const int64_t lo = slice_lo((int64_t)count, p.ndims, c), hi = slice_lo((int64_t)count, p.ndims, c + 1);
+    for (int j = 0; j <= p.n; ++j) bounds[j] = block_lo(lo, hi, p.n, j);
+    return TRV_OK;
+}
+
+trv_status_t trv_plan_message_bytes(trv_plan_t plan, size_t count, size_t elem_size, int32_t c, int32_t row,
+                                    int64_t* bytes) {
+    if (!plan || !bytes || elem_size == 0) return TRV_ERR_INVALID_ARG;
+    const Plan& p = plan->plan;
+    if (c < 0 || c >= p.ndims || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
+    message_bytes(p, (int64_t)count, (int64_t)elem_size, c, row, bytes);
+    return TRV_OK;
+}
+
+int32_t trv_kernel_supported(trv_plan_t plan, trv_kernel_t kernel) {
+    if (!plan || plan->plan.algo != TRV_ALGO_TRIVANCE) return 0;
+    if (kernel == TRV_KERNEL_FUSED) return fused_supported(plan->plan) ? 1 : 0;
+    return (kernel == TRV_KERNEL_AUTO || kernel == TRV_KERNEL_STEP) ? 1 : 0;
+}
+
+trv_status_t trv_scratch_bytes(trv_plan_t plan, size_t count, trv_kernel_t kernel, int32_t in_place, size_t* bytes) {
+    if (!plan || !bytes) return TRV_ERR_INVALID_ARG;
+    const Plan& p = plan->plan;
+    if (p.algo != TRV_ALGO_TRIVANCE) return TRV_ERR_UNSUPPORTED;
+    bool fused = false;
+    if (kernel == TRV_KERNEL_FUSED) {
+        if (!fused_supported(p)) return TRV_ERR_UNSUPPORTED;
+        fused = true;
+    } else if (kernel == TRV_KERNEL_AUTO) {
+        fused = fused_supported(p);
+    } else if (kernel != TRV_KERNEL_STEP) {
+        return TRV_ERR_INVALID_ARG;
+    }
+    *bytes = fused ? 0 : step_scratch_bytes(p, count, in_place != 0);
+    return TRV_OK;
+}
+
+trv_status_t trv_allreduce_ex(trv_plan_t plan, const void* const* in_buffers, void* const* out_buffers, size_t count,
+                              size_t global_count, size_t global_offset, trv_dtype_t dtype, trv_op_t op,
+                              trv_kernel_t kernel, void* scratch, size_t scratch_bytes, void* cuda_stream) {
+    if (!plan) return TRV_ERR_INVALID_ARG;
+    const Plan& p = plan->plan;
+    if (p.algo != TRV_ALGO_TRIVANCE) return TRV_ERR_UNSUPPORTED;
+    if (dtype != TRV_INT32 && dtype != TRV_FLOAT32) return TRV_ERR_INVALID_ARG;
+    if (op != TRV_SUM) return TRV_ERR_UNSUPPORTED;
+    if (kernel != TRV_KERNEL_AUTO && kernel != TRV_KERNEL_STEP && kernel != TRV_KERNEL_FUSED) return TRV_ERR_INVALID_ARG;
+    if (global_offset > global_count || count > global_count - global_offset) return TRV_ERR_INVALID_ARG;
+    if (count >= ((size_t)1 << 40)) return TRV_ERR_UNSUPPORTED;
+    bool in_place = false;
+    trv_status_t st = check_buffers(p, in_buffers, out_buffers, count, &in_place);
+    if (st != TRV_OK) return st;
+    if (scratch_bytes && (!scratch || ((uintptr_t)scratch & 255))) return TRV_ERR_SCRATCH;
+    if (count == 0) return TRV_OK;
+    Call c{&p, in_buffers, out_buffers, count, global_count, global_offset, (int)dtype, in_place,
+           scratch, scratch_bytes, (cudaStream_t)cuda_stream};
+    return dispatch(c, kernel);
+}
+
+trv_status_t trv_allreduce(trv_plan_t plan, void* const* rank_buffers, size_t count, trv_dtype_t dtype, trv_op_t op,
+                           void* cuda_stream) {
+    if (!plan) return TRV_ERR_INVALID_ARG;
+    Plan& p = plan->plan;
+    size_t need = 0;
+    trv_status_t st = trv_scratch_bytes(plan, count, TRV_KERNEL_AUTO, 1, &need);
+    if (st != TRV_OK) return st;
+    if (need > p.scratch_bytes) {
+        // validate before allocating anything
+        bool ip;
+        if (dtype != TRV_INT32 && dtype != TRV_FLOAT32) return TRV_ERR_INVALID_ARG;
+        if (op != TRV_SUM) return TRV_ERR_UNSUPPORTED;
+        st = check_buffers(p, (const void* const*)rank_buffers, rank_buffers, count, &ip);
+        if (st != TRV_OK) return st;
+        if (p.scratch) { cudaFree(p.scratch); p.scratch = nullptr; p.scratch_bytes = 0; }
+        if (cudaMalloc(&p.scratch, need) != cudaSuccess) { (void)cudaGetLastError(); return TRV_ERR_ALLOC; }
+        p.scratch_bytes = need;
+    }
+    return trv_allreduce_ex(plan, (const void* const*)rank_buffers, rank_buffers, count, count, 0, dtype, op,
+                            TRV_KERNEL_AUTO, p.scratch, p.scratch_bytes, cuda_stream);
+}
+
+static size_t host_row_bytes(size_t count) { return ((count * 4) + 255) & ~(size_t)255; }
+
+trv_status_t trv_host_workspace_bytes(trv_plan_t plan, size_t count, size_t* bytes) {
+    if (!plan || !bytes) return TRV_ERR_INVALID_ARG;
+    size_t scratch = 0;
+    trv_status_t st = trv_scratch_bytes(plan, count, TRV_KERNEL_AUTO, 1, &scratch);
+    if (st != TRV_OK) return st;
+    *bytes = (size_t)plan->plan.n * host_row_bytes(count) + scratch;
+    return TRV_OK;
+}
+
+trv_status_t trv_allreduce_host(trv_plan_t plan, const void* const* host_in, void* const* host_out, size_t count,
+                                trv_dtype_t dtype, trv_op_t op, void* workspace, size_t workspace_bytes,
+                                void* cuda_stream) {
+    if (!plan || !host_in || !host_out) return TRV_ERR_INVALID_ARG;
+    const Plan& p = plan->plan;
+    if (p.algo != TRV_ALGO_TRIVANCE) return TRV_ERR_UNSUPPORTED;
+    size_t need = 0;
+    trv_status_t st = trv_host_workspace_bytes(plan, count, &need);
+    if (st != TRV_OK) return st;
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return TRV_ERR_SCRATCH;
+    for (int r = 0; r < p.n; ++r)
+        if (!host_in[r] || !host_out[r]) return TRV_ERR_INVALID_ARG;
+    if (count == 0) return TRV_OK;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const size_t row = host_row_bytes(count);
+    std::vector<void*> dev(p.n);
+    for (int r = 0; r < p.n; ++r) {
+        dev[r] = (char*)workspace + (size_t)r * row;
+        if (cudaMemcpyAsync(dev[r], host_in[r], count * 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return TRV_ERR_CUDA;
+    }
+    void* scratch = (char*)workspace + (size_t)p.n * row;
+    st = trv_allreduce_ex(plan, (const void* const*)dev.data(), dev.data(), count, count, 0, dtype, op, TRV_KERNEL_AUTO,
+                          need > (size_t)p.n * row ? scratch : nullptr, need - (size_t)p.n * row, s);
+    if (st != TRV_OK) return st;
+    for (int r = 0; r < p.n; ++r)
+        if (cudaMemcpyAsync(host_out[r], dev[r], count * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return TRV_ERR_CUDA;
+    return TRV_OK;
+}
+
+trv_status_t trv_link_loads(trv_plan_t plan, size_t count, size_t elem_size, int32_t* msgs, int64_t* bytes,
+                            int32_t* max_msgs, int64_t* max_bytes) {
+    if (!plan || elem_size == 0) return TRV_ERR_INVALID_ARG;
+    return run_link_loads(plan->plan, count, elem_size, msgs, bytes, max_msgs, max_bytes);
+}
+
+const char* trv_strerror(trv_status_t status) {
+    switch (status) {
+        case TRV_OK: return "ok";
+        case TRV_ERR_INVALID_ARG: return "invalid argument";
+        case TRV_ERR_UNSUPPORTED: return "unsupported (side not a power of three, too many ranks, or op/plan kind not executable)";
+        case TRV_ERR_UNDEFINED_SCHEDULE: return "schedule undefined for this number of ranks";
+        case TRV_ERR_ALLOC: return "allocation failed";
+        case TRV_ERR_CUDA: return "CUDA runtime error";
+        case TRV_ERR_SCRATCH: return "scratch or workspace too small or misaligned";
+    }
+    return "unknown status";
+}
+
+uint64_t trv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* trv_last_kernel_name(void) { return g_last_kernel; }
+
+}  // extern "C"

@@ -1,0 +1,85 @@
+// Shared device-side helpers and the internal call descriptor.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+
+#include "trv_plan.h"
+
+namespace trv {
+
+// Rank-pointer table passed BY VALUE in kernel parameter space (sm_100 allows 32 KB of
+// parameters): no device-side table to upload, so a call is a pure launch sequence.
+template <int CAP>
+struct PtrTab {
+    void* p[CAP];
+};
+
+struct Call {
+    const Plan* plan;
+    const void* const* in;      // host array of n device pointers
+    void* const* out;           // host array of n device pointers (may equal in)
+    size_t count;               // local elements per rank
+    size_t gcount, goff;        // global vector length and offset of local element 0
+    int dtype;
+    bool in_place;
+    void* scratch;
+    size_t scratch_bytes;
+    cudaStream_t st;
+};
+
+extern std::atomic<uint64_t> g_launches;
+extern thread_local const char* g_last_kernel;
+
+#define TRV_LAUNCH(kernel, grid, block, smem, stream, ...)                \
+    do {                                                                  \
+        kernel<<<(grid), (block), (smem), (stream)>>>(__VA_ARGS__);       \
+        ::trv::g_launches.fetch_add(1, std::memory_order_relaxed);        \
+    } while (0)
+
+// (a + b) + c, one rounding per add, never contracted or reassociated.
+__device__ __forceinline__ float add3(float a, float b, float c) { return __fadd_rn(__fadd_rn(a, b), c); }
+__device__ __forceinline__ uint32_t add3(uint32_t a, uint32_t b, uint32_t c) { return (a + b) + c; }
+__device__ __forceinline__ float add2(float a, float b) { return __fadd_rn(a, b); }
+__device__ __forceinline__ uint32_t add2(uint32_t a, uint32_t b) { return a + b; }
+
+template <typename T> struct Vec4;
+template <> struct Vec4<float> { using type = float4; };
+template <> struct Vec4<uint32_t> { using type = uint4; };
+
+template <typename V>
+__device__ __forceinline__ V add3v(const V& a, const V& b, const V& c) {
+    V r;
+    r.x = add3(a.x, b.x, c.x); r.y = add3(a.y, b.y, c.y);
+    r.z = add3(a.z, b.z, c.z); r.w = add3(a.w, b.w, c.w);
+    return r;
+}
+
+// step-family launchers (trv_step.cu)
+trv_status_t run_step_latency(const Call& c);
+trv_status_t run_step_bandwidth(const Call& c);
+size_t step_scratch_bytes(const Plan& p, size_t count, bool in_place);
+
+// fused-family launchers (trv_fused_lat.cu / trv_fused_bw.cu)
+bool fused_latency_supported(const Plan& p);
+bool fused_bandwidth_supported(const Plan& p);
+trv_status_t run_fused_latency(const Call& c);
+trv_status_t run_fused_bandwidth(const Call& c);
+
+// link-load tally (trv_linkloads.cu)
+trv_status_t run_link_loads(const Plan& p, size_t count, size_t elem_size, int32_t* msgs, int64_t* bytes,
+                            int32_t* max_msgs, int64_t* max_bytes);
+
+// local column range [lo,hi) of slice c inside the window the call holds
+inline void local_slice(const Call& c, int slice, long long* lo, long long* hi) {
+    const int D = c.plan->ndims;
+    long long glo = slice_lo((int64_t)c.gcount, D, slice), ghi = slice_lo((int64_t)c.gcount, D, slice + 1);
+    long long w0 = (long long)c.goff, w1 = (long long)(c.goff + c.count);
+    glo = glo < w0 ? w0 : (glo > w1 ? w1 : glo);
+    ghi = ghi < w0 ? w0 : (ghi > w1 ? w1 : ghi);
+    *lo = glo - w0;
+    *hi = ghi - w0;
+}
+
+}  // namespace trv

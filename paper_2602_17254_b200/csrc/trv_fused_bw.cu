@@ -1,0 +1,234 @@
+// FUSED kernel of the bandwidth-optimal form (Sec. 4.1): Reduce-Scatter + AllGather in one pass.
+//
+// The Reduce-Scatter phase follows the same communication pattern as the latency-optimal form
+// (Sec. 4.2) and only restricts every message to the blocks of the closed-form set Pi
+// (Sec. 4.3).  The partial of block j that rank q holds after step t is therefore the
+// latency-form partial of rank q after step t, restricted to block j; the owner j ends with
+//      T_S(j),   T_t(p) = (T_{t-1}(p - dist_t) + T_{t-1}(p)) + T_{t-1}(p + dist_t),   T_0(p) = input of p,
+// and the AllGather copies that value to every rank.  T_S(j) is a balanced ternary tree whose
+// 3^S leaves, read left to right, are the ranks j + sum_t eps_t dist_t with the digit of the
+// LAST step most significant and eps = -1, 0, +1 in that order.  A thread streams the n inputs
+// of its element column(s) in exactly that order, nine at a time, through an S-level carry
+// stack (n - 1 adds, the association of the schedule), then writes the value to all n ranks:
+// n*count elements read once, n*count written once, no shared-memory staging of data.
+#include "trv_dev.cuh"
+
+namespace trv {
+
+constexpr int kBwThreads = 256;
+constexpr int kBwMaxD = 4;
+constexpr int kBwMaxS = 6;
+
+struct BwArgs {
+    int n;
+    long long w0;                               // global index of local element 0
+    long long lo[kBwMaxD], hi[kBwMaxD];         // local element range of each slice
+    long long glo[kBwMaxD], ghi[kBwMaxD];       // global element range of each slice
+    int dims[kBwMaxD], dstride[kBwMaxD];
+    int ldim[kBwMaxD][kBwMaxS], ldist[kBwMaxD][kBwMaxS];   // per slice, per step: dimension, distance
+};
+
+template <typename T, int V>
+struct alignas(sizeof(T) * V) Pack {
+    T x[V];
+};
+template <typename T, int V>
+__device__ __forceinline__ Pack<T, V> padd(const Pack<T, V>& a, const Pack<T, V>& b) {
+    Pack<T, V> r;
+#pragma unroll
+    for (int k = 0; k < V; ++k) r.x[k] = add2(a.x[k], b.x[k]);
+    return r;
+}
+template <typename T, int V>
+__device__ __forceinline__ Pack<T, V> padd3(const Pack<T, V>& a, const Pack<T, V>& b, const Pack<T, V>& c) {
+    return padd(padd(a, b), c);
+}
+
+__device__ __forceinline__ int wrap(int x, int a) { return x < 0 ? x + a : (x >= a ? x - a : x); }
+
+// Value of block owner j for the V columns starting at local element e, written to all ranks.
+template <typename T, int V, int S, int D>
+__device__ __forceinline__ void column_tree(const BwArgs& a, int c, const T* const* sin, T* const* sout, long long e, int j) {
+    using P = Pack<T, V>;
+    constexpr int N = (S == 1) ? 3 : (S == 2 ? 9 : 0);
+    (void)N;
+    int base[D];    // coordinates of the centre of the current nine-leaf chunk
+#pragma unroll
+    for (int d = 0; d < D; ++d) base[d] = (j / a.dstride[d]) % a.dims[d];
+    P res;
+    if constexpr (S == 1) {
+        const int d0 = a.ldim[c][0], x0 = a.ldist[c][0];
+        int bd = 0, ad = 1, sd = 1;
+#pragma unroll
+        for (int d = 0; d < D; ++d) if (d == d0) { bd = base[d]; ad = a.dims[d]; sd = a.dstride[d]; }
+        const P l = *reinterpret_cast<const P*>(sin[j + (wrap(bd - x0, ad) - bd) * sd] + e);
+        const P m = *reinterpret_cast<const P*>(sin[j] + e);
+        const P r = *reinterpret_cast<const P*>(sin[j + (wrap(bd + x0, ad) - bd) * sd] + e);
+        res = padd3(l, m, r);
+    } else {
+        // start at the leftmost chunk: every step >= 2 at eps = -1
+#pragma unroll
+        for (int t = 2; t < S; ++t) {
+            const int dt = a.ldim[c][t], xt = a.ldist[c][t];
+#pragma unroll
+            for (int d = 0; d < D; ++d) if (d == dt) base[d] = wrap(base[d] - xt, a.dims[d]);
+        }
+        const int d0 = a.ldim[c][0], x0 = a.ldist[c][0], d1 = a.ldim[c][1], x1 = a.ldist[c][1];
+        int dg[S];      // digit (child number) of each level >= 2
+        P acc[S];
+#pragma unroll
+        for (int t = 0; t < S; ++t) dg[t] = 0;
+        constexpr int CHUNKS = (S == 2) ? 1 : (S == 3 ? 3 : (S == 4 ? 9 : (S == 5 ? 27 : 81)));
+        for (int ch = 0; ch < CHUNKS; ++ch) {
+            int rank_c = 0, b0 = 0, a0 = 1, s0 = 1, b1 = 0, a1 = 1, s1 = 1;
+#pragma unroll
+            for (int d = 0; d < D; ++d) {
+                rank_c += base[d] * a.dstride[d];
+                if (d == d0) { b0 = base[d]; a0 = a.dims[d]; s0 = a.dstride[d]; }
+                if (d == d1) { b1 = base[d]; a1 = a.dims[d]; s1 = a.dstride[d]; }
+            }
+            int rk[9];
+            if (d0 != d1) {
+                int X0[3], X1[3];
+#pragma unroll
+                for (int q = 0; q < 3; ++q) {
+                    X0[q] = (wrap(b0 + (q - 1) * x0, a0) - b0) * s0;
+                    X1[q] = (wrap(b1 + (q - 1) * x1, a1) - b1) * s1;
+                }
+#pragma unroll
+                for (int m = 0; m < 9; ++m) rk[m] = rank_c + X1[m / 3] + X0[m % 3];
+            } else {
+#pragma unroll
+                for (int m = 0; m < 9; ++m) rk[m] = rank_c + (wrap(b0 + (m / 3 - 1) * x1 + (m % 3 - 1) * x0, a0) - b0) * s0;
+            }
+            P l[9];
+#pragma unroll
+            for (int m = 0; m < 9; ++m) l[m] = *reinterpret_cast<const P*>(sin[rk[m]] + e);
+            P r = padd3(padd3(l[0], l[1], l[2]), padd3(l[3], l[4], l[5]), padd3(l[6], l[7], l[8]));
+            // carry the finished 9-leaf subtree up the tree
+            bool carry = true;
+#pragma unroll
+            for (int t = 2; t < S; ++t) {
+                if (carry) {
+                    const int dt = a.ldim[c][t], xt = a.ldist[c][t];
+                    int delta;
+                    if (dg[t] == 0) { acc[t] = r; dg[t] = 1; delta = xt; carry = false; }
+                    else if (dg[t] == 1) { acc[t] = padd(acc[t], r); dg[t] = 2; delta = xt; carry = false; }
+                    else { r = padd(acc[t], r); dg[t] = 0; delta = -2 * xt; }
+#pragma unroll
+                    for (int d = 0; d < D; ++d) if (d == dt) base[d] = wrap(base[d] + delta, a.dims[d]);
+                }
+            }
+            res = r;    // after the last chunk the carry has run through every level
+        }
+    }
+    // AllGather: the owner's value goes to every rank
+#pragma unroll 9
+    for (int r = 0; r < a.n; ++r) *reinterpret_cast<P*>(sout[r] + e) = res;
+}
+
+template <typename T, int V, int S, int D, int CAP>
+__global__ void __launch_bounds__(kBwThreads) k_bw_fused(PtrTab<CAP> in, PtrTab<CAP> out, BwArgs a) {
+    __shared__ const T* sin[CAP];
+    __shared__ T* sout[CAP];
+    for (int r = threadIdx.x; r < a.n; r += kBwThreads) { sin[r] = (const T*)in.p[r]; sout[r] = (T*)out.p[r]; }
+    __syncthreads();
+    const int c = blockIdx.y;
+    const long long lo = a.lo[c], hi = a.hi[c];
+    const long long e = ((lo / V) + (long long)blockIdx.x * kBwThreads + threadIdx.x) * V;
+    if (e >= hi) return;
+    const unsigned long long L = (unsigned long long)(a.ghi[c] - a.glo[c]);
+    auto owner = [&](long long el) -> int {
+        const unsigned long long x = (unsigned long long)(a.w0 + el - a.glo[c]);
+        return (int)(((x + 1) * (unsigned)a.n - 1) / L);
+    };
+    if constexpr (V == 1) {
+        if (e >= lo) column_tree<T, 1, S, D>(a, c, sin, sout, e, owner(e));
+    } else {
+        const bool inside = e >= lo && e + V <= hi;
+        int j0 = 0;
+        bool same = false;
+        if (inside) { j0 = owner(e); same = owner(e + V - 1) == j0; }
+        if (same) {
+            column_tree<T, V, S, D>(a, c, sin, sout, e, j0);
+        } else {
+            for (int k = 0; k < V; ++k)
+                if (e + k >= lo && e + k < hi) column_tree<T, 1, S, D>(a, c, sin, sout, e + k, owner(e + k));
+        }
+    }
+}
+
+// ------------------------------------------------------------------ host side
+
+bool fused_bandwidth_supported(const Plan& p) {
+    return p.algo == TRV_ALGO_TRIVANCE && p.variant == TRV_BANDWIDTH_OPTIMAL && p.ndims <= kBwMaxD && p.S <= kBwMaxS;
+}
+
+template <typename T, int V, int S, int D>
+static void launch_bw(const Call& c, const BwArgs& a) {
+    constexpr int CAP = S <= 3 ? 32 : (S <= 5 ? 256 : TRV_MAX_RANKS);
+    const Plan& p = *c.plan;
+    PtrTab<CAP> in, out;
+    for (int r = 0; r < p.n; ++r) { in.p[r] = const_cast<void*>(c.in[r]); out.p[r] = c.out[r]; }
+    long long tiles = 0;
+    for (int sl = 0; sl < D; ++sl)
+        if (a.hi[sl] > a.lo[sl]) {
+            long long t = (a.hi[sl] - (a.lo[sl] / V) * V + (long long)V * kBwThreads - 1) / ((long long)V * kBwThreads);
+            if (t > tiles) tiles = t;
+        }
+    if (tiles == 0) return;
+    TRV_LAUNCH((k_bw_fused<T, V, S, D, CAP>), dim3((unsigned)tiles, D, 1), kBwThreads, 0, c.st, in, out, a);
+}
+
+template <typename T, int V, int S>
+static trv_status_t bw_by_d(const Call& c, const BwArgs& a) {
+    switch (c.plan->ndims) {
+        case 1: launch_bw<T, V, S, 1>(c, a); return TRV_OK;
+        case 2: if constexpr (S >= 2) { launch_bw<T, V, S, 2>(c, a); return TRV_OK; } break;
+        case 3: if constexpr (S >= 3) { launch_bw<T, V, S, 3>(c, a); return TRV_OK; } break;
+        case 4: if constexpr (S >= 4) { launch_bw<T, V, S, 4>(c, a); return TRV_OK; } break;
+    }
+    return TRV_ERR_UNSUPPORTED;
+}
+
+template <typename T, int V>
+static trv_status_t bw_by_s(const Call& c, const BwArgs& a) {
+    switch (c.plan->S) {
+        case 1: return bw_by_d<T, V, 1>(c, a);
+        case 2: return bw_by_d<T, V, 2>(c, a);
+        case 3: return bw_by_d<T, V, 3>(c, a);
+        case 4: return bw_by_d<T, V, 4>(c, a);
+        case 5: return bw_by_d<T, V, 5>(c, a);
+        case 6: return bw_by_d<T, V, 6>(c, a);
+    }
+    return TRV_ERR_UNSUPPORTED;
+}
+
+trv_status_t run_fused_bandwidth(const Call& c) {
+    const Plan& p = *c.plan;
+    if (!fused_bandwidth_supported(p)) return TRV_ERR_UNSUPPORTED;
+    BwArgs a;
+    a.n = p.n;
+    a.w0 = (long long)c.goff;
+    long long min_block = -1;
+    for (int d = 0; d < kBwMaxD; ++d) { a.dims[d] = d < p.ndims ? p.dims[d] : 1; a.dstride[d] = d < p.ndims ? p.stride[d] : 1; }
+    for (int sl = 0; sl < p.ndims; ++sl) {
+        local_slice(c, sl, &a.lo[sl], &a.hi[sl]);
+        a.glo[sl] = slice_lo((int64_t)c.gcount, p.ndims, sl);
+        a.ghi[sl] = slice_lo((int64_t)c.gcount, p.ndims, sl + 1);
+        const long long bl = (a.ghi[sl] - a.glo[sl]) / p.n;
+        if (min_block < 0 || bl < min_block) min_block = bl;
+        for (int t = 0; t < p.S; ++t) { a.ldim[sl][t] = p.steps[sl][t].dim; a.ldist[sl][t] = p.steps[sl][t].dist; }
+    }
+    // Four columns per thread when blocks are long enough that few threads straddle a block
+    // boundary; one column per thread otherwise (every thread then has its own owner).
+    const bool wide = min_block >= 256;
+    g_last_kernel = wide ? "bw_fused<V=4>" : "bw_fused<V=1>";
+    trv_status_t st;
+    if (c.dtype == TRV_FLOAT32) st = wide ? bw_by_s<float, 4>(c, a) : bw_by_s<float, 1>(c, a);
+    else st = wide ? bw_by_s<uint32_t, 4>(c, a) : bw_by_s<uint32_t, 1>(c, a);
+    if (st != TRV_OK) return st;
+    return cudaGetLastError() == cudaSuccess ? TRV_OK : TRV_ERR_CUDA;
+}
+
+}  // namespace trv

@@ -1,0 +1,126 @@
+// Schedule builder: per-step (dimension, distance) lists, peers, closed-form block sets and
+// per-message byte counts.  Host-only integer work; no CUDA call in this file.
+#include "trv_plan.h"
+
+#include <new>
+
+namespace trv {
+
+static int exact_log(int a, int base) {
+    int s = 0;
+    if (a < 1) return -1;
+    while (a > 1) {
+        if (a % base) return -1;
+        a /= base;
+        ++s;
+    }
+    return s;
+}
+
+trv_status_t build_plan(const int32_t* dims, int32_t ndims, int variant, int algo, trv_plan_s** out) {
+    if (!dims || !out || ndims < 1 || ndims > TRV_MAX_DIMS) return TRV_ERR_INVALID_ARG;
+    if (variant != TRV_LATENCY_OPTIMAL && variant != TRV_BANDWIDTH_OPTIMAL) return TRV_ERR_INVALID_ARG;
+    if (algo != TRV_ALGO_TRIVANCE && algo != TRV_ALGO_BRUCK && algo != TRV_ALGO_RECDOUB) return TRV_ERR_INVALID_ARG;
+    for (int d = 0; d < ndims; ++d)
+        if (dims[d] < 2) return TRV_ERR_INVALID_ARG;
+    const int base = (algo == TRV_ALGO_RECDOUB) ? 2 : 3;
+    if (algo == TRV_ALGO_RECDOUB && ndims != 1) return TRV_ERR_UNSUPPORTED;
+
+    trv_plan_s* holder = new (std::nothrow) trv_plan_s();
+    if (!holder) return TRV_ERR_ALLOC;
+    Plan& p = holder->plan;
+    p.algo = algo; p.variant = variant; p.ndims = ndims; p.base = base;
+    long long n = 1;
+    for (int d = 0; d < ndims; ++d) {
+        int s = exact_log(dims[d], base);
+        if (s < 1) {
+            delete holder;
+            return algo == TRV_ALGO_RECDOUB ? TRV_ERR_UNDEFINED_SCHEDULE : TRV_ERR_UNSUPPORTED;
+        }
+        p.dims[d] = dims[d]; p.sdim[d] = s; p.stride[d] = (int)n;
+        n *= dims[d]; p.S += s;
+        if (n > TRV_MAX_RANKS) { delete holder; return TRV_ERR_UNSUPPORTED; }
+        if (dims[d] != dims[0]) p.equal_dims = false;
+    }
+    p.n = (int)n;
+
+    // Sec. 5: collective c starts on dimension c and moves to the next dimension every step;
+    // a dimension that has used up its log_base(a_d) steps is skipped.
+    p.steps.resize(ndims);
+    p.mod.resize(ndims);
+    for (int c = 0; c < ndims; ++c) {
+        int visits[TRV_MAX_DIMS] = {0};
+        int pw[TRV_MAX_DIMS];
+        for (int d = 0; d < ndims; ++d) pw[d] = 1;
+        int cur = c;
+        for (int t = 0; t < p.S; ++t) {
+            int d = cur;
+            while (visits[d] >= p.sdim[d]) d = (d + 1) % ndims;
+            p.steps[c].push_back(Step{d, pw[d]});
+            visits[d]++; pw[d] *= base;
+            p.mod[c].push_back(std::vector<int>(pw, pw + ndims));
+            cur = (d + 1) % ndims;
+        }
+    }
+    *out = holder;
+    return TRV_OK;
+}
+
+bool in_send_set(const Plan& p, int c, int t, int dst, int j) {
+    for (int d = 0; d < p.ndims; ++d) {
+        int m = p.mod[c][t][d];
+        if ((p.coord(j, d) - p.coord(dst, d)) % m != 0) return false;
+    }
+    return true;
+}
+
+int send_peers(const Plan& p, int r, int dim, int dist, int peer[2], int dir[2], int hops[2]) {
+    switch (p.algo) {
+        case TRV_ALGO_TRIVANCE:
+            peer[0] = p.shift(r, dim, -dist); dir[0] = -1; hops[0] = dist;
+            peer[1] = p.shift(r, dim, +dist); dir[1] = +1; hops[1] = dist;
+            return 2;
+        case TRV_ALGO_BRUCK:
+            peer[0] = p.shift(r, dim, dist);     dir[0] = +1; hops[0] = dist;
+            peer[1] = p.shift(r, dim, 2 * dist); dir[1] = +1; hops[1] = 2 * dist;
+            return 2;
+        default: {
+            int x = p.coord(r, dim), y = x ^ dist;
+            peer[0] = r + (y - x) * p.stride[dim]; dir[0] = y > x ? +1 : -1; hops[0] = dist;
+            peer[1] = -1; dir[1] = 0; hops[1] = 0;
+            return 1;
+        }
+    }
+}
+
+void message_bytes(const Plan& p, int64_t E, int64_t elem_size, int c, int row, int64_t* out) {
+    const int n = p.n, D = p.ndims;
+    const int64_t lo = slice_lo(E, D, c), hi = slice_lo(E, D, c + 1);
+    if (p.variant == TRV_LATENCY_OPTIMAL) {
+        for (int r = 0; r < n; ++r) out[r] = (hi - lo) * elem_size;
+        return;
+    }
+    // The set of row `row` is the same congruence class for Reduce-Scatter (blocks destined to
+    // travel on through the receiver) and for the mirrored AllGather row (finished blocks the
+    // sender holds): all j that agree with the rank modulo mod[c][t][d] in every dimension.
+    const int t = p.step_of_row(row);
+    for (int r = 0; r < n; ++r) {
+        int64_t sum = 0;
+        // enumerate j_d = (r_d mod m_d) + m_d * i_d
+        int idx[TRV_MAX_DIMS] = {0};
+        for (;;) {
+            int j = 0;
+            for (int d = 0; d < D; ++d) j += ((p.coord(r, d) % p.mod[c][t][d]) + p.mod[c][t][d] * idx[d]) * p.stride[d];
+            sum += block_lo(lo, hi, n, j + 1) - block_lo(lo, hi, n, j);
+            int d = 0;
+            for (; d < D; ++d) {
+                if (++idx[d] < p.dims[d] / p.mod[c][t][d]) break;
+                idx[d] = 0;
+            }
+            if (d == D) break;
+        }
+        out[r] = sum * elem_size;
+    }
+}
+
+}  // namespace trv

@@ -1,0 +1,66 @@
+// Host-side schedule of a Trivance (or comparator) plan: integer work only.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <vector>
+
+#include "../../include/trivance.h"
+
+namespace trv {
+
+struct Step {
+    int dim;    // torus dimension the step runs along
+    int dist;   // ring distance inside that dimension: base^(earlier visits of dim)
+};
+
+// What a fused kernel needs to know about one collective (slice).
+struct Plan {
+    int algo = 0, variant = 0, ndims = 0, n = 0, S = 0, base = 3;
+    int dims[TRV_MAX_DIMS] = {0};
+    int stride[TRV_MAX_DIMS] = {0};     // rank = sum_d x_d * stride[d]
+    int sdim[TRV_MAX_DIMS] = {0};       // steps in dimension d = log_base a_d
+    bool equal_dims = true;
+    // steps[c][t]: Reduce-Scatter / latency-form step t of collective c (Sec. 4.1, Sec. 5)
+    std::vector<std::vector<Step>> steps;
+    // mod[c][t][d] = base^(number of steps <= t of collective c that ran along d): block j is in
+    // the message to p at step t iff j_d == p_d (mod mod[c][t][d]) for every d  (closed form Pi)
+    std::vector<std::vector<std::vector<int>>> mod;
+
+    // plan-owned scratch for trv_allreduce (STEP family of the latency form), grown on demand
+    void* scratch = nullptr;
+    size_t scratch_bytes = 0;
+
+    int rows() const { return variant == TRV_BANDWIDTH_OPTIMAL ? 2 * S : S; }
+    // schedule step behind a row: AllGather rows mirror the Reduce-Scatter steps
+    int step_of_row(int row) const { return row < S ? row : 2 * S - 1 - row; }
+    int coord(int r, int d) const { return (r / stride[d]) % dims[d]; }
+    int shift(int r, int d, int delta) const {
+        int a = dims[d], x = coord(r, d);
+        int y = ((x + delta) % a + a) % a;
+        return r + (y - x) * stride[d];
+    }
+};
+
+
+
+// element ranges (global indices)
+inline int64_t slice_lo(int64_t E, int D, int c) { return (int64_t)(((unsigned __int128)c * (unsigned __int128)E) / D); }
+inline int64_t block_lo(int64_t lo, int64_t hi, int n, int j) {
+    return lo + (int64_t)(((unsigned __int128)j * (unsigned __int128)(hi - lo)) / n);
+}
+
+bool in_send_set(const Plan& p, int c, int t, int dst, int j);
+// peers a rank sends to in step (dim, dist); returns how many; dir = +1 / -1, hops = links crossed
+int send_peers(const Plan& p, int r, int dim, int dist, int peer[2], int dir[2], int hops[2]);
+// message bytes of one row, indexed by destination (row < S) or by source (AllGather rows)
+void message_bytes(const Plan& p, int64_t E, int64_t elem_size, int c, int row, int64_t* out);
+
+}  // namespace trv
+
+struct trv_plan_s {
+    trv::Plan plan;
+};
+
+namespace trv {
+trv_status_t build_plan(const int32_t* dims, int32_t ndims, int variant, int algo, trv_plan_s** out);
+}

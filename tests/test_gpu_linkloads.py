@@ -1,0 +1,74 @@
+"""GPU link-load tally (trv_link_loads) vs the oracle's hop-by-hop walk: integer tables, bit-exact."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_17254_b200 import binding, build
+
+pytestmark = pytest.mark.gpu
+LAT, BW = binding.LATENCY_OPTIMAL, binding.BANDWIDTH_OPTIMAL
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    assert torch.cuda.is_available()
+
+
+def _same(a, b):
+    for k in ("msgs", "bytes", "max_msgs", "max_bytes"):
+        assert a[k].dtype == b[k].dtype and np.array_equal(a[k], b[k]), k
+
+
+@pytest.mark.parametrize("dims", [(3,), (9,), (27,), (81,), (243,), (729,), (3, 3), (9, 9), (3, 3, 3), (9, 9, 9), (3, 9),
+                                  (27, 3), (3, 3, 9)])
+@pytest.mark.parametrize("variant", [LAT, BW])
+@pytest.mark.parametrize("count", [1024, 7, 100003])
+def test_trivance_link_loads(dims, variant, count):
+    got = binding.Plan(dims, variant).link_loads(count, 4)
+    _same(got, oracle.link_loads(dims, variant, count, 4))
+
+
+@pytest.mark.parametrize("dims", [(9,), (27,), (243,), (9, 9), (3, 9)])
+@pytest.mark.parametrize("variant", [LAT, BW])
+def test_bruck_link_loads(dims, variant):
+    got = binding.Plan(dims, variant, binding.ALGO_BRUCK).link_loads(100003, 4)
+    _same(got, oracle.link_loads(dims, variant, 100003, 4, algo=oracle.ALGO_BRUCK))
+
+
+@pytest.mark.parametrize("n", [2, 8, 64, 1024])
+@pytest.mark.parametrize("variant", [LAT, BW])
+def test_recursive_doubling_link_loads(n, variant):
+    got = binding.Plan((n,), variant, binding.ALGO_RECDOUB).link_loads(100003, 2)
+    _same(got, oracle.link_loads((n,), variant, 100003, 2, algo=oracle.ALGO_RECDOUB))
+
+
+def test_fig1_values_on_the_gpu():
+    algo = {"trivance": binding.ALGO_TRIVANCE, "bruck": binding.ALGO_BRUCK, "recursive_doubling": binding.ALGO_RECDOUB}
+    with open(os.path.join(GOLD, "fig1_max_link_congestion.txt")) as f:
+        rows = [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+    for name, n, *want in rows:
+        ll = binding.Plan((int(n),), LAT, algo[name]).link_loads(1024, 4)
+        assert ll["max_msgs"].tolist() == [int(v) for v in want]
+
+
+def test_config1_and_config5_tables():
+    ll = binding.Plan((9,), LAT).link_loads(1024, 4)
+    assert np.all(ll["msgs"][0] == 1) and np.all(ll["msgs"][1] == 3)
+    assert np.all(ll["bytes"][0] == 4096) and np.all(ll["bytes"][1] == 12288)
+    for count in (8192, 131072, 2097152, 8388608):
+        for variant in (LAT, BW):
+            tv = binding.Plan((243,), variant).link_loads(count, 4)
+            br = binding.Plan((243,), variant, binding.ALGO_BRUCK).link_loads(count, 4)
+            _same(tv, oracle.link_loads((243,), variant, count, 4))
+            _same(br, oracle.link_loads((243,), variant, count, 4, algo=oracle.ALGO_BRUCK))
+            k = [r if r < 5 else 9 - r for r in range(tv["max_msgs"].size)]
+            assert tv["max_msgs"].tolist() == [3 ** v for v in k]
+            assert br["max_msgs"].tolist() == [3 * 3 ** v for v in k]
+    with pytest.raises(binding.TrivanceError) as e:
+        binding.Plan((243,), LAT, binding.ALGO_RECDOUB)
+    assert e.value.status == binding.ERR_UNDEFINED_SCHEDULE

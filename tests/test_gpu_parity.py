@@ -1,0 +1,180 @@
+"""GPU parity: the CUDA path through the C ABI vs the CPU oracle, element by element, bit-exact.
+
+Small cases: sizes the oracle finishes in seconds that still span several tiles and ragged tails,
+every kernel family, both dtypes, in place and out of place, sharded windows, degenerate sizes.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_17254_b200 import binding, build, synth
+
+from gpu_util import DEV, check_case, compare, run_gpu, torch_dtype, upload_matrix
+
+pytestmark = pytest.mark.gpu
+
+LAT, BW = binding.LATENCY_OPTIMAL, binding.BANDWIDTH_OPTIMAL
+AUTO, STEP, FUSED = binding.KERNEL_AUTO, binding.KERNEL_STEP, binding.KERNEL_FUSED
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    assert torch.cuda.is_available()
+    binding.lib()
+
+
+FUSED_LAT = [(3,), (9,), (27,), (81,), (243,), (729,), (3, 3), (9, 9), (3, 3, 3), (3, 3, 3, 3), (9, 9, 9)]
+ANY = FUSED_LAT + [(3, 9), (27, 3), (3, 3, 9), (27, 27)]
+
+
+@pytest.mark.parametrize("dims", ANY)
+@pytest.mark.parametrize("variant", [LAT, BW])
+def test_step_family_matches_oracle(dims, variant):
+    n = int(np.prod(dims))
+    count = 1531 if n <= 243 else 517
+    check_case(dims, variant, count, "normal", 11, STEP)
+    check_case(dims, variant, count, "int32", 12, STEP, in_place=False)
+
+
+@pytest.mark.parametrize("dims", FUSED_LAT)
+def test_fused_latency_matches_oracle(dims):
+    n = int(np.prod(dims))
+    count = 4133 if n <= 243 else 1029          # several tiles of every kernel + ragged tail
+    check_case(dims, LAT, count, "normal", 21, FUSED)
+    check_case(dims, LAT, count, "int32", 22, FUSED, in_place=False)
+
+
+@pytest.mark.parametrize("dims", ANY)
+def test_fused_bandwidth_matches_oracle(dims):
+    n = int(np.prod(dims))
+    D = len(dims)
+    small = 1531 if n <= 243 else 517                     # one column per thread (short blocks)
+    check_case(dims, BW, small, "normal", 31, FUSED)
+    check_case(dims, BW, small, "int32", 32, FUSED, in_place=False)
+    if n <= 81:                                           # four columns per thread (blocks >= 256 elements)
+        wide = 300 * n * D + 7
+        check_case(dims, BW, wide, "normal", 33, FUSED)
+        check_case(dims, BW, wide, "int32", 34, FUSED, in_place=False)
+
+
+def test_fused_bandwidth_wide_path_on_729_ranks_sampled():
+    """9x9x9 with blocks of >= 256 elements: the oracle checks windows around slice and block
+    boundaries and in block interiors."""
+    dims, count = (9, 9, 9), 300 * 729 * 3 + 5
+    plan = binding.Plan(dims, BW)
+    wins = [(0, 700), (count // 3 - 400, count // 3 + 400), (2 * count // 3 - 333, 2 * count // 3 + 777),
+            (count - 900, count), (123456, 124000)]
+    xd, keep = upload_matrix("uniform", 35, 729, count, wins)
+    res = run_gpu(plan, xd, FUSED, in_place=False)
+    assert binding.last_kernel_name() == "bw_fused<V=4>"
+    for (w0, w1), xh in zip(wins, keep):
+        compare(dims, BW, xh, res[:, w0:w1].cpu().numpy(), E=count, e0=w0)
+
+
+@pytest.mark.parametrize("dims,variant", [((27,), LAT), ((9, 9), LAT), ((9, 9, 9), LAT), ((243,), LAT), ((81,), BW), ((9, 9, 9), BW)])
+@pytest.mark.parametrize("count", [1, 2, 3, 4, 5, 31, 32, 33, 127])
+def test_degenerate_sizes(dims, variant, count):
+    """Fewer elements than ranks / than dimensions: empty slices and empty blocks."""
+    for kernel in (STEP, FUSED):
+        check_case(dims, variant, count, "int32", count, kernel)
+        check_case(dims, variant, count, "normal", count, kernel, in_place=False)
+
+
+@pytest.mark.parametrize("dims,variant", [((27,), LAT), ((9, 9, 9), LAT), ((243,), LAT), ((9, 9), BW), ((9, 9, 9), BW), ((81,), BW)])
+def test_sharded_windows_equal_the_unsharded_run(dims, variant):
+    """Element-range shards carry the global element index: concatenating the shards' results gives
+    the unsharded result (slice and block membership must not move)."""
+    n = int(np.prod(dims))
+    total = 3001
+    for kernel in (STEP, FUSED):
+        pieces = []
+        for (go, cnt) in [(0, 1000), (1000, 996), (1996, 1005)]:
+            x = synth.rank_matrix("normal", 41, n, total)[:, go:go + cnt]
+            plan = binding.Plan(dims, variant)
+            pad = (cnt + 3) // 4 * 4
+            buf = torch.zeros((n, pad), dtype=torch.float32, device=DEV)
+            xd = buf[:, :cnt]
+            xd.copy_(torch.from_numpy(np.ascontiguousarray(x)))
+            got = run_gpu(plan, xd, kernel, True, total, go).cpu().numpy()
+            compare(dims, variant, np.ascontiguousarray(x), got, E=total, e0=go)
+            pieces.append(got)
+        full = oracle.allreduce(dims, variant, synth.rank_matrix("normal", 41, n, total))
+        assert np.array_equal(np.concatenate(pieces, axis=1), full)
+
+
+def test_default_entry_point_and_plan_owned_scratch():
+    """trv_allreduce (in place, AUTO) incl. the case where the plan has to allocate scratch itself."""
+    for dims, variant in [((27,), LAT), ((27, 3), LAT), ((81,), BW)]:
+        plan = binding.Plan(dims, variant)
+        n = plan.n
+        x = synth.rank_matrix("normal", 51, n, 2048)
+        xd = torch.from_numpy(x).to(DEV)
+        for _ in range(2):      # second call reuses the plan's scratch
+            xd.copy_(torch.from_numpy(x))
+            plan.allreduce([xd[r].data_ptr() for r in range(n)], 2048, binding.FLOAT32,
+                           torch.cuda.current_stream().cuda_stream)
+            torch.cuda.synchronize()
+            compare(dims, variant, x, xd.cpu().numpy())
+        plan.destroy()
+
+
+def test_separate_rank_allocations_and_side_stream():
+    """Rank buffers need not be rows of one tensor; work is queued on the caller's stream."""
+    dims = (9, 9)
+    plan = binding.Plan(dims, LAT)
+    x = synth.rank_matrix("normal", 61, 81, 1000)
+    bufs = [torch.from_numpy(x[r]).to(DEV) for r in range(81)]
+    s = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s):
+        plan.allreduce_ex([b.data_ptr() for b in bufs], None, 1000, binding.FLOAT32, stream=s.cuda_stream)
+    s.synchronize()
+    compare(dims, LAT, x, np.stack([b.cpu().numpy() for b in bufs]))
+
+
+def test_host_buffer_entry_point():
+    dims, count = (27,), 5000
+    plan = binding.Plan(dims, LAT)
+    x = synth.rank_matrix("normal", 71, 27, count)
+    hin = torch.from_numpy(x.copy()).pin_memory()
+    hout = torch.empty_like(hin).pin_memory()
+    ws = torch.empty(plan.host_workspace_bytes(count), dtype=torch.uint8, device=DEV)
+    plan.allreduce_host([hin[r].data_ptr() for r in range(27)], [hout[r].data_ptr() for r in range(27)], count,
+                        binding.FLOAT32, ws.data_ptr(), ws.numel(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    compare(dims, LAT, x, hout.numpy())
+    with pytest.raises(binding.TrivanceError) as e:
+        plan.allreduce_host([hin[r].data_ptr() for r in range(27)], None, count, binding.FLOAT32, ws.data_ptr(), 1024)
+    assert e.value.status == binding.ERR_SCRATCH
+
+
+def test_fp32_tolerance_against_naive_and_exact_sums():
+    """|err| <= 2e-6 * sum|x| against the naive sequential binary32 sum (and the fp64 sum)."""
+    for dims, variant, dist in [((27,), LAT, "normal"), ((81,), BW, "normal"), ((9, 9, 9), LAT, "uniform"),
+                                ((9, 9, 9), BW, "uniform"), ((243,), LAT, "normal"), ((243,), BW, "normal")]:
+        plan = binding.Plan(dims, variant)
+        x = synth.rank_matrix(dist, 81, plan.n, 2048)
+        got = run_gpu(plan, torch.from_numpy(x).to(DEV)).cpu().numpy().astype(np.float64)
+        sabs = np.abs(x.astype(np.float64)).sum(0)
+        assert np.all(np.abs(got - oracle.naive_sum_f32(x).astype(np.float64)) <= 2e-6 * sabs)
+        assert np.all(np.abs(got - x.astype(np.float64).sum(0)) <= 2e-6 * sabs)
+
+
+def test_latency_rows_differ_and_bandwidth_rows_agree():
+    x = synth.rank_matrix("normal", 91, 27, 4096)
+    lat = run_gpu(binding.Plan((27,), LAT), torch.from_numpy(x).to(DEV)).cpu().numpy()
+    bw = run_gpu(binding.Plan((27,), BW), torch.from_numpy(x).to(DEV)).cpu().numpy()
+    assert any(not np.array_equal(lat[0], lat[r]) for r in range(1, 27))
+    assert all(np.array_equal(bw[0], bw[r]) for r in range(1, 27))
+
+
+def test_launch_counter_and_kernel_names():
+    plan = binding.Plan((27,), LAT)
+    xd = torch.zeros((27, 1024), device=DEV)
+    before = binding.launch_count()
+    run_gpu(plan, xd, FUSED)
+    assert binding.launch_count() == before + 1 and binding.last_kernel_name() == "lat_reg<27>"
+    run_gpu(plan, xd, STEP)
+    assert binding.launch_count() == before + 1 + 3 and binding.last_kernel_name() == "step_latency"
