@@ -32,7 +32,8 @@ typedef enum {
     TRV_ERR_UNDEFINED_SCHEDULE = 3, /* the schedule does not exist for this n (Recursive Doubling, n != 2^q) */
     TRV_ERR_ALLOC = 4,
     TRV_ERR_CUDA = 5,               /* a CUDA runtime call failed; cudaGetLastError has the reason */
-    TRV_ERR_SCRATCH = 6             /* caller-provided scratch/workspace too small or misaligned */
+    TRV_ERR_SCRATCH = 6,            /* caller-provided scratch/workspace too small or misaligned */
+    TRV_ERR_TOO_LARGE = 7           /* the call needs more than the fixed capacity of a no-allocation entry point */
 } trv_status_t;
 
 typedef enum { TRV_LATENCY_OPTIMAL = 0, TRV_BANDWIDTH_OPTIMAL = 1 } trv_variant_t;
@@ -153,6 +154,32 @@ trv_status_t trv_allreduce_host(trv_plan_t plan, const void *const *host_in, voi
                                 trv_dtype_t dtype, trv_op_t op, void *workspace, size_t workspace_bytes,
                                 void *cuda_stream);
 trv_status_t trv_host_workspace_bytes(trv_plan_t plan, size_t count, size_t *bytes);
+
+/* AllReduce for callers that cannot allocate device memory.  (The paper has no counterpart: this
+ * is a packaging of the step-by-step latency form, not a part of the method.)
+ *
+ * Some callers may not call cudaMalloc or cudaFree at all: code running while a stream is being
+ * captured into a CUDA graph, code inside a framework that owns all device memory and forbids
+ * allocation outside its pool, or a process whose memory budget is fixed at start-up.  The step
+ * family of the latency form needs ping-pong scratch; here that scratch is a fixed array of
+ * trv_noalloc_max_scratch_bytes() = 16 MiB that is part of the library image.  Every GPU that
+ * loads the library gives up those 16 MiB until the process exits.
+ *
+ * Semantics are those of trv_allreduce (in place, HOST array of n DEVICE pointers, asynchronous on
+ * cuda_stream) for latency-optimal Trivance plans, executed by the STEP kernel family; results are
+ * bit-identical to trv_allreduce.  The call makes no cudaMalloc, cudaFree or other allocating call.
+ *   - The scratch needed is buffers * n * round_up(count, 64) * 4 bytes, buffers = 1 if the plan
+ *     has an even number of steps, 2 if odd (1 for a single step).  A call that needs more than the
+ *     16 MiB returns TRV_ERR_TOO_LARGE and launches nothing; other plan kinds return UNSUPPORTED.
+ *   - The first call on each device looks up the array's device address (once per device, with that
+ *     device current).  Make that first call outside any stream capture.
+ *   - All calls in the process share the one array, and it keeps whatever the last call left in it.
+ *     Nothing in it has to start at zero (every step writes what it later reads), but two calls that
+ *     overlap on the GPU (different streams, or different host threads without ordering) race on
+ *     it: order them yourself. */
+trv_status_t trv_allreduce_noalloc(trv_plan_t plan, void *const *rank_buffers, size_t count, trv_dtype_t dtype,
+                                   trv_op_t op, void *cuda_stream);
+size_t trv_noalloc_max_scratch_bytes(void);
 
 /* ---------------------------------------------------------------- link loads
  *

@@ -19,7 +19,7 @@ SUM = 0
 KERNEL_AUTO, KERNEL_STEP, KERNEL_FUSED = 0, 1, 2
 MAX_RANKS = 1024
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_UNDEFINED_SCHEDULE, ERR_ALLOC, ERR_CUDA, ERR_SCRATCH = range(7)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_UNDEFINED_SCHEDULE, ERR_ALLOC, ERR_CUDA, ERR_SCRATCH, ERR_TOO_LARGE = range(8)
 
 # every symbol include/trivance.h declares
 SYMBOLS = [
@@ -27,6 +27,7 @@ SYMBOLS = [
     "trv_plan_peers", "trv_plan_send_set", "trv_plan_block_bounds", "trv_allreduce", "trv_scratch_bytes",
     "trv_kernel_supported", "trv_allreduce_ex", "trv_allreduce_host", "trv_host_workspace_bytes",
     "trv_link_loads", "trv_plan_message_bytes", "trv_strerror", "trv_launch_count", "trv_last_kernel_name",
+    "trv_allreduce_noalloc", "trv_noalloc_max_scratch_bytes",
 ]
 
 _lib = None
@@ -61,6 +62,9 @@ def lib():
         L.trv_kernel_supported.argtypes = [vp, ctypes.c_int]
         L.trv_kernel_supported.restype = i32
         L.trv_allreduce_ex.argtypes = [vp, vp, vp, sz, sz, sz, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, sz, vp]
+        L.trv_allreduce_noalloc.argtypes = [vp, vp, sz, ctypes.c_int, ctypes.c_int, vp]
+        L.trv_noalloc_max_scratch_bytes.argtypes = []
+        L.trv_noalloc_max_scratch_bytes.restype = sz
         L.trv_allreduce_host.argtypes = [vp, vp, vp, sz, ctypes.c_int, ctypes.c_int, vp, sz, vp]
         L.trv_host_workspace_bytes.argtypes = [vp, sz, ctypes.POINTER(sz)]
         L.trv_link_loads.argtypes = [vp, sz, sz, vp, vp, vp, vp]
@@ -76,6 +80,10 @@ def lib():
 
 def strerror(status):
     return lib().trv_strerror(int(status)).decode()
+
+
+def noalloc_max_scratch_bytes():
+    return int(lib().trv_noalloc_max_scratch_bytes())
 
 
 def launch_count():
@@ -177,6 +185,13 @@ class Plan:
         _check(lib().trv_allreduce_ex(self._h, a_in, a_out, count, gc, global_offset, int(dtype), int(op), int(kernel),
                                       ctypes.c_void_p(int(scratch_ptr)), scratch_bytes, ctypes.c_void_p(int(stream))),
                "trv_allreduce_ex")
+
+    def allreduce_noalloc(self, rank_ptrs, count, dtype, stream=0, op=SUM):
+        """trv_allreduce_noalloc: in-place latency-form AllReduce whose scratch is a fixed array inside the
+        library (16 MiB), for callers that may not allocate device memory.  Calls sharing a GPU must not overlap."""
+        arr = _ptr_array(rank_ptrs)
+        _check(lib().trv_allreduce_noalloc(self._h, arr, count, int(dtype), int(op), ctypes.c_void_p(int(stream))),
+               "trv_allreduce_noalloc")
 
     def allreduce_host(self, host_in_ptrs, host_out_ptrs, count, dtype, workspace_ptr, workspace_bytes, stream=0, op=SUM):
         a_in = _ptr_array(host_in_ptrs)

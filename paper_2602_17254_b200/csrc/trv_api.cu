@@ -258,6 +258,7 @@ const char* trv_strerror(trv_status_t status) {
         case TRV_ERR_ALLOC: return "allocation failed";
         case TRV_ERR_CUDA: return "CUDA runtime error";
         case TRV_ERR_SCRATCH: return "scratch or workspace too small or misaligned";
+        case TRV_ERR_TOO_LARGE: return "size exceeds the fixed scratch capacity of the no-allocation entry point";
     }
     return "unknown status";
 }

@@ -32,11 +32,11 @@ def test_header_symbols_are_exported(library):
 
 def test_strerror_covers_every_status(library):
     seen = set()
-    for s in range(7):
+    for s in range(8):
         msg = binding.strerror(s)
         assert msg and msg != "unknown status"
         seen.add(msg)
-    assert len(seen) == 7
+    assert len(seen) == 8
     assert binding.strerror(99) == "unknown status"
 
 
