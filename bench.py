@@ -242,8 +242,8 @@ def run_ours(args, w):
         g.manual_seed(1000 * w.seed + rank)
         for b in range(batch):
             ins[b].normal_(generator=g) if w.dist == "normal" else ins[b].uniform_(-1.0, 1.0, generator=g)
-    in_ptrs = [[ins[b, r].data_ptr() for r in range(n)] for b in range(batch)]
-    out_ptrs = [[outs[b, r].data_ptr() for r in range(n)] for b in range(batch)]
+    in_ptrs = [binding.ptr_array([ins[b, r].data_ptr() for r in range(n)]) for b in range(batch)]
+    out_ptrs = [binding.ptr_array([outs[b, r].data_ptr() for r in range(n)]) for b in range(batch)]
     need = plan.scratch_bytes(count, binding.KERNEL_AUTO, in_place=False)
     scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
@@ -276,7 +276,7 @@ def run_ours(args, w):
     launches = binding.launch_count() - l0
     ms = ev0.elapsed_time(ev1)
     note = "sampled during the timed region"
-    if len(sampler.samples) < 8:        # region too short for NVML: keep the same load running ~0.4 s more
+    if len(sampler.samples) < 8 and not args.profile:        # region too short for NVML: keep the same load running ~0.4 s more
         t_end = time.perf_counter() + 0.4
         while time.perf_counter() < t_end:
             step()
@@ -304,8 +304,8 @@ def run_ours(args, w):
     wsb = plan.host_workspace_bytes(count)
     ws = [torch.empty(wsb, dtype=torch.uint8, device=dev) for _ in range(2)]
     streams = [torch.cuda.Stream(), torch.cuda.Stream()]
-    hin_p = [[hin[b][r].data_ptr() for r in range(n)] for b in range(e2e_sets)]
-    hout_p = [[hout[b][r].data_ptr() for r in range(n)] for b in range(e2e_sets)]
+    hin_p = [binding.ptr_array([hin[b][r].data_ptr() for r in range(n)]) for b in range(e2e_sets)]
+    hout_p = [binding.ptr_array([hout[b][r].data_ptr() for r in range(n)]) for b in range(e2e_sets)]
 
     def e2e_step():
         for b in range(e2e_sets):
@@ -391,10 +391,17 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-check", action="store_true", help="skip the parity spot check")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--count", type=int, default=0, help="override the workload's elements per rank")
+    ap.add_argument("--profile", action="store_true",
+                    help="for runs under ncu: only warm-up and timed launches (implies --no-cpu --no-check --no-e2e)")
     args = ap.parse_args()
+    if args.profile:
+        args.no_cpu = args.no_check = args.no_e2e = True
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     w = synth.CONFIGS[args.workload]
+    if args.count:      # same topology and form, shorter vectors (small cases for ncu captures)
+        w = synth.Workload(w.name + "@%d" % args.count, w.dims, w.variant, args.count, w.dist, w.seed)
     if args.impl == "reference":
         run_reference(args, w)
     else:

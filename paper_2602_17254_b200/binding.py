@@ -99,9 +99,15 @@ def _check(status, what):
         raise TrivanceError(status, what)
 
 
-def _ptr_array(ptrs):
-    arr = (ctypes.c_void_p * len(ptrs))(*[int(p) for p in ptrs])
-    return arr
+def ptr_array(ptrs):
+    """HOST array of pointers in the form the C ABI takes.  Build it once and pass it to the Plan's
+    calls instead of a list when the same buffers are used repeatedly (saves the per-call conversion)."""
+    if isinstance(ptrs, ctypes.Array):
+        return ptrs
+    return (ctypes.c_void_p * len(ptrs))(*[int(p) for p in ptrs])
+
+
+_ptr_array = ptr_array
 
 
 def _np_ptr(a):

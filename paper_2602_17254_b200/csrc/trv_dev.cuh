@@ -4,6 +4,7 @@
 
 #include <atomic>
 #include <cstdint>
+#include <type_traits>
 
 #include "trv_plan.h"
 
@@ -43,6 +44,64 @@ __device__ __forceinline__ float add3(float a, float b, float c) { return __fadd
 __device__ __forceinline__ uint32_t add3(uint32_t a, uint32_t b, uint32_t c) { return (a + b) + c; }
 __device__ __forceinline__ float add2(float a, float b) { return __fadd_rn(a, b); }
 __device__ __forceinline__ uint32_t add2(uint32_t a, uint32_t b) { return a + b; }
+
+// Two binary32 adds in one instruction (sm_100 packed FP32): each lane is an independent IEEE add,
+// round to nearest even, no flush to zero -- bit-identical to two scalar adds, half the issue slots.
+__device__ __forceinline__ float2 add2_f32x2(float2 a, float2 b) {
+    unsigned long long ra = *reinterpret_cast<unsigned long long*>(&a);
+    unsigned long long rb = *reinterpret_cast<unsigned long long*>(&b);
+    unsigned long long rd;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
+    return *reinterpret_cast<float2*>(&rd);
+}
+
+// V consecutive elements of one rank
+template <typename T, int V>
+struct alignas(sizeof(T) * V) Elem {
+    T x[V];
+};
+
+template <typename T, int V>
+__device__ __forceinline__ Elem<T, V> add2(const Elem<T, V>& a, const Elem<T, V>& b) {
+    Elem<T, V> r;
+    if constexpr (std::is_same<T, float>::value && V % 2 == 0) {      // even width: packed adds
+#pragma unroll
+        for (int k = 0; k < V; k += 2) {
+            const float2 s = add2_f32x2(make_float2(a.x[k], a.x[k + 1]), make_float2(b.x[k], b.x[k + 1]));
+            r.x[k] = s.x;
+            r.x[k + 1] = s.y;
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < V; ++k) r.x[k] = add2(a.x[k], b.x[k]);
+    }
+    return r;
+}
+template <typename T, int V>
+__device__ __forceinline__ Elem<T, V> add3(const Elem<T, V>& a, const Elem<T, V>& b, const Elem<T, V>& c) {
+    return add2(add2(a, b), c);
+}
+
+// Where rank r's buffer starts: either a table of n pointers in parameter space, or, when the
+// caller's buffers are equally spaced (rows of one tensor), base + r * stride with no table at all.
+template <int CAP>
+struct TabAddr {
+    PtrTab<CAP> t;
+    __device__ __forceinline__ char* ptr(int rank) const { return (char*)t.p[rank]; }
+};
+struct StrideAddr {
+    char* base;
+    long long stride;   // bytes
+    __device__ __forceinline__ char* ptr(int rank) const { return base + (long long)rank * stride; }
+};
+// true (and base/stride filled) iff p[r] == p[0] + r * stride for all r
+inline bool uniform_stride(const void* const* p, int n, StrideAddr* out) {
+    out->base = (char*)const_cast<void*>(p[0]);
+    out->stride = n > 1 ? (long long)((const char*)p[1] - (const char*)p[0]) : 0;
+    for (int r = 2; r < n; ++r)
+        if ((const char*)p[r] - (const char*)p[r - 1] != out->stride) return false;
+    return true;
+}
 
 template <typename T> struct Vec4;
 template <> struct Vec4<float> { using type = float4; };

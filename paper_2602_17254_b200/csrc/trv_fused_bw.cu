@@ -15,7 +15,7 @@
 
 namespace trv {
 
-constexpr int kBwThreads = 256;
+constexpr int kBwThreads = 128;
 constexpr int kBwMaxD = 4;
 constexpr int kBwMaxS = 6;
 
@@ -28,30 +28,27 @@ struct BwArgs {
     int ldim[kBwMaxD][kBwMaxS], ldist[kBwMaxD][kBwMaxS];   // per slice, per step: dimension, distance
 };
 
-template <typename T, int V>
-struct alignas(sizeof(T) * V) Pack {
-    T x[V];
-};
-template <typename T, int V>
-__device__ __forceinline__ Pack<T, V> padd(const Pack<T, V>& a, const Pack<T, V>& b) {
-    Pack<T, V> r;
-#pragma unroll
-    for (int k = 0; k < V; ++k) r.x[k] = add2(a.x[k], b.x[k]);
-    return r;
-}
-template <typename T, int V>
-__device__ __forceinline__ Pack<T, V> padd3(const Pack<T, V>& a, const Pack<T, V>& b, const Pack<T, V>& c) {
-    return padd(padd(a, b), c);
-}
-
 __device__ __forceinline__ int wrap(int x, int a) { return x < 0 ? x + a : (x >= a ? x - a : x); }
 
+// rank -> buffer start: a pointer table staged in shared memory, or base + rank * stride
+template <typename T>
+struct SmemTabs {
+    const T* const* sin;
+    T* const* sout;
+    __device__ __forceinline__ const T* in(int r) const { return sin[r]; }
+    __device__ __forceinline__ T* out(int r) const { return sout[r]; }
+};
+template <typename T>
+struct StrideTabs {
+    StrideAddr i, o;
+    __device__ __forceinline__ const T* in(int r) const { return reinterpret_cast<const T*>(i.ptr(r)); }
+    __device__ __forceinline__ T* out(int r) const { return reinterpret_cast<T*>(o.ptr(r)); }
+};
+
 // Value of block owner j for the V columns starting at local element e, written to all ranks.
-template <typename T, int V, int S, int D>
-__device__ __forceinline__ void column_tree(const BwArgs& a, int c, const T* const* sin, T* const* sout, long long e, int j) {
-    using P = Pack<T, V>;
-    constexpr int N = (S == 1) ? 3 : (S == 2 ? 9 : 0);
-    (void)N;
+template <typename T, int V, int S, int D, typename Tabs>
+__device__ __forceinline__ void column_tree(const BwArgs& a, int c, const Tabs& tabs, long long e, int j) {
+    using P = Elem<T, V>;
     int base[D];    // coordinates of the centre of the current nine-leaf chunk
 #pragma unroll
     for (int d = 0; d < D; ++d) base[d] = (j / a.dstride[d]) % a.dims[d];
@@ -61,10 +58,10 @@ __device__ __forceinline__ void column_tree(const BwArgs& a, int c, const T* con
         int bd = 0, ad = 1, sd = 1;
 #pragma unroll
         for (int d = 0; d < D; ++d) if (d == d0) { bd = base[d]; ad = a.dims[d]; sd = a.dstride[d]; }
-        const P l = *reinterpret_cast<const P*>(sin[j + (wrap(bd - x0, ad) - bd) * sd] + e);
-        const P m = *reinterpret_cast<const P*>(sin[j] + e);
-        const P r = *reinterpret_cast<const P*>(sin[j + (wrap(bd + x0, ad) - bd) * sd] + e);
-        res = padd3(l, m, r);
+        const P l = *reinterpret_cast<const P*>(tabs.in(j + (wrap(bd - x0, ad) - bd) * sd) + e);
+        const P m = *reinterpret_cast<const P*>(tabs.in(j) + e);
+        const P r = *reinterpret_cast<const P*>(tabs.in(j + (wrap(bd + x0, ad) - bd) * sd) + e);
+        res = add3(l, m, r);
     } else {
         // start at the leftmost chunk: every step >= 2 at eps = -1
 #pragma unroll
@@ -74,12 +71,8 @@ __device__ __forceinline__ void column_tree(const BwArgs& a, int c, const T* con
             for (int d = 0; d < D; ++d) if (d == dt) base[d] = wrap(base[d] - xt, a.dims[d]);
         }
         const int d0 = a.ldim[c][0], x0 = a.ldist[c][0], d1 = a.ldim[c][1], x1 = a.ldist[c][1];
-        int dg[S];      // digit (child number) of each level >= 2
-        P acc[S];
-#pragma unroll
-        for (int t = 0; t < S; ++t) dg[t] = 0;
-        constexpr int CHUNKS = (S == 2) ? 1 : (S == 3 ? 3 : (S == 4 ? 9 : (S == 5 ? 27 : 81)));
-        for (int ch = 0; ch < CHUNKS; ++ch) {
+        // the nine leaves of the chunk centred at base[]: leaf m <-> (eps_1, eps_0) = (m / 3 - 1, m % 3 - 1)
+        auto load_chunk = [&](P (&l)[9]) {
             int rank_c = 0, b0 = 0, a0 = 1, s0 = 1, b1 = 0, a1 = 1, s1 = 1;
 #pragma unroll
             for (int d = 0; d < D; ++d) {
@@ -101,22 +94,43 @@ __device__ __forceinline__ void column_tree(const BwArgs& a, int c, const T* con
 #pragma unroll
                 for (int m = 0; m < 9; ++m) rk[m] = rank_c + (wrap(b0 + (m / 3 - 1) * x1 + (m % 3 - 1) * x0, a0) - b0) * s0;
             }
+#pragma unroll
+            for (int m = 0; m < 9; ++m) l[m] = *reinterpret_cast<const P*>(tabs.in(rk[m]) + e);
+        };
+        int pd[S], vd[S];   // position / value digit (child number) of each level >= 2
+        P acc[S];
+#pragma unroll
+        for (int t = 0; t < S; ++t) { pd[t] = 0; vd[t] = 0; }
+        constexpr int CHUNKS = (S == 2) ? 1 : (S == 3 ? 3 : (S == 4 ? 9 : (S == 5 ? 27 : 81)));
+        P nxt[9];
+        load_chunk(nxt);
+        for (int ch = 0; ch < CHUNKS; ++ch) {
             P l[9];
 #pragma unroll
-            for (int m = 0; m < 9; ++m) l[m] = *reinterpret_cast<const P*>(sin[rk[m]] + e);
-            P r = padd3(padd3(l[0], l[1], l[2]), padd3(l[3], l[4], l[5]), padd3(l[6], l[7], l[8]));
-            // carry the finished 9-leaf subtree up the tree
+            for (int m = 0; m < 9; ++m) l[m] = nxt[m];
+            // move to the next chunk and start its loads before reducing this one
+            bool go = true;
+#pragma unroll
+            for (int t = 2; t < S; ++t) {
+                if (go) {
+                    const int dt = a.ldim[c][t], xt = a.ldist[c][t];
+                    int delta;
+                    if (pd[t] < 2) { pd[t]++; delta = xt; go = false; }
+                    else { pd[t] = 0; delta = -2 * xt; }
+#pragma unroll
+                    for (int d = 0; d < D; ++d) if (d == dt) base[d] = wrap(base[d] + delta, a.dims[d]);
+                }
+            }
+            if (ch + 1 < CHUNKS) load_chunk(nxt);
+            P r = add3(add3(l[0], l[1], l[2]), add3(l[3], l[4], l[5]), add3(l[6], l[7], l[8]));
+            // carry the finished 9-leaf subtree up the tree: (first + second) + third at every level
             bool carry = true;
 #pragma unroll
             for (int t = 2; t < S; ++t) {
                 if (carry) {
-                    const int dt = a.ldim[c][t], xt = a.ldist[c][t];
-                    int delta;
-                    if (dg[t] == 0) { acc[t] = r; dg[t] = 1; delta = xt; carry = false; }
-                    else if (dg[t] == 1) { acc[t] = padd(acc[t], r); dg[t] = 2; delta = xt; carry = false; }
-                    else { r = padd(acc[t], r); dg[t] = 0; delta = -2 * xt; }
-#pragma unroll
-                    for (int d = 0; d < D; ++d) if (d == dt) base[d] = wrap(base[d] + delta, a.dims[d]);
+                    if (vd[t] == 0) { acc[t] = r; vd[t] = 1; carry = false; }
+                    else if (vd[t] == 1) { acc[t] = add2(acc[t], r); vd[t] = 2; carry = false; }
+                    else { r = add2(acc[t], r); vd[t] = 0; }
                 }
             }
             res = r;    // after the last chunk the carry has run through every level
@@ -124,7 +138,35 @@ __device__ __forceinline__ void column_tree(const BwArgs& a, int c, const T* con
     }
     // AllGather: the owner's value goes to every rank
 #pragma unroll 9
-    for (int r = 0; r < a.n; ++r) *reinterpret_cast<P*>(sout[r] + e) = res;
+    for (int r = 0; r < a.n; ++r) *reinterpret_cast<P*>(tabs.out(r) + e) = res;
+}
+
+template <typename T, int V, int S, int D, typename Tabs>
+__device__ __forceinline__ void bw_tile(const BwArgs& a, const Tabs& tabs) {
+    const int c = blockIdx.y;
+    const long long lo = a.lo[c], hi = a.hi[c];
+    // tiles start on multiples of 32*V elements: a warp's access to one rank is one aligned run
+    const long long e = (lo / (32 * V)) * (32 * V) + ((long long)blockIdx.x * kBwThreads + threadIdx.x) * V;
+    if (e >= hi || e + V <= lo) return;
+    const unsigned long long L = (unsigned long long)(a.ghi[c] - a.glo[c]);
+    auto owner = [&](long long el) -> int {
+        const unsigned long long x = (unsigned long long)(a.w0 + el - a.glo[c]);
+        return (int)(((x + 1) * (unsigned)a.n - 1) / L);
+    };
+    if constexpr (V == 1) {
+        column_tree<T, 1, S, D>(a, c, tabs, e, owner(e));
+    } else {
+        const bool inside = e >= lo && e + V <= hi;
+        int j0 = 0;
+        bool same = false;
+        if (inside) { j0 = owner(e); same = owner(e + V - 1) == j0; }
+        if (same) {
+            column_tree<T, V, S, D>(a, c, tabs, e, j0);
+        } else {
+            for (int k = 0; k < V; ++k)
+                if (e + k >= lo && e + k < hi) column_tree<T, 1, S, D>(a, c, tabs, e + k, owner(e + k));
+        }
+    }
 }
 
 template <typename T, int V, int S, int D, int CAP>
@@ -133,29 +175,12 @@ __global__ void __launch_bounds__(kBwThreads) k_bw_fused(PtrTab<CAP> in, PtrTab<
     __shared__ T* sout[CAP];
     for (int r = threadIdx.x; r < a.n; r += kBwThreads) { sin[r] = (const T*)in.p[r]; sout[r] = (T*)out.p[r]; }
     __syncthreads();
-    const int c = blockIdx.y;
-    const long long lo = a.lo[c], hi = a.hi[c];
-    const long long e = ((lo / V) + (long long)blockIdx.x * kBwThreads + threadIdx.x) * V;
-    if (e >= hi) return;
-    const unsigned long long L = (unsigned long long)(a.ghi[c] - a.glo[c]);
-    auto owner = [&](long long el) -> int {
-        const unsigned long long x = (unsigned long long)(a.w0 + el - a.glo[c]);
-        return (int)(((x + 1) * (unsigned)a.n - 1) / L);
-    };
-    if constexpr (V == 1) {
-        if (e >= lo) column_tree<T, 1, S, D>(a, c, sin, sout, e, owner(e));
-    } else {
-        const bool inside = e >= lo && e + V <= hi;
-        int j0 = 0;
-        bool same = false;
-        if (inside) { j0 = owner(e); same = owner(e + V - 1) == j0; }
-        if (same) {
-            column_tree<T, V, S, D>(a, c, sin, sout, e, j0);
-        } else {
-            for (int k = 0; k < V; ++k)
-                if (e + k >= lo && e + k < hi) column_tree<T, 1, S, D>(a, c, sin, sout, e + k, owner(e + k));
-        }
-    }
+    bw_tile<T, V, S, D>(a, SmemTabs<T>{sin, sout});
+}
+
+template <typename T, int V, int S, int D>
+__global__ void __launch_bounds__(kBwThreads) k_bw_fused_strided(StrideAddr in, StrideAddr out, BwArgs a) {
+    bw_tile<T, V, S, D>(a, StrideTabs<T>{in, out});
 }
 
 // ------------------------------------------------------------------ host side
@@ -168,15 +193,20 @@ template <typename T, int V, int S, int D>
 static void launch_bw(const Call& c, const BwArgs& a) {
     constexpr int CAP = S <= 3 ? 32 : (S <= 5 ? 256 : TRV_MAX_RANKS);
     const Plan& p = *c.plan;
-    PtrTab<CAP> in, out;
-    for (int r = 0; r < p.n; ++r) { in.p[r] = const_cast<void*>(c.in[r]); out.p[r] = c.out[r]; }
     long long tiles = 0;
     for (int sl = 0; sl < D; ++sl)
         if (a.hi[sl] > a.lo[sl]) {
-            long long t = (a.hi[sl] - (a.lo[sl] / V) * V + (long long)V * kBwThreads - 1) / ((long long)V * kBwThreads);
+            long long t = (a.hi[sl] - (a.lo[sl] / (32 * V)) * (32 * V) + (long long)V * kBwThreads - 1) / ((long long)V * kBwThreads);
             if (t > tiles) tiles = t;
         }
     if (tiles == 0) return;
+    StrideAddr sin, sout;
+    if (uniform_stride(c.in, p.n, &sin) && uniform_stride((const void* const*)c.out, p.n, &sout)) {
+        TRV_LAUNCH((k_bw_fused_strided<T, V, S, D>), dim3((unsigned)tiles, D, 1), kBwThreads, 0, c.st, sin, sout, a);
+        return;
+    }
+    PtrTab<CAP> in, out;
+    for (int r = 0; r < p.n; ++r) { in.p[r] = const_cast<void*>(c.in[r]); out.p[r] = c.out[r]; }
     TRV_LAUNCH((k_bw_fused<T, V, S, D, CAP>), dim3((unsigned)tiles, D, 1), kBwThreads, 0, c.st, in, out, a);
 }
 

@@ -7,13 +7,15 @@
 // every step maps the set onto itself, e.g. the ranks {q + 9 i} of a ring under the steps
 // with distances 9, 27, 81.  Inside a closed group a step is a compile-time permutation of
 // registers plus two adds per value; between groups the column tile goes through shared
-// memory once (lane = element column, so every access is bank-conflict free).
+// memory once.  A thread owns V adjacent columns, so float adds issue as packed f32x2.
 //
 //   k_lat_reg   : n <= 81 (rings 3..81, tori 3x3, 9x9, 3x3x3, 3x3x3x3): one group, no shared memory
 //   k_lat_ring  : rings of 243 and 729: steps {1,3} on windows of consecutive ranks with a
 //                 halo of 4, then the remaining steps on the closed sets {q + 9 i}
 //   k_lat_t999  : 9x9x9 torus: steps (A,1)(B,1) on 9x9 planes, then (C,1)(A,3)(B,3)(C,3) on the
 //                 3x3x9 closed sets; A,B,C = the slice's dimension order
+#include <type_traits>
+
 #include "trv_dev.cuh"
 
 namespace trv {
@@ -22,24 +24,14 @@ constexpr int ipow3(int e) { return e <= 0 ? 1 : 3 * ipow3(e - 1); }
 constexpr int ipow(int b, int e) { return e <= 0 ? 1 : b * ipow(b, e - 1); }
 constexpr int ilog3(int n) { return n <= 1 ? 0 : 1 + ilog3(n / 3); }
 
-// V consecutive elements of one rank
-template <typename T, int V>
-struct alignas(sizeof(T) * V) Elem {
-    T x[V];
-};
-
-template <typename T, int V>
-__device__ __forceinline__ Elem<T, V> add3(const Elem<T, V>& a, const Elem<T, V>& b, const Elem<T, V>& c) {
+// FULL is a compile-time property of the whole tile (every column of the CTA lies inside the
+// slice): the common case is then straight-line code whose loads the compiler can batch; only the
+// one or two edge tiles of a slice take the masked, element-by-element form.
+template <typename T, int V, bool FULL>
+__device__ __forceinline__ Elem<T, V> load_elem(const char* row, long long e, long long lo, long long hi) {
+    const T* p = reinterpret_cast<const T*>(row);
     Elem<T, V> r;
-#pragma unroll
-    for (int k = 0; k < V; ++k) r.x[k] = add3(a.x[k], b.x[k], c.x[k]);
-    return r;
-}
-
-template <typename T, int V>
-__device__ __forceinline__ Elem<T, V> load_elem(const T* p, long long e, long long lo, long long hi, bool full) {
-    Elem<T, V> r;
-    if (full) {
+    if constexpr (FULL) {
         r = *reinterpret_cast<const Elem<T, V>*>(p + e);
     } else {
 #pragma unroll
@@ -47,9 +39,10 @@ __device__ __forceinline__ Elem<T, V> load_elem(const T* p, long long e, long lo
     }
     return r;
 }
-template <typename T, int V>
-__device__ __forceinline__ void store_elem(T* p, long long e, long long lo, long long hi, bool full, const Elem<T, V>& v) {
-    if (full) {
+template <typename T, int V, bool FULL>
+__device__ __forceinline__ void store_elem(char* row, long long e, long long lo, long long hi, const Elem<T, V>& v) {
+    T* p = reinterpret_cast<T*>(row);
+    if constexpr (FULL) {
         *reinterpret_cast<Elem<T, V>*>(p + e) = v;
     } else {
 #pragma unroll
@@ -91,22 +84,20 @@ __device__ __forceinline__ void reg_all_steps(E (&v)[N]) {
     }
 }
 
-template <typename T, int A, int D, int V, int THREADS, int CAP>
-__global__ void __launch_bounds__(THREADS) k_lat_reg(PtrTab<CAP> in, PtrTab<CAP> out, LatArgs a) {
+// Tiles start on multiples of 32*V elements of the buffers (128*V bytes) so that a warp's
+// access to one rank is one aligned, contiguous run.
+template <typename T, int A, int D, int V, bool FULL, typename Addr>
+__device__ __forceinline__ void lat_reg_body(const Addr& in, const Addr& out, const LatArgs& a, int c, long long e) {
     constexpr int N = ipow(A, D);
     using E = Elem<T, V>;
-    const int c = blockIdx.y;
     const long long lo = a.lo[c], hi = a.hi[c];
-    const long long e = ((lo / V) + (long long)blockIdx.x * THREADS + threadIdx.x) * V;
-    if (e >= hi) return;
-    const bool full = e >= lo && e + V <= hi;
     E v[N];
 #pragma unroll
     for (int idx = 0; idx < N; ++idx) {
         int rank = 0, rem = idx;
 #pragma unroll
         for (int k = 0; k < D; ++k) { rank += (rem % A) * a.rs[c][k]; rem /= A; }
-        v[idx] = load_elem<T, V>((const T*)in.p[rank], e, lo, hi, full);
+        v[idx] = load_elem<T, V, FULL>(in.ptr(rank), e, lo, hi);
     }
     reg_all_steps<A, D, 0>(v);
 #pragma unroll
@@ -114,7 +105,20 @@ __global__ void __launch_bounds__(THREADS) k_lat_reg(PtrTab<CAP> in, PtrTab<CAP>
         int rank = 0, rem = idx;
 #pragma unroll
         for (int k = 0; k < D; ++k) { rank += (rem % A) * a.rs[c][k]; rem /= A; }
-        store_elem<T, V>((T*)out.p[rank], e, lo, hi, full, v[idx]);
+        store_elem<T, V, FULL>(out.ptr(rank), e, lo, hi, v[idx]);
+    }
+}
+
+template <typename T, int A, int D, int V, int THREADS, typename Addr>
+__global__ void __launch_bounds__(THREADS) k_lat_reg(Addr in, Addr out, LatArgs a) {
+    const int c = blockIdx.y;
+    const long long lo = a.lo[c], hi = a.hi[c];
+    const long long t0 = (lo / (32 * V)) * (32 * V) + (long long)blockIdx.x * THREADS * V;    // first column of the tile
+    const long long e = t0 + (long long)threadIdx.x * V;
+    if (t0 >= lo && t0 + (long long)THREADS * V <= hi) {
+        lat_reg_body<T, A, D, V, true>(in, out, a, c, e);
+    } else if (e < hi && e + V > lo) {
+        lat_reg_body<T, A, D, V, false>(in, out, a, c, e);
     }
 }
 
@@ -128,98 +132,144 @@ __device__ __forceinline__ void ring_tail_steps(E (&v)[N]) {     // distances 1,
     }
 }
 
-template <typename T, int M, int CAP>
-__global__ void __launch_bounds__(288) k_lat_ring(PtrTab<CAP> in, PtrTab<CAP> out, LatArgs a) {
-    constexpr int NR = 9 * M;
-    extern __shared__ uint32_t slab_raw[];
-    T* slab = reinterpret_cast<T*>(slab_raw);       // [NR][32]
-    const int lane = threadIdx.x & 31, set = threadIdx.x >> 5;
+// 32-column tiles; a thread owns V adjacent columns of one of 9 rank sets: 9 * 32 / V threads.
+template <typename T, int M, int V, bool FULL, typename Addr>
+__device__ __forceinline__ void lat_ring_body(const Addr& in, const Addr& out, const LatArgs& a, T* slab, long long t0) {
+    constexpr int NR = 9 * M, LANES = 32 / V;
+    using E = Elem<T, V>;
+    const int lane = threadIdx.x % LANES, set = threadIdx.x / LANES;
     const long long lo = a.lo[0], hi = a.hi[0];
-    const long long e = (lo & ~31LL) + (long long)blockIdx.x * 32 + lane;
-    const bool valid = e >= lo && e < hi;
+    const long long e = t0 + lane * V;
+    auto sl = [&](int r) -> E& { return *reinterpret_cast<E*>(slab + r * 32 + lane * V); };
 
     // group 1: window of M consecutive ranks [set*M, set*M + M) plus a halo of 4 on each side
-    T x[M + 8];
+    E x[M + 8];
 #pragma unroll
-    for (int i = 0; i < M; ++i) {
-        const int r = set * M + i;
-        x[4 + i] = valid ? ((const T*)in.p[r])[e] : T(0);
-        slab[r * 32 + lane] = x[4 + i];
-    }
+    for (int i = 0; i < M; ++i) x[4 + i] = load_elem<T, V, FULL>(in.ptr(set * M + i), e, lo, hi);
+#pragma unroll
+    for (int i = 0; i < M; ++i) sl(set * M + i) = x[4 + i];
     __syncthreads();
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
         int rl = set * M - 4 + k; if (rl < 0) rl += NR;
         int rr = set * M + M + k; if (rr >= NR) rr -= NR;
-        x[k] = slab[rl * 32 + lane];
-        x[M + 4 + k] = slab[rr * 32 + lane];
+        x[k] = sl(rl);
+        x[M + 4 + k] = sl(rr);
     }
-    T y[M + 8];
+    E y[M + 8];
 #pragma unroll
     for (int i = 1; i < M + 7; ++i) y[i] = add3(x[i - 1], x[i], x[i + 1]);          // distance 1
     __syncthreads();                                                                // halos read
 #pragma unroll
-    for (int i = 4; i < M + 4; ++i) slab[(set * M + i - 4) * 32 + lane] = add3(y[i - 3], y[i], y[i + 3]);   // distance 3
+    for (int i = 4; i < M + 4; ++i) sl(set * M + i - 4) = add3(y[i - 3], y[i], y[i + 3]);   // distance 3
     __syncthreads();
 
     // group 2: ranks {set + 9 i}: closed under the distances 9, 27, .. ; a ring of M with distances 1, 3, ..
-    T v[M];
+    E v[M];
 #pragma unroll
-    for (int i = 0; i < M; ++i) v[i] = slab[(set + 9 * i) * 32 + lane];
+    for (int i = 0; i < M; ++i) v[i] = sl(set + 9 * i);
     ring_tail_steps<M, 0>(v);
-    if (valid) {
+    if (FULL || (e < hi && e + V > lo)) {
 #pragma unroll
-        for (int i = 0; i < M; ++i) ((T*)out.p[set + 9 * i])[e] = v[i];
+        for (int i = 0; i < M; ++i) store_elem<T, V, FULL>(out.ptr(set + 9 * i), e, lo, hi, v[i]);
     }
+}
+
+template <typename T, int M, int V, typename Addr>
+__global__ void __launch_bounds__(288 / V) k_lat_ring(Addr in, Addr out, LatArgs a) {
+    extern __shared__ uint4 slab_raw[];
+    T* slab = reinterpret_cast<T*>(slab_raw);       // [9 M][32]
+    const long long t0 = (a.lo[0] & ~31LL) + (long long)blockIdx.x * 32;
+    if (t0 >= a.lo[0] && t0 + 32 <= a.hi[0]) lat_ring_body<T, M, V, true>(in, out, a, slab, t0);   // CTA-uniform
+    else lat_ring_body<T, M, V, false>(in, out, a, slab, t0);
 }
 
 // ------------------------------------------------------------------ 9 x 9 x 9 torus
 
-template <typename T, int CAP>
-__global__ void __launch_bounds__(288, 2) k_lat_t999(PtrTab<CAP> in, PtrTab<CAP> out, LatArgs a) {
-    extern __shared__ uint32_t slab_raw[];
-    T* slab = reinterpret_cast<T*>(slab_raw);       // [729][32]
-    const int c = blockIdx.y;
-    const int lane = threadIdx.x & 31, set = threadIdx.x >> 5;
+// 32-column tiles; a thread owns 2 adjacent columns (packed adds) and one ninth of the ranks:
+// 9 * 16 = 144 threads, two CTAs per SM.  A, B, C = the slice's dimensions in its own order.
+//   group 1: steps (A,1) (B,1) on the 9x9 plane C = set, streamed row by row (a row = 9 values
+//            along A): (A,1) inside a row, (B,1) over a sliding window of three rows
+//   group 2: steps (C,1) (A,3) on the closed sets {A in a0+3i, B = j, all C}   (27 values, 3 sets per thread)
+//   group 3: steps (B,3) (C,3) on the closed sets {A = i, B in b0+3j, C in c0+3k} (9 values, 9 sets per thread)
+// Between groups the tile stays in shared memory; inside a group every set is read and written
+// by one thread only, so the two barriers between the groups are the only synchronisation.
+template <typename T, bool FULL, typename Addr>
+__device__ __forceinline__ void lat_t999_body(const Addr& in, const Addr& out, const LatArgs& a, T* slab, int c, long long t0) {
+    constexpr int V = 2, LANES = 16;
+    using E = Elem<T, V>;
+    const int lane = threadIdx.x % LANES, set = threadIdx.x / LANES;
     const long long lo = a.lo[c], hi = a.hi[c];
-    const long long e = (lo & ~31LL) + (long long)blockIdx.x * 32 + lane;
-    const bool valid = e >= lo && e < hi;
+    const long long e = t0 + lane * V;
     const int sA = a.rs[c][0], sB = a.rs[c][1], sC = a.rs[c][2];
+    auto sl = [&](int r) -> E& { return *reinterpret_cast<E*>(slab + r * 32 + lane * V); };
 
-    T v[81];
-    // group 1: plane C = set; flat index i + 9 j  <->  rank i sA + j sB + set sC; steps (A,1), (B,1)
+    {   // ---- group 1
+        auto load_row = [&](int j, E (&row)[9]) {
 #pragma unroll
-    for (int idx = 0; idx < 81; ++idx) {
-        const int rank = (idx % 9) * sA + (idx / 9) * sB + set * sC;
-        v[idx] = valid ? ((const T*)in.p[rank])[e] : T(0);
-    }
-    reg_step<81, 1, 9, 1>(v);
-    reg_step<81, 9, 9, 1>(v);
+            for (int i = 0; i < 9; ++i) row[i] = load_elem<T, V, FULL>(in.ptr(i * sA + j * sB + set * sC), e, lo, hi);
+            reg_step<9, 1, 9, 1>(row);                                      // (A,1)
+        };
+        auto emit = [&](int j, const E (&p)[9], const E (&q)[9], const E (&r)[9]) {     // (B,1) for row j
 #pragma unroll
-    for (int idx = 0; idx < 81; ++idx) {
-        const int rank = (idx % 9) * sA + (idx / 9) * sB + set * sC;
-        slab[rank * 32 + lane] = v[idx];
+            for (int i = 0; i < 9; ++i) sl(i * sA + j * sB + set * sC) = add3(p[i], q[i], r[i]);
+        };
+        E r0[9], r1[9], prev[9], cur[9], next[9];
+        load_row(0, r0);
+        load_row(1, r1);
+#pragma unroll
+        for (int i = 0; i < 9; ++i) { prev[i] = r0[i]; cur[i] = r1[i]; }
+#pragma unroll
+        for (int j = 1; j < 8; ++j) {
+            load_row(j + 1, next);
+            emit(j, prev, cur, next);
+#pragma unroll
+            for (int i = 0; i < 9; ++i) { prev[i] = cur[i]; cur[i] = next[i]; }
+        }
+        emit(8, prev, cur, r0);     // row 8: rows 7, 8, 0
+        emit(0, cur, r0, r1);       // row 0: rows 8, 0, 1
     }
     __syncthreads();
-    // group 2: A in {a0, a0+3, a0+6}, B in {b0, b0+3, b0+6}, all of C; flat index i + 3 j + 9 k;
-    // steps (C,1), (A,3), (B,3), (C,3): in this set A and B are rings of 3 with distance 1
-    const int a0 = set % 3, b0 = set / 3;
+    // ---- group 2: flat index k + 9 i  <->  rank (a0 + 3 i) sA + j sB + k sC
+#pragma unroll 1
+    for (int m = 0; m < 3; ++m) {
+        const int q = set + 9 * m, a0 = q % 3, j = q / 3;
+        E v[27];
 #pragma unroll
-    for (int idx = 0; idx < 81; ++idx) {
-        const int rank = (a0 + 3 * (idx % 3)) * sA + (b0 + 3 * ((idx / 3) % 3)) * sB + (idx / 9) * sC;
-        v[idx] = slab[rank * 32 + lane];
+        for (int idx = 0; idx < 27; ++idx) v[idx] = sl((a0 + 3 * (idx / 9)) * sA + j * sB + (idx % 9) * sC);
+        reg_step<27, 1, 9, 1>(v);       // (C,1)
+        reg_step<27, 9, 3, 1>(v);       // (A,3): a ring of three with distance one inside this set
+#pragma unroll
+        for (int idx = 0; idx < 27; ++idx) sl((a0 + 3 * (idx / 9)) * sA + j * sB + (idx % 9) * sC) = v[idx];
     }
-    reg_step<81, 9, 9, 1>(v);
-    reg_step<81, 1, 3, 1>(v);
-    reg_step<81, 3, 3, 1>(v);
-    reg_step<81, 9, 9, 3>(v);
-    if (valid) {
+    __syncthreads();
+    // ---- group 3: flat index jj + 3 kk  <->  rank i sA + (b0 + 3 jj) sB + (c0 + 3 kk) sC
+    const bool any = FULL || (e < hi && e + V > lo);
+#pragma unroll 1
+    for (int m = 0; m < 9; ++m) {
+        const int q = set + 9 * m, i = q % 9, b0 = (q / 9) % 3, c0 = q / 27;
+        E v[9];
 #pragma unroll
-        for (int idx = 0; idx < 81; ++idx) {
-            const int rank = (a0 + 3 * (idx % 3)) * sA + (b0 + 3 * ((idx / 3) % 3)) * sB + (idx / 9) * sC;
-            ((T*)out.p[rank])[e] = v[idx];
+        for (int idx = 0; idx < 9; ++idx) v[idx] = sl(i * sA + (b0 + 3 * (idx % 3)) * sB + (c0 + 3 * (idx / 3)) * sC);
+        reg_step<9, 1, 3, 1>(v);        // (B,3)
+        reg_step<9, 3, 3, 1>(v);        // (C,3)
+        if (any) {
+#pragma unroll
+            for (int idx = 0; idx < 9; ++idx)
+                store_elem<T, V, FULL>(out.ptr(i * sA + (b0 + 3 * (idx % 3)) * sB + (c0 + 3 * (idx / 3)) * sC), e, lo, hi, v[idx]);
         }
     }
+}
+
+template <typename T, typename Addr>
+__global__ void __launch_bounds__(144, 2) k_lat_t999(Addr in, Addr out, LatArgs a) {
+    extern __shared__ uint4 slab_raw[];
+    T* slab = reinterpret_cast<T*>(slab_raw);       // [729][32]
+    const int c = blockIdx.y;
+    const long long t0 = (a.lo[c] & ~31LL) + (long long)blockIdx.x * 32;
+    if (t0 >= a.hi[c]) return;                                                                      // CTA-uniform
+    if (t0 >= a.lo[c] && t0 + 32 <= a.hi[c]) lat_t999_body<T, true>(in, out, a, slab, c, t0);      // CTA-uniform
+    else lat_t999_body<T, false>(in, out, a, slab, c, t0);
 }
 
 // ------------------------------------------------------------------ host side
@@ -236,94 +286,72 @@ static LatKind classify(const Plan& p) {
 
 bool fused_latency_supported(const Plan& p) { return classify(p) != LatKind::None; }
 
-static void fill_args(const Call& c, LatArgs* a, long long* max_len) {
+static void fill_args(const Call& c, LatArgs* a) {
     const Plan& p = *c.plan;
     a->nslices = p.ndims;
-    *max_len = 0;
     for (int sl = 0; sl < p.ndims; ++sl) {
         local_slice(c, sl, &a->lo[sl], &a->hi[sl]);
         for (int k = 0; k < 4; ++k) a->rs[sl][k] = k < p.ndims ? p.stride[(sl + k) % p.ndims] : 0;
     }
 }
 
-template <typename T, int A, int D, int V, int THREADS, int CAP>
-static void launch_reg(const Call& c, const PtrTab<CAP>& in, const PtrTab<CAP>& out, const LatArgs& a) {
+// number of tiles of `tile` elements, starting at a multiple of `align`, that cover the longest slice
+static long long tiles_for(const LatArgs& a, int nslices, long long tile, long long align) {
     long long tiles = 0;
-    for (int sl = 0; sl < D; ++sl)
+    for (int sl = 0; sl < nslices; ++sl)
         if (a.hi[sl] > a.lo[sl]) {
-            long long t = (a.hi[sl] - (a.lo[sl] / V) * V + (long long)V * THREADS - 1) / ((long long)V * THREADS);
+            const long long t = (a.hi[sl] - (a.lo[sl] / align) * align + tile - 1) / tile;
             if (t > tiles) tiles = t;
         }
-    if (tiles == 0) return;
-    dim3 grid((unsigned)tiles, D, 1);
-    TRV_LAUNCH((k_lat_reg<T, A, D, V, THREADS, CAP>), grid, THREADS, 0, c.st, in, out, a);
+    return tiles;
 }
 
-template <typename T, int CAP>
-static trv_status_t lat_fused_impl(const Call& c) {
+template <typename T, int A, int D, int V, int THREADS, typename Addr>
+static void launch_reg(const Call& c, const Addr& in, const Addr& out, const LatArgs& a) {
+    const long long tiles = tiles_for(a, D, (long long)V * THREADS, 32 * V);
+    if (tiles == 0) return;
+    TRV_LAUNCH((k_lat_reg<T, A, D, V, THREADS, Addr>), dim3((unsigned)tiles, D, 1), THREADS, 0, c.st, in, out, a);
+}
+
+template <typename T, typename Addr>
+static trv_status_t lat_fused_launch(const Call& c, const Addr& in, const Addr& out) {
     const Plan& p = *c.plan;
-    PtrTab<CAP> in, out;
-    for (int r = 0; r < p.n; ++r) { in.p[r] = const_cast<void*>(c.in[r]); out.p[r] = c.out[r]; }
     LatArgs a;
-    long long unused;
-    fill_args(c, &a, &unused);
+    fill_args(c, &a);
     const LatKind kind = classify(p);
     if (kind == LatKind::Reg) {
         const int A = p.dims[0], D = p.ndims;
-        if constexpr (CAP == 32) {
-            if (A == 3 && D == 1) { g_last_kernel = "lat_reg<3>"; launch_reg<T, 3, 1, 4, 128>(c, in, out, a); }
-            else if (A == 9 && D == 1) { g_last_kernel = "lat_reg<9>"; launch_reg<T, 9, 1, 4, 128>(c, in, out, a); }
-            else if (A == 27 && D == 1) { g_last_kernel = "lat_reg<27>"; launch_reg<T, 27, 1, 4, 128>(c, in, out, a); }
-            else if (A == 3 && D == 2) { g_last_kernel = "lat_reg<3x3>"; launch_reg<T, 3, 2, 4, 128>(c, in, out, a); }
-            else if (A == 3 && D == 3) { g_last_kernel = "lat_reg<3x3x3>"; launch_reg<T, 3, 3, 4, 128>(c, in, out, a); }
-            else return TRV_ERR_UNSUPPORTED;
-        } else if constexpr (CAP == 256) {
-            if (A == 81 && D == 1) { g_last_kernel = "lat_reg<81>"; launch_reg<T, 81, 1, 1, 128>(c, in, out, a); }
-            else if (A == 9 && D == 2) { g_last_kernel = "lat_reg<9x9>"; launch_reg<T, 9, 2, 1, 128>(c, in, out, a); }
-            else if (A == 3 && D == 4) { g_last_kernel = "lat_reg<3x3x3x3>"; launch_reg<T, 3, 4, 1, 128>(c, in, out, a); }
-            else return TRV_ERR_UNSUPPORTED;
-        } else {
-            return TRV_ERR_UNSUPPORTED;
-        }
+        if (A == 3 && D == 1) { g_last_kernel = "lat_reg<3>"; launch_reg<T, 3, 1, 4, 64>(c, in, out, a); }
+        else if (A == 9 && D == 1) { g_last_kernel = "lat_reg<9>"; launch_reg<T, 9, 1, 4, 64>(c, in, out, a); }
+        else if (A == 27 && D == 1) { g_last_kernel = "lat_reg<27>"; launch_reg<T, 27, 1, 4, 64>(c, in, out, a); }
+        else if (A == 3 && D == 2) { g_last_kernel = "lat_reg<3x3>"; launch_reg<T, 3, 2, 4, 64>(c, in, out, a); }
+        else if (A == 3 && D == 3) { g_last_kernel = "lat_reg<3x3x3>"; launch_reg<T, 3, 3, 4, 64>(c, in, out, a); }
+        else if (A == 81 && D == 1) { g_last_kernel = "lat_reg<81>"; launch_reg<T, 81, 1, 2, 64>(c, in, out, a); }
+        else if (A == 9 && D == 2) { g_last_kernel = "lat_reg<9x9>"; launch_reg<T, 9, 2, 2, 64>(c, in, out, a); }
+        else if (A == 3 && D == 4) { g_last_kernel = "lat_reg<3x3x3x3>"; launch_reg<T, 3, 4, 2, 64>(c, in, out, a); }
+        else return TRV_ERR_UNSUPPORTED;
     } else if (kind == LatKind::Ring) {
-        if (a.hi[0] > a.lo[0]) {
-            const long long tiles = (a.hi[0] - (a.lo[0] & ~31LL) + 31) / 32;
+        const long long tiles = tiles_for(a, 1, 32, 32);
+        if (tiles > 0) {
             if (p.n == 243) {
-                if constexpr (CAP == 256) {
-                    g_last_kernel = "lat_ring<243>";
-                    TRV_LAUNCH((k_lat_ring<T, 27, CAP>), dim3((unsigned)tiles), 288, 243 * 32 * 4, c.st, in, out, a);
-                }
+                g_last_kernel = "lat_ring<243>";
+                TRV_LAUNCH((k_lat_ring<T, 27, 2, Addr>), dim3((unsigned)tiles), 144, 243 * 32 * 4, c.st, in, out, a);
             } else {
-                if constexpr (CAP == TRV_MAX_RANKS) {
-                    g_last_kernel = "lat_ring<729>";
-                    static bool attr_done[2] = {false, false};
-                    auto kfn = k_lat_ring<T, 81, CAP>;
-                    if (!attr_done[sizeof(T) == 4 && std::is_same<T, float>::value]) {
-                        cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, 729 * 32 * 4);
-                        attr_done[std::is_same<T, float>::value] = true;
-                    }
-                    TRV_LAUNCH(kfn, dim3((unsigned)tiles), 288, 729 * 32 * 4, c.st, in, out, a);
-                }
+                g_last_kernel = "lat_ring<729>";
+                auto kfn = k_lat_ring<T, 81, 1, Addr>;
+                static const cudaError_t once = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, 729 * 32 * 4);
+                (void)once;
+                TRV_LAUNCH(kfn, dim3((unsigned)tiles), 288, 729 * 32 * 4, c.st, in, out, a);
             }
         }
     } else if (kind == LatKind::T999) {
-        if constexpr (CAP == TRV_MAX_RANKS) {
-            g_last_kernel = "lat_t999";
-            long long tiles = 0;
-            for (int sl = 0; sl < 3; ++sl)
-                if (a.hi[sl] > a.lo[sl]) {
-                    long long t = (a.hi[sl] - (a.lo[sl] & ~31LL) + 31) / 32;
-                    if (t > tiles) tiles = t;
-                }
-            if (tiles > 0) {
-                auto kfn = k_lat_t999<T, CAP>;
-                static bool attr_done[2] = {false, false};
-                if (!attr_done[std::is_same<T, float>::value]) {
-                    cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, 729 * 32 * 4);
-                    attr_done[std::is_same<T, float>::value] = true;
-                }
-                TRV_LAUNCH(kfn, dim3((unsigned)tiles, 3, 1), 288, 729 * 32 * 4, c.st, in, out, a);
-            }
+        g_last_kernel = "lat_t999";
+        const long long tiles = tiles_for(a, 3, 32, 32);
+        if (tiles > 0) {
+            auto kfn = k_lat_t999<T, Addr>;
+            static const cudaError_t once = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, 729 * 32 * 4);
+            (void)once;
+            TRV_LAUNCH(kfn, dim3((unsigned)tiles, 3, 1), 144, 729 * 32 * 4, c.st, in, out, a);
         }
     } else {
         return TRV_ERR_UNSUPPORTED;
@@ -331,16 +359,24 @@ static trv_status_t lat_fused_impl(const Call& c) {
     return cudaGetLastError() == cudaSuccess ? TRV_OK : TRV_ERR_CUDA;
 }
 
-trv_status_t run_fused_latency(const Call& c) {
+template <typename T>
+static trv_status_t lat_fused_addr(const Call& c) {
     const int n = c.plan->n;
-    if (c.dtype == TRV_FLOAT32) {
-        if (n <= 32) return lat_fused_impl<float, 32>(c);
-        if (n <= 256) return lat_fused_impl<float, 256>(c);
-        return lat_fused_impl<float, TRV_MAX_RANKS>(c);
+    StrideAddr sin, sout;
+    if (uniform_stride(c.in, n, &sin) && uniform_stride((const void* const*)c.out, n, &sout))
+        return lat_fused_launch<T, StrideAddr>(c, sin, sout);
+    if (n <= 81) {      // k_lat_reg shapes
+        TabAddr<81> in, out;
+        for (int r = 0; r < n; ++r) { in.t.p[r] = const_cast<void*>(c.in[r]); out.t.p[r] = c.out[r]; }
+        return lat_fused_launch<T, TabAddr<81>>(c, in, out);
     }
-    if (n <= 32) return lat_fused_impl<uint32_t, 32>(c);
-    if (n <= 256) return lat_fused_impl<uint32_t, 256>(c);
-    return lat_fused_impl<uint32_t, TRV_MAX_RANKS>(c);
+    TabAddr<729> in, out;
+    for (int r = 0; r < n; ++r) { in.t.p[r] = const_cast<void*>(c.in[r]); out.t.p[r] = c.out[r]; }
+    return lat_fused_launch<T, TabAddr<729>>(c, in, out);
+}
+
+trv_status_t run_fused_latency(const Call& c) {
+    return c.dtype == TRV_FLOAT32 ? lat_fused_addr<float>(c) : lat_fused_addr<uint32_t>(c);
 }
 
 }  // namespace trv

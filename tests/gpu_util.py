@@ -62,6 +62,32 @@ def compare(dims, variant, x_host, got_host, E=None, e0=0):
     return want
 
 
+def check_scattered(dims, variant, count, dist, seed, kernel):
+    """Same as check_case, in place, but the rank buffers are NOT equally spaced (rows of a pool
+    in shuffled order): exercises the pointer-table addressing of the kernels."""
+    plan = binding.Plan(dims, variant)
+    n = plan.n
+    x = synth.rank_matrix(dist, seed, n, count)
+    pad = (count + 3) // 4 * 4 + 4
+    pool = torch.zeros((n + 1, pad), dtype=torch_dtype(x.dtype), device=DEV)
+    order = np.random.default_rng(seed).permutation(n + 1)[:n]
+    rows = [pool[int(order[r])] for r in range(n)]
+    for r in range(n):
+        rows[r][:count].copy_(torch.from_numpy(x[r]))
+    ptrs = [rows[r].data_ptr() for r in range(n)]
+    need = plan.scratch_bytes(count, kernel, in_place=True)
+    scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=DEV)
+    plan.allreduce_ex(ptrs, None, count, binding.INT32 if x.dtype == np.int32 else binding.FLOAT32, kernel=kernel,
+                      scratch_ptr=scratch.data_ptr() if need else 0, scratch_bytes=need,
+                      stream=torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    got = np.stack([rows[r][:count].cpu().numpy() for r in range(n)])
+    compare(dims, variant, x, got)
+    for r in range(n):
+        assert torch.count_nonzero(rows[r][count:]).item() == 0, "wrote past the end of a rank buffer"
+    plan.destroy()
+
+
 def check_case(dims, variant, count, dist, seed, kernel, in_place=True, shard=None):
     """Full element-by-element parity on a case the oracle finishes quickly.
     shard = (global_count, global_offset): the buffers hold only that window of a longer vector."""

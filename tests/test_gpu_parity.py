@@ -10,7 +10,7 @@ import torch
 import oracle
 from paper_2602_17254_b200 import binding, build, synth
 
-from gpu_util import DEV, check_case, compare, run_gpu, torch_dtype, upload_matrix
+from gpu_util import DEV, check_case, check_scattered, compare, run_gpu, torch_dtype, upload_matrix
 
 pytestmark = pytest.mark.gpu
 
@@ -36,6 +36,7 @@ def test_step_family_matches_oracle(dims, variant):
     count = 1531 if n <= 243 else 517
     check_case(dims, variant, count, "normal", 11, STEP)
     check_case(dims, variant, count, "int32", 12, STEP, in_place=False)
+    check_scattered(dims, variant, count, "normal", 13, STEP)
 
 
 @pytest.mark.parametrize("dims", FUSED_LAT)
@@ -44,6 +45,8 @@ def test_fused_latency_matches_oracle(dims):
     count = 4133 if n <= 243 else 1029          # several tiles of every kernel + ragged tail
     check_case(dims, LAT, count, "normal", 21, FUSED)
     check_case(dims, LAT, count, "int32", 22, FUSED, in_place=False)
+    check_scattered(dims, LAT, count, "normal", 23, FUSED)
+    check_scattered(dims, LAT, count, "int32", 24, FUSED)
 
 
 @pytest.mark.parametrize("dims", ANY)
@@ -53,10 +56,12 @@ def test_fused_bandwidth_matches_oracle(dims):
     small = 1531 if n <= 243 else 517                     # one column per thread (short blocks)
     check_case(dims, BW, small, "normal", 31, FUSED)
     check_case(dims, BW, small, "int32", 32, FUSED, in_place=False)
+    check_scattered(dims, BW, small, "normal", 36, FUSED)
     if n <= 81:                                           # four columns per thread (blocks >= 256 elements)
         wide = 300 * n * D + 7
         check_case(dims, BW, wide, "normal", 33, FUSED)
         check_case(dims, BW, wide, "int32", 34, FUSED, in_place=False)
+        check_scattered(dims, BW, wide, "int32", 37, FUSED)
 
 
 def test_fused_bandwidth_wide_path_on_729_ranks_sampled():
