@@ -39,6 +39,26 @@ extern thread_local const char* g_last_kernel;
         ::trv::g_launches.fetch_add(1, std::memory_order_relaxed);        \
     } while (0)
 
+// Programmatic dependent launch: a kernel launched with TRV_LAUNCH_PDL may become resident while
+// the previous kernel of the stream is still draining.  pdl_trigger() (first thing in a kernel)
+// lets the NEXT kernel do that; pdl_wait() (before the first global-memory access) blocks until the
+// PREVIOUS kernel has completed and its writes are visible, so stream order is fully preserved:
+// only launch latency and the prologue overlap.  Both are no-ops without the launch attribute.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+}
+
 // (a + b) + c, one rounding per add, never contracted or reassociated.
 __device__ __forceinline__ float add3(float a, float b, float c) { return __fadd_rn(__fadd_rn(a, b), c); }
 __device__ __forceinline__ uint32_t add3(uint32_t a, uint32_t b, uint32_t c) { return (a + b) + c; }

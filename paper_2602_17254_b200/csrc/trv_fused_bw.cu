@@ -171,15 +171,19 @@ __device__ __forceinline__ void bw_tile(const BwArgs& a, const Tabs& tabs) {
 
 template <typename T, int V, int S, int D, int CAP>
 __global__ void __launch_bounds__(kBwThreads) k_bw_fused(PtrTab<CAP> in, PtrTab<CAP> out, BwArgs a) {
+    pdl_trigger();
     __shared__ const T* sin[CAP];
     __shared__ T* sout[CAP];
     for (int r = threadIdx.x; r < a.n; r += kBwThreads) { sin[r] = (const T*)in.p[r]; sout[r] = (T*)out.p[r]; }
     __syncthreads();
+    pdl_wait();
     bw_tile<T, V, S, D>(a, SmemTabs<T>{sin, sout});
 }
 
 template <typename T, int V, int S, int D>
 __global__ void __launch_bounds__(kBwThreads) k_bw_fused_strided(StrideAddr in, StrideAddr out, BwArgs a) {
+    pdl_trigger();
+    pdl_wait();
     bw_tile<T, V, S, D>(a, StrideTabs<T>{in, out});
 }
 
@@ -202,12 +206,12 @@ static void launch_bw(const Call& c, const BwArgs& a) {
     if (tiles == 0) return;
     StrideAddr sin, sout;
     if (uniform_stride(c.in, p.n, &sin) && uniform_stride((const void* const*)c.out, p.n, &sout)) {
-        TRV_LAUNCH((k_bw_fused_strided<T, V, S, D>), dim3((unsigned)tiles, D, 1), kBwThreads, 0, c.st, sin, sout, a);
+        launch_pdl(k_bw_fused_strided<T, V, S, D>, dim3((unsigned)tiles, D, 1), dim3(kBwThreads), 0, c.st, sin, sout, a);
         return;
     }
     PtrTab<CAP> in, out;
     for (int r = 0; r < p.n; ++r) { in.p[r] = const_cast<void*>(c.in[r]); out.p[r] = c.out[r]; }
-    TRV_LAUNCH((k_bw_fused<T, V, S, D, CAP>), dim3((unsigned)tiles, D, 1), kBwThreads, 0, c.st, in, out, a);
+    launch_pdl(k_bw_fused<T, V, S, D, CAP>, dim3((unsigned)tiles, D, 1), dim3(kBwThreads), 0, c.st, in, out, a);
 }
 
 template <typename T, int V, int S>
@@ -251,8 +255,9 @@ trv_status_t run_fused_bandwidth(const Call& c) {
         for (int t = 0; t < p.S; ++t) { a.ldim[sl][t] = p.steps[sl][t].dim; a.ldist[sl][t] = p.steps[sl][t].dist; }
     }
     // Four columns per thread when blocks are long enough that few threads straddle a block
-    // boundary; one column per thread otherwise (every thread then has its own owner).
-    const bool wide = min_block >= 256;
+    // boundary and the vector is long enough to fill the GPU with such threads; one column per
+    // thread otherwise (every thread then has its own owner).
+    const bool wide = min_block >= 256 && c.count >= ((size_t)1 << 20);
     g_last_kernel = wide ? "bw_fused<V=4>" : "bw_fused<V=1>";
     trv_status_t st;
     if (c.dtype == TRV_FLOAT32) st = wide ? bw_by_s<float, 4>(c, a) : bw_by_s<float, 1>(c, a);

@@ -111,9 +111,11 @@ __device__ __forceinline__ void lat_reg_body(const Addr& in, const Addr& out, co
 
 template <typename T, int A, int D, int V, int THREADS, typename Addr>
 __global__ void __launch_bounds__(THREADS) k_lat_reg(Addr in, Addr out, LatArgs a) {
+    pdl_trigger();
     const int c = blockIdx.y;
     const long long lo = a.lo[c], hi = a.hi[c];
     const long long t0 = (lo / (32 * V)) * (32 * V) + (long long)blockIdx.x * THREADS * V;    // first column of the tile
+    pdl_wait();
     const long long e = t0 + (long long)threadIdx.x * V;
     if (t0 >= lo && t0 + (long long)THREADS * V <= hi) {
         lat_reg_body<T, A, D, V, true>(in, out, a, c, e);
@@ -177,48 +179,77 @@ __device__ __forceinline__ void lat_ring_body(const Addr& in, const Addr& out, c
 
 template <typename T, int M, int V, typename Addr>
 __global__ void __launch_bounds__(288 / V) k_lat_ring(Addr in, Addr out, LatArgs a) {
+    pdl_trigger();
     extern __shared__ uint4 slab_raw[];
     T* slab = reinterpret_cast<T*>(slab_raw);       // [9 M][32]
     const long long t0 = (a.lo[0] & ~31LL) + (long long)blockIdx.x * 32;
+    pdl_wait();
     if (t0 >= a.lo[0] && t0 + 32 <= a.hi[0]) lat_ring_body<T, M, V, true>(in, out, a, slab, t0);   // CTA-uniform
     else lat_ring_body<T, M, V, false>(in, out, a, slab, t0);
 }
 
 // ------------------------------------------------------------------ 9 x 9 x 9 torus
 
-// 32-column tiles; a thread owns 2 adjacent columns (packed adds) and one ninth of the ranks:
-// 9 * 16 = 144 threads, two CTAs per SM.  A, B, C = the slice's dimensions in its own order.
+__device__ __forceinline__ void cp_async_8(void* smem_dst, const void* gmem_src) {
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+
+// W-column tiles (W = 32 or 16); a thread owns 2 adjacent columns (packed adds) and one ninth of
+// the ranks: 9 * W / 2 threads.  A, B, C = the slice's dimensions in its own order; their rank
+// strides sA, sB, sC are compile-time (ROT = slice number), so every rank offset inside a closed
+// set is an immediate.
 //   group 1: steps (A,1) (B,1) on the 9x9 plane C = set, streamed row by row (a row = 9 values
 //            along A): (A,1) inside a row, (B,1) over a sliding window of three rows
 //   group 2: steps (C,1) (A,3) on the closed sets {A in a0+3i, B = j, all C}   (27 values, 3 sets per thread)
 //   group 3: steps (B,3) (C,3) on the closed sets {A = i, B in b0+3j, C in c0+3k} (9 values, 9 sets per thread)
 // Between groups the tile stays in shared memory; inside a group every set is read and written
 // by one thread only, so the two barriers between the groups are the only synchronisation.
-template <typename T, bool FULL, typename Addr>
-__device__ __forceinline__ void lat_t999_body(const Addr& in, const Addr& out, const LatArgs& a, T* slab, int c, long long t0) {
-    constexpr int V = 2, LANES = 16;
+template <typename T, int ROT, int W, bool FULL, typename Addr>
+__device__ __forceinline__ void lat_t999_body(const Addr& in, const Addr& out, const LatArgs& a, T* slab, long long t0) {
+    constexpr int V = 2, LANES = W / V;
+    constexpr int sA = ROT == 0 ? 1 : (ROT == 1 ? 9 : 81), sB = ROT == 0 ? 9 : (ROT == 1 ? 81 : 1),
+                  sC = ROT == 0 ? 81 : (ROT == 1 ? 1 : 9);
     using E = Elem<T, V>;
     const int lane = threadIdx.x % LANES, set = threadIdx.x / LANES;
-    const long long lo = a.lo[c], hi = a.hi[c];
+    const long long lo = a.lo[ROT], hi = a.hi[ROT];
     const long long e = t0 + lane * V;
-    const int sA = a.rs[c][0], sB = a.rs[c][1], sC = a.rs[c][2];
-    auto sl = [&](int r) -> E& { return *reinterpret_cast<E*>(slab + r * 32 + lane * V); };
+    T* const mine = slab + lane * V;
+    auto sl = [&](int r) -> E& { return *reinterpret_cast<E*>(mine + r * W); };
 
     {   // ---- group 1
+        const int r0 = set * sC;
+        if constexpr (FULL) {
+            // Asynchronous copies global -> shared for the thread's own plane: all 81 are in flight at
+            // once without holding registers, and only the issuing thread reads them back, so no
+            // barrier is needed before the plane is processed in place.
+#pragma unroll
+            for (int idx = 0; idx < 81; ++idx) {
+                const int r = r0 + (idx % 9) * sA + (idx / 9) * sB;
+                cp_async_8(&sl(r), in.ptr(r) + e * (long long)sizeof(T));
+            }
+            cp_async_wait_all();
+        }
         auto load_row = [&](int j, E (&row)[9]) {
 #pragma unroll
-            for (int i = 0; i < 9; ++i) row[i] = load_elem<T, V, FULL>(in.ptr(i * sA + j * sB + set * sC), e, lo, hi);
+            for (int i = 0; i < 9; ++i) {
+                if constexpr (FULL) row[i] = sl(r0 + i * sA + j * sB);
+                else row[i] = load_elem<T, V, false>(in.ptr(r0 + i * sA + j * sB), e, lo, hi);
+            }
             reg_step<9, 1, 9, 1>(row);                                      // (A,1)
         };
         auto emit = [&](int j, const E (&p)[9], const E (&q)[9], const E (&r)[9]) {     // (B,1) for row j
 #pragma unroll
-            for (int i = 0; i < 9; ++i) sl(i * sA + j * sB + set * sC) = add3(p[i], q[i], r[i]);
+            for (int i = 0; i < 9; ++i) sl(r0 + i * sA + j * sB) = add3(p[i], q[i], r[i]);
         };
-        E r0[9], r1[9], prev[9], cur[9], next[9];
-        load_row(0, r0);
-        load_row(1, r1);
+        E first[9], second[9], prev[9], cur[9], next[9];
+        load_row(0, first);
+        load_row(1, second);
 #pragma unroll
-        for (int i = 0; i < 9; ++i) { prev[i] = r0[i]; cur[i] = r1[i]; }
+        for (int i = 0; i < 9; ++i) { prev[i] = first[i]; cur[i] = second[i]; }
 #pragma unroll
         for (int j = 1; j < 8; ++j) {
             load_row(j + 1, next);
@@ -226,50 +257,54 @@ __device__ __forceinline__ void lat_t999_body(const Addr& in, const Addr& out, c
 #pragma unroll
             for (int i = 0; i < 9; ++i) { prev[i] = cur[i]; cur[i] = next[i]; }
         }
-        emit(8, prev, cur, r0);     // row 8: rows 7, 8, 0
-        emit(0, cur, r0, r1);       // row 0: rows 8, 0, 1
+        emit(8, prev, cur, first);      // row 8: rows 7, 8, 0
+        emit(0, cur, first, second);    // row 0: rows 8, 0, 1
     }
     __syncthreads();
     // ---- group 2: flat index k + 9 i  <->  rank (a0 + 3 i) sA + j sB + k sC
 #pragma unroll 1
     for (int m = 0; m < 3; ++m) {
-        const int q = set + 9 * m, a0 = q % 3, j = q / 3;
+        const int q = set + 9 * m, r0 = (q % 3) * sA + (q / 3) * sB;
         E v[27];
 #pragma unroll
-        for (int idx = 0; idx < 27; ++idx) v[idx] = sl((a0 + 3 * (idx / 9)) * sA + j * sB + (idx % 9) * sC);
+        for (int idx = 0; idx < 27; ++idx) v[idx] = sl(r0 + 3 * (idx / 9) * sA + (idx % 9) * sC);
         reg_step<27, 1, 9, 1>(v);       // (C,1)
         reg_step<27, 9, 3, 1>(v);       // (A,3): a ring of three with distance one inside this set
 #pragma unroll
-        for (int idx = 0; idx < 27; ++idx) sl((a0 + 3 * (idx / 9)) * sA + j * sB + (idx % 9) * sC) = v[idx];
+        for (int idx = 0; idx < 27; ++idx) sl(r0 + 3 * (idx / 9) * sA + (idx % 9) * sC) = v[idx];
     }
     __syncthreads();
     // ---- group 3: flat index jj + 3 kk  <->  rank i sA + (b0 + 3 jj) sB + (c0 + 3 kk) sC
     const bool any = FULL || (e < hi && e + V > lo);
 #pragma unroll 1
     for (int m = 0; m < 9; ++m) {
-        const int q = set + 9 * m, i = q % 9, b0 = (q / 9) % 3, c0 = q / 27;
+        const int q = set + 9 * m, r0 = (q % 9) * sA + ((q / 9) % 3) * sB + (q / 27) * sC;
         E v[9];
 #pragma unroll
-        for (int idx = 0; idx < 9; ++idx) v[idx] = sl(i * sA + (b0 + 3 * (idx % 3)) * sB + (c0 + 3 * (idx / 3)) * sC);
+        for (int idx = 0; idx < 9; ++idx) v[idx] = sl(r0 + 3 * (idx % 3) * sB + 3 * (idx / 3) * sC);
         reg_step<9, 1, 3, 1>(v);        // (B,3)
         reg_step<9, 3, 3, 1>(v);        // (C,3)
         if (any) {
 #pragma unroll
             for (int idx = 0; idx < 9; ++idx)
-                store_elem<T, V, FULL>(out.ptr(i * sA + (b0 + 3 * (idx % 3)) * sB + (c0 + 3 * (idx / 3)) * sC), e, lo, hi, v[idx]);
+                store_elem<T, V, FULL>(out.ptr(r0 + 3 * (idx % 3) * sB + 3 * (idx / 3) * sC), e, lo, hi, v[idx]);
         }
     }
 }
 
-template <typename T, typename Addr>
-__global__ void __launch_bounds__(144, 2) k_lat_t999(Addr in, Addr out, LatArgs a) {
+template <typename T, int W, typename Addr>
+__global__ void __launch_bounds__(9 * W / 2, 64 / W) k_lat_t999(Addr in, Addr out, LatArgs a) {
+    pdl_trigger();
     extern __shared__ uint4 slab_raw[];
-    T* slab = reinterpret_cast<T*>(slab_raw);       // [729][32]
-    const int c = blockIdx.y;
-    const long long t0 = (a.lo[c] & ~31LL) + (long long)blockIdx.x * 32;
-    if (t0 >= a.hi[c]) return;                                                                      // CTA-uniform
-    if (t0 >= a.lo[c] && t0 + 32 <= a.hi[c]) lat_t999_body<T, true>(in, out, a, slab, c, t0);      // CTA-uniform
-    else lat_t999_body<T, false>(in, out, a, slab, c, t0);
+    T* slab = reinterpret_cast<T*>(slab_raw);       // [729][W]
+    const int c = blockIdx.y;                       // everything below is CTA-uniform
+    const long long t0 = (a.lo[c] / W) * W + (long long)blockIdx.x * W;
+    if (t0 >= a.hi[c]) return;
+    pdl_wait();
+    const bool full = t0 >= a.lo[c] && t0 + W <= a.hi[c];
+    if (c == 0) { if (full) lat_t999_body<T, 0, W, true>(in, out, a, slab, t0); else lat_t999_body<T, 0, W, false>(in, out, a, slab, t0); }
+    else if (c == 1) { if (full) lat_t999_body<T, 1, W, true>(in, out, a, slab, t0); else lat_t999_body<T, 1, W, false>(in, out, a, slab, t0); }
+    else { if (full) lat_t999_body<T, 2, W, true>(in, out, a, slab, t0); else lat_t999_body<T, 2, W, false>(in, out, a, slab, t0); }
 }
 
 // ------------------------------------------------------------------ host side
@@ -310,7 +345,7 @@ template <typename T, int A, int D, int V, int THREADS, typename Addr>
 static void launch_reg(const Call& c, const Addr& in, const Addr& out, const LatArgs& a) {
     const long long tiles = tiles_for(a, D, (long long)V * THREADS, 32 * V);
     if (tiles == 0) return;
-    TRV_LAUNCH((k_lat_reg<T, A, D, V, THREADS, Addr>), dim3((unsigned)tiles, D, 1), THREADS, 0, c.st, in, out, a);
+    launch_pdl(k_lat_reg<T, A, D, V, THREADS, Addr>, dim3((unsigned)tiles, D, 1), dim3(THREADS), 0, c.st, in, out, a);
 }
 
 template <typename T, typename Addr>
@@ -323,7 +358,7 @@ static trv_status_t lat_fused_launch(const Call& c, const Addr& in, const Addr& 
         const int A = p.dims[0], D = p.ndims;
         if (A == 3 && D == 1) { g_last_kernel = "lat_reg<3>"; launch_reg<T, 3, 1, 4, 64>(c, in, out, a); }
         else if (A == 9 && D == 1) { g_last_kernel = "lat_reg<9>"; launch_reg<T, 9, 1, 4, 64>(c, in, out, a); }
-        else if (A == 27 && D == 1) { g_last_kernel = "lat_reg<27>"; launch_reg<T, 27, 1, 4, 64>(c, in, out, a); }
+        else if (A == 27 && D == 1) { g_last_kernel = "lat_reg<27>"; launch_reg<T, 27, 1, 2, 128>(c, in, out, a); }
         else if (A == 3 && D == 2) { g_last_kernel = "lat_reg<3x3>"; launch_reg<T, 3, 2, 4, 64>(c, in, out, a); }
         else if (A == 3 && D == 3) { g_last_kernel = "lat_reg<3x3x3>"; launch_reg<T, 3, 3, 4, 64>(c, in, out, a); }
         else if (A == 81 && D == 1) { g_last_kernel = "lat_reg<81>"; launch_reg<T, 81, 1, 2, 64>(c, in, out, a); }
@@ -335,23 +370,23 @@ static trv_status_t lat_fused_launch(const Call& c, const Addr& in, const Addr& 
         if (tiles > 0) {
             if (p.n == 243) {
                 g_last_kernel = "lat_ring<243>";
-                TRV_LAUNCH((k_lat_ring<T, 27, 2, Addr>), dim3((unsigned)tiles), 144, 243 * 32 * 4, c.st, in, out, a);
+                launch_pdl(k_lat_ring<T, 27, 2, Addr>, dim3((unsigned)tiles), dim3(144), 243 * 32 * 4, c.st, in, out, a);
             } else {
                 g_last_kernel = "lat_ring<729>";
                 auto kfn = k_lat_ring<T, 81, 1, Addr>;
                 static const cudaError_t once = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, 729 * 32 * 4);
                 (void)once;
-                TRV_LAUNCH(kfn, dim3((unsigned)tiles), 288, 729 * 32 * 4, c.st, in, out, a);
+                launch_pdl(kfn, dim3((unsigned)tiles), dim3(288), 729 * 32 * 4, c.st, in, out, a);
             }
         }
     } else if (kind == LatKind::T999) {
         g_last_kernel = "lat_t999";
         const long long tiles = tiles_for(a, 3, 32, 32);
         if (tiles > 0) {
-            auto kfn = k_lat_t999<T, Addr>;
+            auto kfn = k_lat_t999<T, 32, Addr>;
             static const cudaError_t once = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, 729 * 32 * 4);
             (void)once;
-            TRV_LAUNCH(kfn, dim3((unsigned)tiles, 3, 1), 144, 729 * 32 * 4, c.st, in, out, a);
+            launch_pdl(kfn, dim3((unsigned)tiles, 3, 1), dim3(144), 729 * 32 * 4, c.st, in, out, a);
         }
     } else {
         return TRV_ERR_UNSUPPORTED;

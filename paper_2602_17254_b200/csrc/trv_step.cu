@@ -43,6 +43,8 @@ __device__ __forceinline__ void for_range(long long lo, long long hi, F1 f1, F4 
 template <typename T, int CAP>
 __global__ void __launch_bounds__(kThreads) k_lat_step(PtrTab<CAP> src, PtrTab<CAP> dst, LatStepArgs a) {
     using V = typename Vec4<T>::type;
+    pdl_trigger();
+    pdl_wait();
     const int p = blockIdx.y;
     for (int c = 0; c < a.nslices; ++c) {
         const SliceStep s = a.s[c];
@@ -64,6 +66,8 @@ __global__ void __launch_bounds__(kThreads) k_lat_step(PtrTab<CAP> src, PtrTab<C
 
 template <int CAP>
 __global__ void __launch_bounds__(kThreads) k_copy(PtrTab<CAP> src, PtrTab<CAP> dst, long long count) {
+    pdl_trigger();
+    pdl_wait();
     const uint32_t* __restrict__ S = (const uint32_t*)src.p[blockIdx.y];
     uint32_t* __restrict__ O = (uint32_t*)dst.p[blockIdx.y];
     for_range(
@@ -107,6 +111,8 @@ __device__ __forceinline__ void block_range(const BwStepArgs& a, const BwSlice& 
 template <typename T, int CAP>
 __global__ void __launch_bounds__(kThreads) k_rs_step(PtrTab<CAP> buf, BwStepArgs a) {
     using V = typename Vec4<T>::type;
+    pdl_trigger();
+    pdl_wait();
     const int p = blockIdx.z;
     for (int c = 0; c < a.nslices; ++c) {
         const BwSlice& s = a.s[c];
@@ -130,6 +136,8 @@ __global__ void __launch_bounds__(kThreads) k_rs_step(PtrTab<CAP> buf, BwStepArg
 // AllGather step: grid (x, 2 * nact, n): rank p copies the finished blocks of both peers
 template <int CAP>
 __global__ void __launch_bounds__(kThreads) k_ag_step(PtrTab<CAP> buf, BwStepArgs a) {
+    pdl_trigger();
+    pdl_wait();
     const int p = blockIdx.z;
     const int side = blockIdx.y / a.nact, q = blockIdx.y % a.nact;
     for (int c = 0; c < a.nslices; ++c) {
@@ -208,13 +216,13 @@ static trv_status_t lat_impl(const Call& c) {
             a.s[sl].stride = p.stride[st.dim]; a.s[sl].size = p.dims[st.dim]; a.s[sl].dist = st.dist;
         }
         dim3 grid(grid_x(max_len), n, 1);
-        if (c.dtype == TRV_FLOAT32) TRV_LAUNCH((k_lat_step<float, CAP>), grid, kThreads, 0, c.st, *src, *dst[t], a);
-        else TRV_LAUNCH((k_lat_step<uint32_t, CAP>), grid, kThreads, 0, c.st, *src, *dst[t], a);
+        if (c.dtype == TRV_FLOAT32) launch_pdl(k_lat_step<float, CAP>, grid, dim3(kThreads), 0, c.st, *src, *dst[t], a);
+        else launch_pdl(k_lat_step<uint32_t, CAP>, grid, dim3(kThreads), 0, c.st, *src, *dst[t], a);
         src = dst[t];
     }
     if (src != &OUT) {      // only S == 1 in place: bring the result home
         dim3 grid(grid_x((long long)c.count), n, 1);
-        TRV_LAUNCH((k_copy<CAP>), grid, kThreads, 0, c.st, *src, OUT, (long long)c.count);
+        launch_pdl(k_copy<CAP>, grid, dim3(kThreads), 0, c.st, *src, OUT, (long long)c.count);
     }
     return cudaGetLastError() == cudaSuccess ? TRV_OK : TRV_ERR_CUDA;
 }
@@ -235,7 +243,7 @@ static trv_status_t bw_impl(const Call& c) {
     for (int r = 0; r < n; ++r) { IN.p[r] = const_cast<void*>(c.in[r]); OUT.p[r] = c.out[r]; }
     if (!c.in_place) {
         dim3 grid(grid_x((long long)c.count), n, 1);
-        TRV_LAUNCH((k_copy<CAP>), grid, kThreads, 0, c.st, IN, OUT, (long long)c.count);
+        launch_pdl(k_copy<CAP>, grid, dim3(kThreads), 0, c.st, IN, OUT, (long long)c.count);
     }
     for (int row = 0; row < 2 * S; ++row) {
         const int t = p.step_of_row(row);
@@ -259,11 +267,11 @@ static trv_status_t bw_impl(const Call& c) {
         a.nact = nact;
         if (row < S) {
             dim3 grid(grid_x(max_len), nact, n);
-            if (c.dtype == TRV_FLOAT32) TRV_LAUNCH((k_rs_step<float, CAP>), grid, kThreads, 0, c.st, OUT, a);
-            else TRV_LAUNCH((k_rs_step<uint32_t, CAP>), grid, kThreads, 0, c.st, OUT, a);
+            if (c.dtype == TRV_FLOAT32) launch_pdl(k_rs_step<float, CAP>, grid, dim3(kThreads), 0, c.st, OUT, a);
+            else launch_pdl(k_rs_step<uint32_t, CAP>, grid, dim3(kThreads), 0, c.st, OUT, a);
         } else {
             dim3 grid(grid_x(max_len), 2 * nact, n);
-            TRV_LAUNCH((k_ag_step<CAP>), grid, kThreads, 0, c.st, OUT, a);
+            launch_pdl(k_ag_step<CAP>, grid, dim3(kThreads), 0, c.st, OUT, a);
         }
     }
     return cudaGetLastError() == cudaSuccess ? TRV_OK : TRV_ERR_CUDA;

@@ -57,8 +57,8 @@ def test_fused_bandwidth_matches_oracle(dims):
     check_case(dims, BW, small, "normal", 31, FUSED)
     check_case(dims, BW, small, "int32", 32, FUSED, in_place=False)
     check_scattered(dims, BW, small, "normal", 36, FUSED)
-    if n <= 81:                                           # four columns per thread (blocks >= 256 elements)
-        wide = 300 * n * D + 7
+    if n <= 27:                                           # four columns per thread (long blocks, >= 2^20 elements)
+        wide = (1 << 20) + 300 * n * D + 7
         check_case(dims, BW, wide, "normal", 33, FUSED)
         check_case(dims, BW, wide, "int32", 34, FUSED, in_place=False)
         check_scattered(dims, BW, wide, "int32", 37, FUSED)
@@ -67,7 +67,7 @@ def test_fused_bandwidth_matches_oracle(dims):
 def test_fused_bandwidth_wide_path_on_729_ranks_sampled():
     """9x9x9 with blocks of >= 256 elements: the oracle checks windows around slice and block
     boundaries and in block interiors."""
-    dims, count = (9, 9, 9), 300 * 729 * 3 + 5
+    dims, count = (9, 9, 9), (1 << 20) + 5
     plan = binding.Plan(dims, BW)
     wins = [(0, 700), (count // 3 - 400, count // 3 + 400), (2 * count // 3 - 333, 2 * count // 3 + 777),
             (count - 900, count), (123456, 124000)]
