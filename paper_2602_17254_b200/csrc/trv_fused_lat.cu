@@ -12,65 +12,13 @@
 //   k_lat_reg   : n <= 81 (rings 3..81, tori 3x3, 9x9, 3x3x3, 3x3x3x3): one group, no shared memory
 //   k_lat_ring  : rings of 243 and 729: steps {1,3} on windows of consecutive ranks with a
 //                 halo of 4, then the remaining steps on the closed sets {q + 9 i}
-//   k_lat_t999  : 9x9x9 torus: steps (A,1)(B,1) on 9x9 planes, then (C,1)(A,3)(B,3)(C,3) on the
-//                 3x3x9 closed sets; A,B,C = the slice's dimension order
+//   k_lat_t999_ws (trv_fused_t999.cu): 9x9x9 torus, three groups of two steps, warp-specialised
 #include <type_traits>
 
 #include "trv_dev.cuh"
+#include "trv_fused_lat.cuh"
 
 namespace trv {
-
-constexpr int ipow3(int e) { return e <= 0 ? 1 : 3 * ipow3(e - 1); }
-constexpr int ipow(int b, int e) { return e <= 0 ? 1 : b * ipow(b, e - 1); }
-constexpr int ilog3(int n) { return n <= 1 ? 0 : 1 + ilog3(n / 3); }
-
-// FULL is a compile-time property of the whole tile (every column of the CTA lies inside the
-// slice): the common case is then straight-line code whose loads the compiler can batch; only the
-// one or two edge tiles of a slice take the masked, element-by-element form.
-template <typename T, int V, bool FULL>
-__device__ __forceinline__ Elem<T, V> load_elem(const char* row, long long e, long long lo, long long hi) {
-    const T* p = reinterpret_cast<const T*>(row);
-    Elem<T, V> r;
-    if constexpr (FULL) {
-        r = *reinterpret_cast<const Elem<T, V>*>(p + e);
-    } else {
-#pragma unroll
-        for (int k = 0; k < V; ++k) r.x[k] = (e + k >= lo && e + k < hi) ? p[e + k] : T(0);
-    }
-    return r;
-}
-template <typename T, int V, bool FULL>
-__device__ __forceinline__ void store_elem(char* row, long long e, long long lo, long long hi, const Elem<T, V>& v) {
-    T* p = reinterpret_cast<T*>(row);
-    if constexpr (FULL) {
-        *reinterpret_cast<Elem<T, V>*>(p + e) = v;
-    } else {
-#pragma unroll
-        for (int k = 0; k < V; ++k)
-            if (e + k >= lo && e + k < hi) p[e + k] = v.x[k];
-    }
-}
-
-// One joint-reduction step on a register array: along the axis with flat stride STRIDE and ring
-// length L, new[i] = (old[i - DIST] + old[i]) + old[i + DIST], indices modulo L.
-template <int N, int STRIDE, int L, int DIST, typename E>
-__device__ __forceinline__ void reg_step(E (&v)[N]) {
-#pragma unroll
-    for (int base = 0; base < N; ++base) {
-        if ((base / STRIDE) % L != 0) continue;
-        E line[L];
-#pragma unroll
-        for (int i = 0; i < L; ++i) line[i] = v[base + i * STRIDE];
-#pragma unroll
-        for (int i = 0; i < L; ++i) v[base + i * STRIDE] = add3(line[(i - DIST + L) % L], line[i], line[(i + DIST) % L]);
-    }
-}
-
-struct LatArgs {
-    int nslices;
-    long long lo[TRV_MAX_DIMS], hi[TRV_MAX_DIMS];   // local element range of each slice
-    int rs[TRV_MAX_DIMS][4];                        // rank stride of the slice's k-th dimension in its own order
-};
 
 // ------------------------------------------------------------------ n <= 81: registers only
 
@@ -188,125 +136,6 @@ __global__ void __launch_bounds__(288 / V) k_lat_ring(Addr in, Addr out, LatArgs
     else lat_ring_body<T, M, V, false>(in, out, a, slab, t0);
 }
 
-// ------------------------------------------------------------------ 9 x 9 x 9 torus
-
-__device__ __forceinline__ void cp_async_8(void* smem_dst, const void* gmem_src) {
-    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(d), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() {
-    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
-}
-
-// W-column tiles (W = 32 or 16); a thread owns 2 adjacent columns (packed adds) and one ninth of
-// the ranks: 9 * W / 2 threads.  A, B, C = the slice's dimensions in its own order; their rank
-// strides sA, sB, sC are compile-time (ROT = slice number), so every rank offset inside a closed
-// set is an immediate.
-//   group 1: steps (A,1) (B,1) on the 9x9 plane C = set, streamed row by row (a row = 9 values
-//            along A): (A,1) inside a row, (B,1) over a sliding window of three rows
-//   group 2: steps (C,1) (A,3) on the closed sets {A in a0+3i, B = j, all C}   (27 values, 3 sets per thread)
-//   group 3: steps (B,3) (C,3) on the closed sets {A = i, B in b0+3j, C in c0+3k} (9 values, 9 sets per thread)
-// Between groups the tile stays in shared memory; inside a group every set is read and written
-// by one thread only, so the two barriers between the groups are the only synchronisation.
-template <typename T, int ROT, int W, bool FULL, typename Addr>
-__device__ __forceinline__ void lat_t999_body(const Addr& in, const Addr& out, const LatArgs& a, T* slab, long long t0) {
-    constexpr int V = 2, LANES = W / V;
-    constexpr int sA = ROT == 0 ? 1 : (ROT == 1 ? 9 : 81), sB = ROT == 0 ? 9 : (ROT == 1 ? 81 : 1),
-                  sC = ROT == 0 ? 81 : (ROT == 1 ? 1 : 9);
-    using E = Elem<T, V>;
-    const int lane = threadIdx.x % LANES, set = threadIdx.x / LANES;
-    const long long lo = a.lo[ROT], hi = a.hi[ROT];
-    const long long e = t0 + lane * V;
-    T* const mine = slab + lane * V;
-    auto sl = [&](int r) -> E& { return *reinterpret_cast<E*>(mine + r * W); };
-
-    {   // ---- group 1
-        const int r0 = set * sC;
-        if constexpr (FULL) {
-            // Asynchronous copies global -> shared for the thread's own plane: all 81 are in flight at
-            // once without holding registers, and only the issuing thread reads them back, so no
-            // barrier is needed before the plane is processed in place.
-#pragma unroll
-            for (int idx = 0; idx < 81; ++idx) {
-                const int r = r0 + (idx % 9) * sA + (idx / 9) * sB;
-                cp_async_8(&sl(r), in.ptr(r) + e * (long long)sizeof(T));
-            }
-            cp_async_wait_all();
-        }
-        auto load_row = [&](int j, E (&row)[9]) {
-#pragma unroll
-            for (int i = 0; i < 9; ++i) {
-                if constexpr (FULL) row[i] = sl(r0 + i * sA + j * sB);
-                else row[i] = load_elem<T, V, false>(in.ptr(r0 + i * sA + j * sB), e, lo, hi);
-            }
-            reg_step<9, 1, 9, 1>(row);                                      // (A,1)
-        };
-        auto emit = [&](int j, const E (&p)[9], const E (&q)[9], const E (&r)[9]) {     // (B,1) for row j
-#pragma unroll
-            for (int i = 0; i < 9; ++i) sl(r0 + i * sA + j * sB) = add3(p[i], q[i], r[i]);
-        };
-        E first[9], second[9], prev[9], cur[9], next[9];
-        load_row(0, first);
-        load_row(1, second);
-#pragma unroll
-        for (int i = 0; i < 9; ++i) { prev[i] = first[i]; cur[i] = second[i]; }
-#pragma unroll
-        for (int j = 1; j < 8; ++j) {
-            load_row(j + 1, next);
-            emit(j, prev, cur, next);
-#pragma unroll
-            for (int i = 0; i < 9; ++i) { prev[i] = cur[i]; cur[i] = next[i]; }
-        }
-        emit(8, prev, cur, first);      // row 8: rows 7, 8, 0
-        emit(0, cur, first, second);    // row 0: rows 8, 0, 1
-    }
-    __syncthreads();
-    // ---- group 2: flat index k + 9 i  <->  rank (a0 + 3 i) sA + j sB + k sC
-#pragma unroll 1
-    for (int m = 0; m < 3; ++m) {
-        const int q = set + 9 * m, r0 = (q % 3) * sA + (q / 3) * sB;
-        E v[27];
-#pragma unroll
-        for (int idx = 0; idx < 27; ++idx) v[idx] = sl(r0 + 3 * (idx / 9) * sA + (idx % 9) * sC);
-        reg_step<27, 1, 9, 1>(v);       // (C,1)
-        reg_step<27, 9, 3, 1>(v);       // (A,3): a ring of three with distance one inside this set
-#pragma unroll
-        for (int idx = 0; idx < 27; ++idx) sl(r0 + 3 * (idx / 9) * sA + (idx % 9) * sC) = v[idx];
-    }
-    __syncthreads();
-    // ---- group 3: flat index jj + 3 kk  <->  rank i sA + (b0 + 3 jj) sB + (c0 + 3 kk) sC
-    const bool any = FULL || (e < hi && e + V > lo);
-#pragma unroll 1
-    for (int m = 0; m < 9; ++m) {
-        const int q = set + 9 * m, r0 = (q % 9) * sA + ((q / 9) % 3) * sB + (q / 27) * sC;
-        E v[9];
-#pragma unroll
-        for (int idx = 0; idx < 9; ++idx) v[idx] = sl(r0 + 3 * (idx % 3) * sB + 3 * (idx / 3) * sC);
-        reg_step<9, 1, 3, 1>(v);        // (B,3)
-        reg_step<9, 3, 3, 1>(v);        // (C,3)
-        if (any) {
-#pragma unroll
-            for (int idx = 0; idx < 9; ++idx)
-                store_elem<T, V, FULL>(out.ptr(r0 + 3 * (idx % 3) * sB + 3 * (idx / 3) * sC), e, lo, hi, v[idx]);
-        }
-    }
-}
-
-template <typename T, int W, typename Addr>
-__global__ void __launch_bounds__(9 * W / 2, 64 / W) k_lat_t999(Addr in, Addr out, LatArgs a) {
-    pdl_trigger();
-    extern __shared__ uint4 slab_raw[];
-    T* slab = reinterpret_cast<T*>(slab_raw);       // [729][W]
-    const int c = blockIdx.y;                       // everything below is CTA-uniform
-    const long long t0 = (a.lo[c] / W) * W + (long long)blockIdx.x * W;
-    if (t0 >= a.hi[c]) return;
-    pdl_wait();
-    const bool full = t0 >= a.lo[c] && t0 + W <= a.hi[c];
-    if (c == 0) { if (full) lat_t999_body<T, 0, W, true>(in, out, a, slab, t0); else lat_t999_body<T, 0, W, false>(in, out, a, slab, t0); }
-    else if (c == 1) { if (full) lat_t999_body<T, 1, W, true>(in, out, a, slab, t0); else lat_t999_body<T, 1, W, false>(in, out, a, slab, t0); }
-    else { if (full) lat_t999_body<T, 2, W, true>(in, out, a, slab, t0); else lat_t999_body<T, 2, W, false>(in, out, a, slab, t0); }
-}
-
 // ------------------------------------------------------------------ host side
 
 enum class LatKind { None, Reg, Ring, T999 };
@@ -381,13 +210,7 @@ static trv_status_t lat_fused_launch(const Call& c, const Addr& in, const Addr& 
         }
     } else if (kind == LatKind::T999) {
         g_last_kernel = "lat_t999";
-        const long long tiles = tiles_for(a, 3, 32, 32);
-        if (tiles > 0) {
-            auto kfn = k_lat_t999<T, 32, Addr>;
-            static const cudaError_t once = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, 729 * 32 * 4);
-            (void)once;
-            launch_pdl(kfn, dim3((unsigned)tiles, 3, 1), dim3(144), 729 * 32 * 4, c.st, in, out, a);
-        }
+        return run_fused_t999(c, a);
     } else {
         return TRV_ERR_UNSUPPORTED;
     }

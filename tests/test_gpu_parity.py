@@ -64,6 +64,15 @@ def test_fused_bandwidth_matches_oracle(dims):
         check_scattered(dims, BW, wide, "int32", 37, FUSED)
 
 
+def test_fused_latency_9x9x9_many_tiles_per_cta():
+    """The 9x9x9 kernel is persistent (one CTA per SM looping over tiles, two tiles in flight): sizes
+    where a CTA gets 1, 2, 3 and about 9 tiles, with ragged slice edges, and scattered buffers."""
+    for count in (148 * 32 // 3 * 3 + 96, 9000, 14211, 40003):
+        check_case((9, 9, 9), LAT, count, "normal", count, FUSED)
+    check_case((9, 9, 9), LAT, 20011, "int32", 5, FUSED, in_place=False)
+    check_scattered((9, 9, 9), LAT, 20011, "normal", 6, FUSED)
+
+
 def test_fused_bandwidth_wide_path_on_729_ranks_sampled():
     """9x9x9 with blocks of >= 256 elements: the oracle checks windows around slice and block
     boundaries and in block interiors."""
