@@ -252,7 +252,8 @@ def run_ours(args, w):
     def step():
         for b in range(batch):
             plan.allreduce_ex(in_ptrs[b], out_ptrs[b], count, dcode, kernel=binding.KERNEL_AUTO,
-                              scratch_ptr=scratch.data_ptr() if need else 0, scratch_bytes=need, stream=sh)
+                              scratch_ptr=scratch.data_ptr() if need else 0, scratch_bytes=need,
+                              stream=torch.cuda.current_stream().cuda_stream)
 
     def barrier():
         torch.cuda.synchronize()
@@ -264,6 +265,17 @@ def run_ours(args, w):
         step()
     barrier()
     kernel_name = binding.last_kernel_name()
+    launches_per_step = None
+    if args.graph:      # one step captured once, replayed: removes the per-call host cost (launch-bound sizes)
+        l_before = binding.launch_count()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+        launches_per_step = binding.launch_count() - l_before
+        step = graph.replay
+        for _ in range(args.warmup):
+            step()
+        barrier()
     sampler = ClockSampler(local)
     l0 = binding.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -274,6 +286,8 @@ def run_ours(args, w):
     ev1.record(stream)
     barrier()
     launches = binding.launch_count() - l0
+    if launches_per_step is not None:
+        launches = launches_per_step * args.steps       # replayed launches are not seen by the library's counter
     ms = ev0.elapsed_time(ev1)
     note = "sampled during the timed region"
     if len(sampler.samples) < 8 and not args.profile:        # region too short for NVML: keep the same load running ~0.4 s more
@@ -357,7 +371,8 @@ def run_ours(args, w):
                        "ranks": n, "bytes_per_rank": w.bytes_per_rank, "calls_per_step": batch,
                        "l2": "each step touches %d distinct buffer sets = %.0f MiB read + %.0f MiB written (L2 is 126 MiB): "
                              "inputs larger than L2, no flush" % (batch, batch * set_bytes / 2**20, batch * set_bytes / 2**20),
-                       "kernel": kernel_name, "call": "trv_allreduce_ex, separate output buffers, TRV_KERNEL_AUTO",
+                       "kernel": kernel_name, "call": "trv_allreduce_ex, separate output buffers, TRV_KERNEL_AUTO"
+                       + (", one step captured in a CUDA graph and replayed" if args.graph else ""),
                        "parallelism": "replicas" if world > 1 else "single GPU"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": _traffic(kernel_name, w.name), "peak_source": peak_src,
@@ -391,6 +406,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-check", action="store_true", help="skip the parity spot check")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--graph", action="store_true", help="capture one step in a CUDA graph and time its replays")
     ap.add_argument("--count", type=int, default=0, help="override the workload's elements per rank")
     ap.add_argument("--profile", action="store_true",
                     help="for runs under ncu: only warm-up and timed launches (implies --no-cpu --no-check --no-e2e)")

@@ -192,3 +192,28 @@ def test_launch_counter_and_kernel_names():
     assert binding.launch_count() == before + 1 and binding.last_kernel_name() == "lat_reg<27>"
     run_gpu(plan, xd, STEP)
     assert binding.launch_count() == before + 1 + 3 and binding.last_kernel_name() == "step_latency"
+
+
+def test_calls_can_be_captured_in_a_cuda_graph():
+    """The AllReduce call is a pure launch sequence (no allocation, no synchronisation): it can be
+    captured into a CUDA graph and replayed; replays give the oracle's bits."""
+    for dims, variant, kernel in [((27,), LAT, FUSED), ((243,), BW, FUSED), ((9, 9), LAT, STEP), ((9, 9, 9), LAT, FUSED)]:
+        plan = binding.Plan(dims, variant)
+        n, count = plan.n, 2048
+        x = synth.rank_matrix("normal", 77, n, count)
+        xin = torch.from_numpy(x).to(DEV)
+        xout = torch.zeros_like(xin)
+        need = plan.scratch_bytes(count, kernel, in_place=False)
+        scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=DEV)
+        ip = binding.ptr_array([xin[r].data_ptr() for r in range(n)])
+        op = binding.ptr_array([xout[r].data_ptr() for r in range(n)])
+        g = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g):
+            plan.allreduce_ex(ip, op, count, binding.FLOAT32, kernel=kernel, scratch_ptr=scratch.data_ptr() if need else 0,
+                              scratch_bytes=need, stream=torch.cuda.current_stream().cuda_stream)
+        for _ in range(2):
+            xout.zero_()
+            g.replay()
+            torch.cuda.synchronize()
+            compare(dims, variant, x, xout.cpu().numpy())
