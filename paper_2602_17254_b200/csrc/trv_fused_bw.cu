@@ -141,6 +141,70 @@ __device__ __forceinline__ void column_tree(const BwArgs& a, int c, const Tabs& 
     for (int r = 0; r < a.n; ++r) *reinterpret_cast<P*>(tabs.out(r) + e) = res;
 }
 
+// Same value, for short vectors: one column per thread, 27 leaves (three tree levels) loaded at
+// once, so a thread needs n / 27 dependent memory round trips instead of n / 9.  S >= 3.
+template <typename T, int S, int D, typename Tabs>
+__device__ __forceinline__ void column_tree27(const BwArgs& a, int c, const Tabs& tabs, long long e, int j) {
+    int base[D];    // coordinates of the centre of the current 27-leaf chunk
+#pragma unroll
+    for (int d = 0; d < D; ++d) base[d] = (j / a.dstride[d]) % a.dims[d];
+#pragma unroll
+    for (int t = 3; t < S; ++t) {   // leftmost chunk: every step >= 3 at eps = -1
+        const int dt = a.ldim[c][t], xt = a.ldist[c][t];
+#pragma unroll
+        for (int d = 0; d < D; ++d) if (d == dt) base[d] = wrap(base[d] - xt, a.dims[d]);
+    }
+    int ldm[3], ldx[3];
+#pragma unroll
+    for (int t = 0; t < 3; ++t) { ldm[t] = a.ldim[c][t]; ldx[t] = a.ldist[c][t]; }
+    int vd[S];
+    T acc[S];
+#pragma unroll
+    for (int t = 0; t < S; ++t) vd[t] = 0;
+    constexpr int CHUNKS = (S == 3) ? 1 : (S == 4 ? 3 : (S == 5 ? 9 : 27));
+    T res = T(0);
+    for (int ch = 0; ch < CHUNKS; ++ch) {
+        T l[27];
+#pragma unroll
+        for (int m = 0; m < 27; ++m) {      // leaf m <-> (eps_2, eps_1, eps_0) = (m / 9 - 1, (m / 3) % 3 - 1, m % 3 - 1)
+            const int eps[3] = {m % 3 - 1, (m / 3) % 3 - 1, m / 9 - 1};
+            int rank = 0;
+#pragma unroll
+            for (int d = 0; d < D; ++d) {
+                int off = 0;
+#pragma unroll
+                for (int t = 0; t < 3; ++t) off += (ldm[t] == d) ? eps[t] * ldx[t] : 0;
+                int x = base[d] + off;      // |off| < a_d: the steps of one dimension sum to less than its side
+                x = x < 0 ? x + a.dims[d] : (x >= a.dims[d] ? x - a.dims[d] : x);
+                rank += x * a.dstride[d];
+            }
+            l[m] = tabs.in(rank)[e];
+        }
+        T r9[3];
+#pragma unroll
+        for (int g = 0; g < 3; ++g)
+            r9[g] = add3(add3(l[9 * g], l[9 * g + 1], l[9 * g + 2]), add3(l[9 * g + 3], l[9 * g + 4], l[9 * g + 5]),
+                         add3(l[9 * g + 6], l[9 * g + 7], l[9 * g + 8]));
+        T r = add3(r9[0], r9[1], r9[2]);
+        bool carry = true;
+#pragma unroll
+        for (int t = 3; t < S; ++t) {
+            if (carry) {
+                const int dt = a.ldim[c][t], xt = a.ldist[c][t];
+                int delta;
+                if (vd[t] == 0) { acc[t] = r; vd[t] = 1; delta = xt; carry = false; }
+                else if (vd[t] == 1) { acc[t] = add2(acc[t], r); vd[t] = 2; delta = xt; carry = false; }
+                else { r = add2(acc[t], r); vd[t] = 0; delta = -2 * xt; }
+#pragma unroll
+                for (int d = 0; d < D; ++d) if (d == dt) base[d] = wrap(base[d] + delta, a.dims[d]);
+            }
+        }
+        res = r;
+    }
+#pragma unroll 9
+    for (int r = 0; r < a.n; ++r) tabs.out(r)[e] = res;
+}
+
 template <typename T, int V, int S, int D, typename Tabs>
 __device__ __forceinline__ void bw_tile(const BwArgs& a, const Tabs& tabs) {
     const int c = blockIdx.y;
@@ -154,7 +218,8 @@ __device__ __forceinline__ void bw_tile(const BwArgs& a, const Tabs& tabs) {
         return (int)(((x + 1) * (unsigned)a.n - 1) / L);
     };
     if constexpr (V == 1) {
-        column_tree<T, 1, S, D>(a, c, tabs, e, owner(e));
+        if constexpr (S >= 3) column_tree27<T, S, D>(a, c, tabs, e, owner(e));
+        else column_tree<T, 1, S, D>(a, c, tabs, e, owner(e));
     } else {
         const bool inside = e >= lo && e + V <= hi;
         int j0 = 0;
@@ -254,14 +319,15 @@ trv_status_t run_fused_bandwidth(const Call& c) {
         if (min_block < 0 || bl < min_block) min_block = bl;
         for (int t = 0; t < p.S; ++t) { a.ldim[sl][t] = p.steps[sl][t].dim; a.ldist[sl][t] = p.steps[sl][t].dist; }
     }
-    // Four columns per thread when blocks are long enough that few threads straddle a block
-    // boundary and the vector is long enough to fill the GPU with such threads; one column per
-    // thread otherwise (every thread then has its own owner).
+    // Two columns per thread (8-byte accesses, packed adds) when blocks are long enough that few
+    // threads straddle a block boundary and the vector is long enough to fill the GPU with such
+    // threads; one column per thread otherwise (every thread then has its own owner).  Measured on
+    // B200: two columns beat four at every size (shorter thread lifetimes, more warps per SM).
     const bool wide = min_block >= 256 && c.count >= ((size_t)1 << 20);
-    g_last_kernel = wide ? "bw_fused<V=4>" : "bw_fused<V=1>";
+    g_last_kernel = wide ? "bw_fused<V=2>" : "bw_fused<V=1>";
     trv_status_t st;
-    if (c.dtype == TRV_FLOAT32) st = wide ? bw_by_s<float, 4>(c, a) : bw_by_s<float, 1>(c, a);
-    else st = wide ? bw_by_s<uint32_t, 4>(c, a) : bw_by_s<uint32_t, 1>(c, a);
+    if (c.dtype == TRV_FLOAT32) st = wide ? bw_by_s<float, 2>(c, a) : bw_by_s<float, 1>(c, a);
+    else st = wide ? bw_by_s<uint32_t, 2>(c, a) : bw_by_s<uint32_t, 1>(c, a);
     if (st != TRV_OK) return st;
     return cudaGetLastError() == cudaSuccess ? TRV_OK : TRV_ERR_CUDA;
 }

@@ -57,7 +57,7 @@ def test_fused_bandwidth_matches_oracle(dims):
     check_case(dims, BW, small, "normal", 31, FUSED)
     check_case(dims, BW, small, "int32", 32, FUSED, in_place=False)
     check_scattered(dims, BW, small, "normal", 36, FUSED)
-    if n <= 27:                                           # four columns per thread (long blocks, >= 2^20 elements)
+    if n <= 27:                                           # two columns per thread (long blocks, >= 2^20 elements)
         wide = (1 << 20) + 300 * n * D + 7
         check_case(dims, BW, wide, "normal", 33, FUSED)
         check_case(dims, BW, wide, "int32", 34, FUSED, in_place=False)
@@ -82,7 +82,7 @@ def test_fused_bandwidth_wide_path_on_729_ranks_sampled():
             (count - 900, count), (123456, 124000)]
     xd, keep = upload_matrix("uniform", 35, 729, count, wins)
     res = run_gpu(plan, xd, FUSED, in_place=False)
-    assert binding.last_kernel_name() == "bw_fused<V=4>"
+    assert binding.last_kernel_name() == "bw_fused<V=2>"
     for (w0, w1), xh in zip(wins, keep):
         compare(dims, BW, xh, res[:, w0:w1].cpu().numpy(), E=count, e0=w0)
 
