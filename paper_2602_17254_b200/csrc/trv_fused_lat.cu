@@ -12,7 +12,7 @@
 //   k_lat_reg   : n <= 81 (rings 3..81, tori 3x3, 9x9, 3x3x3, 3x3x3x3): one group, no shared memory
 //   k_lat_ring  : rings of 243 and 729: steps {1,3} on windows of consecutive ranks with a
 //                 halo of 4, then the remaining steps on the closed sets {q + 9 i}
-//   k_lat_t999_ws (trv_fused_t999.cu): 9x9x9 torus, three groups of two steps, warp-specialised
+//   k_lat_t999 (trv_fused_t999.cu): 9x9x9 torus, three closed groups of two steps each
 #include <type_traits>
 
 #include "trv_dev.cuh"
