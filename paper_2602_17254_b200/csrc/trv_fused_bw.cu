@@ -141,68 +141,94 @@ __device__ __forceinline__ void column_tree(const BwArgs& a, int c, const Tabs& 
     for (int r = 0; r < a.n; ++r) *reinterpret_cast<P*>(tabs.out(r) + e) = res;
 }
 
-// Same value, for short vectors: one column per thread, 27 leaves (three tree levels) loaded at
-// once, so a thread needs n / 27 dependent memory round trips instead of n / 9.  S >= 3.
+// Short vectors: too few columns to fill the GPU with one thread per column, and a thread walking
+// all n leaves needs n / 9 dependent memory round trips.  Here G = 3^(S-L) threads share a column:
+// thread g reduces the g-th subtree of 3^L leaves (one round of independent loads), the G subtree
+// values are combined in tree order through shared memory (S - L rounds of (first + second) +
+// third over neighbours at distance 1, 3, 9), and every thread stores the result to n / G ranks.
+// Block = 32 columns x G threads; a warp reads 128 contiguous bytes of one rank.
+constexpr int coop_L(int S) { return S >= 5 ? 3 : 2; }
+constexpr int coop_G(int S) { return S == 6 ? 27 : (S == 5 ? 9 : (S == 4 ? 9 : 3)); }
+
 template <typename T, int S, int D, typename Tabs>
-__device__ __forceinline__ void column_tree27(const BwArgs& a, int c, const Tabs& tabs, long long e, int j) {
-    int base[D];    // coordinates of the centre of the current 27-leaf chunk
+__device__ __forceinline__ void bw_coop_tile(const BwArgs& a, const Tabs& tabs, T* xch) {
+    constexpr int L = coop_L(S), G = coop_G(S), LEAVES = (L == 3 ? 27 : 9);
+    const int lane = threadIdx.x, g = threadIdx.y;
+    const int c = blockIdx.y;
+    const long long lo = a.lo[c], hi = a.hi[c];
+    const long long e = (lo / 32) * 32 + (long long)blockIdx.x * 32 + lane;
+    const bool live = e >= lo && e < hi;            // every thread takes part in the barriers
+    T val = T(0);
+    if (live) {
+        const unsigned long long len = (unsigned long long)(a.ghi[c] - a.glo[c]);
+        const unsigned long long x0 = (unsigned long long)(a.w0 + e - a.glo[c]);
+        const int j = (int)(((x0 + 1) * (unsigned)a.n - 1) / len);      // owner of the column's block
+        int base[D];
 #pragma unroll
-    for (int d = 0; d < D; ++d) base[d] = (j / a.dstride[d]) % a.dims[d];
+        for (int d = 0; d < D; ++d) base[d] = (j / a.dstride[d]) % a.dims[d];
+        int gg = g;
 #pragma unroll
-    for (int t = 3; t < S; ++t) {   // leftmost chunk: every step >= 3 at eps = -1
-        const int dt = a.ldim[c][t], xt = a.ldist[c][t];
+        for (int t = L; t < S; ++t) {               // centre of this thread's subtree: digits of g, level L lowest
+            const int eps = gg % 3 - 1, dt = a.ldim[c][t], xt = a.ldist[c][t];
+            gg /= 3;
 #pragma unroll
-        for (int d = 0; d < D; ++d) if (d == dt) base[d] = wrap(base[d] - xt, a.dims[d]);
-    }
-    int ldm[3], ldx[3];
+            for (int d = 0; d < D; ++d) if (d == dt) base[d] = wrap(base[d] + eps * xt, a.dims[d]);
+        }
+        int ldm[L], ldx[L];
 #pragma unroll
-    for (int t = 0; t < 3; ++t) { ldm[t] = a.ldim[c][t]; ldx[t] = a.ldist[c][t]; }
-    int vd[S];
-    T acc[S];
+        for (int t = 0; t < L; ++t) { ldm[t] = a.ldim[c][t]; ldx[t] = a.ldist[c][t]; }
+        T l[LEAVES];
 #pragma unroll
-    for (int t = 0; t < S; ++t) vd[t] = 0;
-    constexpr int CHUNKS = (S == 3) ? 1 : (S == 4 ? 3 : (S == 5 ? 9 : 27));
-    T res = T(0);
-    for (int ch = 0; ch < CHUNKS; ++ch) {
-        T l[27];
-#pragma unroll
-        for (int m = 0; m < 27; ++m) {      // leaf m <-> (eps_2, eps_1, eps_0) = (m / 9 - 1, (m / 3) % 3 - 1, m % 3 - 1)
+        for (int m = 0; m < LEAVES; ++m) {          // leaf m <-> eps_t = (m / 3^t) % 3 - 1
             const int eps[3] = {m % 3 - 1, (m / 3) % 3 - 1, m / 9 - 1};
             int rank = 0;
 #pragma unroll
             for (int d = 0; d < D; ++d) {
                 int off = 0;
 #pragma unroll
-                for (int t = 0; t < 3; ++t) off += (ldm[t] == d) ? eps[t] * ldx[t] : 0;
-                int x = base[d] + off;      // |off| < a_d: the steps of one dimension sum to less than its side
-                x = x < 0 ? x + a.dims[d] : (x >= a.dims[d] ? x - a.dims[d] : x);
-                rank += x * a.dstride[d];
+                for (int t = 0; t < L; ++t) off += (ldm[t] == d) ? eps[t] * ldx[t] : 0;
+                rank += wrap(base[d] + off, a.dims[d]) * a.dstride[d];   // |off| < a_d
             }
             l[m] = tabs.in(rank)[e];
         }
-        T r9[3];
+        T r9[LEAVES / 9];
 #pragma unroll
-        for (int g = 0; g < 3; ++g)
-            r9[g] = add3(add3(l[9 * g], l[9 * g + 1], l[9 * g + 2]), add3(l[9 * g + 3], l[9 * g + 4], l[9 * g + 5]),
-                         add3(l[9 * g + 6], l[9 * g + 7], l[9 * g + 8]));
-        T r = add3(r9[0], r9[1], r9[2]);
-        bool carry = true;
-#pragma unroll
-        for (int t = 3; t < S; ++t) {
-            if (carry) {
-                const int dt = a.ldim[c][t], xt = a.ldist[c][t];
-                int delta;
-                if (vd[t] == 0) { acc[t] = r; vd[t] = 1; delta = xt; carry = false; }
-                else if (vd[t] == 1) { acc[t] = add2(acc[t], r); vd[t] = 2; delta = xt; carry = false; }
-                else { r = add2(acc[t], r); vd[t] = 0; delta = -2 * xt; }
-#pragma unroll
-                for (int d = 0; d < D; ++d) if (d == dt) base[d] = wrap(base[d] + delta, a.dims[d]);
-            }
-        }
-        res = r;
+        for (int q = 0; q < LEAVES / 9; ++q)
+            r9[q] = add3(add3(l[9 * q], l[9 * q + 1], l[9 * q + 2]), add3(l[9 * q + 3], l[9 * q + 4], l[9 * q + 5]),
+                         add3(l[9 * q + 6], l[9 * q + 7], l[9 * q + 8]));
+        if constexpr (L == 3) val = add3(r9[0], r9[1], r9[2]);
+        else val = r9[0];
     }
-#pragma unroll 9
-    for (int r = 0; r < a.n; ++r) tabs.out(r)[e] = res;
+    xch[g * 32 + lane] = val;
+    __syncthreads();
+#pragma unroll
+    for (int step = 1; step < G; step *= 3) {
+        if (g % (3 * step) == 0) xch[g * 32 + lane] = add3(xch[g * 32 + lane], xch[(g + step) * 32 + lane], xch[(g + 2 * step) * 32 + lane]);
+        __syncthreads();
+    }
+    const T res = xch[lane];
+    if (live)
+        for (int r = g; r < a.n; r += G) tabs.out(r)[e] = res;
+}
+
+template <typename T, int S, int D, int CAP>
+__global__ void __launch_bounds__(32 * coop_G(S)) k_bw_coop(PtrTab<CAP> in, PtrTab<CAP> out, BwArgs a) {
+    pdl_trigger();
+    __shared__ const T* sin[CAP];
+    __shared__ T* sout[CAP];
+    __shared__ T xch[coop_G(S) * 32];
+    for (int r = threadIdx.y * 32 + threadIdx.x; r < a.n; r += 32 * coop_G(S)) { sin[r] = (const T*)in.p[r]; sout[r] = (T*)out.p[r]; }
+    __syncthreads();
+    pdl_wait();
+    bw_coop_tile<T, S, D>(a, SmemTabs<T>{sin, sout}, xch);
+}
+
+template <typename T, int S, int D>
+__global__ void __launch_bounds__(32 * coop_G(S)) k_bw_coop_strided(StrideAddr in, StrideAddr out, BwArgs a) {
+    pdl_trigger();
+    __shared__ T xch[coop_G(S) * 32];
+    pdl_wait();
+    bw_coop_tile<T, S, D>(a, StrideTabs<T>{in, out}, xch);
 }
 
 template <typename T, int V, int S, int D, typename Tabs>
@@ -218,8 +244,7 @@ __device__ __forceinline__ void bw_tile(const BwArgs& a, const Tabs& tabs) {
         return (int)(((x + 1) * (unsigned)a.n - 1) / L);
     };
     if constexpr (V == 1) {
-        if constexpr (S >= 3) column_tree27<T, S, D>(a, c, tabs, e, owner(e));
-        else column_tree<T, 1, S, D>(a, c, tabs, e, owner(e));
+        column_tree<T, 1, S, D>(a, c, tabs, e, owner(e));
     } else {
         const bool inside = e >= lo && e + V <= hi;
         int j0 = 0;
@@ -270,13 +295,29 @@ static void launch_bw(const Call& c, const BwArgs& a) {
         }
     if (tiles == 0) return;
     StrideAddr sin, sout;
-    if (uniform_stride(c.in, p.n, &sin) && uniform_stride((const void* const*)c.out, p.n, &sout)) {
+    const bool strided = uniform_stride(c.in, p.n, &sin) && uniform_stride((const void* const*)c.out, p.n, &sout);
+    if constexpr (V == 1 && S >= 3) {       // short vectors: several threads per column
+        long long ct = 0;
+        for (int sl = 0; sl < D; ++sl)
+            if (a.hi[sl] > a.lo[sl]) {
+                const long long t = (a.hi[sl] - (a.lo[sl] / 32) * 32 + 31) / 32;
+                if (t > ct) ct = t;
+            }
+        const dim3 grid((unsigned)ct, D, 1), block(32, coop_G(S), 1);
+        if (strided) {
+            launch_pdl(k_bw_coop_strided<T, S, D>, grid, block, 0, c.st, sin, sout, a);
+        } else {
+            PtrTab<CAP> in, out;
+            for (int r = 0; r < p.n; ++r) { in.p[r] = const_cast<void*>(c.in[r]); out.p[r] = c.out[r]; }
+            launch_pdl(k_bw_coop<T, S, D, CAP>, grid, block, 0, c.st, in, out, a);
+        }
+    } else if (strided) {
         launch_pdl(k_bw_fused_strided<T, V, S, D>, dim3((unsigned)tiles, D, 1), dim3(kBwThreads), 0, c.st, sin, sout, a);
-        return;
+    } else {
+        PtrTab<CAP> in, out;
+        for (int r = 0; r < p.n; ++r) { in.p[r] = const_cast<void*>(c.in[r]); out.p[r] = c.out[r]; }
+        launch_pdl(k_bw_fused<T, V, S, D, CAP>, dim3((unsigned)tiles, D, 1), dim3(kBwThreads), 0, c.st, in, out, a);
     }
-    PtrTab<CAP> in, out;
-    for (int r = 0; r < p.n; ++r) { in.p[r] = const_cast<void*>(c.in[r]); out.p[r] = c.out[r]; }
-    launch_pdl(k_bw_fused<T, V, S, D, CAP>, dim3((unsigned)tiles, D, 1), dim3(kBwThreads), 0, c.st, in, out, a);
 }
 
 template <typename T, int V, int S>
@@ -321,10 +362,10 @@ trv_status_t run_fused_bandwidth(const Call& c) {
     }
     // Two columns per thread (8-byte accesses, packed adds) when blocks are long enough that few
     // threads straddle a block boundary and the vector is long enough to fill the GPU with such
-    // threads; one column per thread otherwise (every thread then has its own owner).  Measured on
-    // B200: two columns beat four at every size (shorter thread lifetimes, more warps per SM).
+    // threads; otherwise several threads per column (k_bw_coop; n <= 9: one thread per column).
+    // Measured on B200: two columns beat four at every size (shorter thread lifetimes, more warps).
     const bool wide = min_block >= 256 && c.count >= ((size_t)1 << 20);
-    g_last_kernel = wide ? "bw_fused<V=2>" : "bw_fused<V=1>";
+    g_last_kernel = wide ? "bw_fused<V=2>" : (p.S >= 3 ? "bw_coop" : "bw_fused<V=1>");
     trv_status_t st;
     if (c.dtype == TRV_FLOAT32) st = wide ? bw_by_s<float, 2>(c, a) : bw_by_s<float, 1>(c, a);
     else st = wide ? bw_by_s<uint32_t, 2>(c, a) : bw_by_s<uint32_t, 1>(c, a);
