@@ -203,6 +203,27 @@ trv_status_t trv_link_loads(trv_plan_t plan, size_t count, size_t elem_size, int
 trv_status_t trv_plan_message_bytes(trv_plan_t plan, size_t count, size_t elem_size, int32_t c, int32_t row,
                                     int64_t *bytes);
 
+/* ---------------------------------------------------------------- cost model
+ *
+ * Congestion-aware cost of the plan's schedule (Sec. 2.1):
+ *     C(m, A) = steps(A) * alpha + sum_k beta * m_k * c_k,
+ * where the product m_k * c_k of step k is taken as the largest number of bytes any directed link
+ * carries in that step (for Trivance every link carries exactly chunk size x congestion).  The
+ * link loads come from the same GPU tally as trv_link_loads; synchronous.
+ *   alpha: start-up latency per step (seconds); beta: seconds per byte (1 / link bandwidth)
+ * Besides the cost, the three optimality factors of Tables 1 and 2 are returned:
+ *   lambda = steps / log3 n                        (latency;   Trivance: 1 or 2)
+ *   delta  = bytes a node sends in total / (2 m)   (bandwidth; m = count * elem_size)
+ *   theta  = sum_k m_k c_k / (m / D)               (transmission delay) */
+typedef struct {
+    int32_t steps;
+    int64_t bytes_sent_per_node;    /* maximum over nodes */
+    int64_t tx_bytes;               /* sum over steps of the most loaded link's bytes */
+    double latency_term, tx_term, total;   /* seconds */
+    double lambda, delta, theta;
+} trv_cost_t;
+trv_status_t trv_cost_model(trv_plan_t plan, size_t count, size_t elem_size, double alpha, double beta, trv_cost_t *out);
+
 /* ---------------------------------------------------------------- misc */
 
 const char *trv_strerror(trv_status_t status);

@@ -6,6 +6,6 @@ imports it.
 """
 from .oracle import (  # noqa: F401
     ALGO_BRUCK, ALGO_RECDOUB, ALGO_TRIVANCE, VARIANT_BANDWIDTH, VARIANT_LATENCY,
-    OracleError, allreduce, block_bounds, block_propagation, build, link_loads,
+    OracleError, allreduce, block_bounds, bytes_sent, cost_model, block_propagation, build, link_loads,
     naive_sum_f32, num_steps, peers, send_set, step_list,
 )

@@ -170,3 +170,28 @@ def link_loads(dims, variant, E, elem_size=4, algo=ALGO_TRIVANCE):
                                   byts.ctypes.data_as(ctypes.c_void_p), mm.ctypes.data_as(ctypes.c_void_p),
                                   mb.ctypes.data_as(ctypes.c_void_p)))
     return {"msgs": msgs, "bytes": byts, "max_msgs": mm, "max_bytes": mb}
+
+
+def bytes_sent(dims, variant, E, elem_size=4, algo=ALGO_TRIVANCE):
+    """[n] int64: bytes every node sends over the whole AllReduce."""
+    _, p, nd = _dims(dims)
+    n, _ = num_steps(dims, algo)
+    out = np.zeros(n, np.int64)
+    _check(_load().orc_bytes_sent(p, nd, ctypes.c_int(variant), ctypes.c_int(algo), ctypes.c_int64(E),
+                                  ctypes.c_int64(elem_size), out.ctypes.data_as(ctypes.c_void_p)))
+    return out
+
+
+def cost_model(dims, variant, E, elem_size, alpha, beta, algo=ALGO_TRIVANCE):
+    """Sec. 2.1: C = steps * alpha + sum_k beta * m_k * c_k, with m_k * c_k = bytes on the most loaded
+    link of step k; plus the optimality factors of Tables 1 and 2 (lambda, delta, theta)."""
+    ll = link_loads(dims, variant, E, elem_size, algo)
+    n, _ = num_steps(dims, algo)
+    T = ll["max_bytes"].size
+    tx = int(ll["max_bytes"].sum())
+    sent = int(bytes_sent(dims, variant, E, elem_size, algo).max())
+    m = float(E) * float(elem_size)
+    D = len(np.atleast_1d(dims))
+    return {"steps": T, "bytes_sent_per_node": sent, "tx_bytes": tx, "latency_term": T * alpha, "tx_term": beta * tx,
+            "total": T * alpha + beta * tx, "lambda": T / (np.log(n) / np.log(3.0)), "delta": sent / (2.0 * m),
+            "theta": tx / (m / D)}

@@ -413,6 +413,60 @@ int orc_allreduce(const int32_t *dims, int ndims, int variant, int dtype,
     return ORC_OK;
 }
 
+/* ------------------------------------------------------------------ bytes sent per node */
+
+/*
+ * Total bytes every node sends over the whole AllReduce (both phases of the bandwidth form), by
+ * walking every message of every step (Sec. 2.3: bandwidth optimality is relative to 2m).
+ * sent: [n] int64.
+ */
+int orc_bytes_sent(const int32_t *dims, int ndims, int variant, int algo, int64_t E, int64_t elem_size, int64_t *sent) {
+    orc_topo tp; int rc = topo_init(&tp, dims, ndims, algo);
+    if (rc) return rc;
+    if (E < 0 || elem_size < 1 || !sent) return ORC_BAD_ARG;
+    if (variant != ORC_LATENCY && variant != ORC_BANDWIDTH) return ORC_BAD_ARG;
+    int n = tp.n, D = tp.ndims, S = tp.S, T = (variant == ORC_BANDWIDTH) ? 2 * S : S;
+    uint8_t *set = (uint8_t *)malloc((size_t)n);
+    uint8_t *have = (uint8_t *)malloc((size_t)n * n), *snap = (uint8_t *)malloc((size_t)n * n);
+    int64_t *blen = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);
+    if (!set || !have || !snap || !blen) { free(set); free(have); free(snap); free(blen); return ORC_NOMEM; }
+    memset(sent, 0, sizeof(int64_t) * (size_t)n);
+    for (int c = 0; c < D; ++c) {
+        int sd[64], sx[64];
+        int64_t slo, shi;
+        step_list(&tp, c, sd, sx);
+        slice_bounds(E, D, c, &slo, &shi);
+        for (int j = 0; j < n; ++j) blen[j] = block_bound(slo, shi, n, j + 1) - block_bound(slo, shi, n, j);
+        memset(have, 0, (size_t)n * n);
+        for (int r = 0; r < n; ++r) have[(size_t)r * n + r] = 1;
+        for (int row = 0; row < T; ++row) {
+            int t = (row < S) ? row : (2 * S - 1 - row);
+            if (row >= S) memcpy(snap, have, (size_t)n * n);
+            for (int r = 0; r < n; ++r) {
+                int peer[2], dir[2], hops[2];
+                int np = send_peers(&tp, r, sd[t], sx[t], peer, dir, hops);
+                for (int i = 0; i < np; ++i) {
+                    int64_t mbytes = 0;
+                    if (variant == ORC_LATENCY) {
+                        mbytes = (shi - slo) * elem_size;
+                    } else if (row < S) {
+                        send_set(&tp, sd, sx, peer[i], t, set);
+                        for (int j = 0; j < n; ++j) if (set[j]) mbytes += blen[j] * elem_size;
+                    } else {
+                        for (int j = 0; j < n; ++j) if (snap[(size_t)r * n + j]) {
+                            mbytes += blen[j] * elem_size;
+                            have[(size_t)peer[i] * n + j] = 1;
+                        }
+                    }
+                    sent[r] += mbytes;
+                }
+            }
+        }
+    }
+    free(set); free(have); free(snap); free(blen);
+    return ORC_OK;
+}
+
 /* ------------------------------------------------------------------ link loads */
 
 /*

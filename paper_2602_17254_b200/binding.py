@@ -27,8 +27,15 @@ SYMBOLS = [
     "trv_plan_peers", "trv_plan_send_set", "trv_plan_block_bounds", "trv_allreduce", "trv_scratch_bytes",
     "trv_kernel_supported", "trv_allreduce_ex", "trv_allreduce_host", "trv_host_workspace_bytes",
     "trv_link_loads", "trv_plan_message_bytes", "trv_strerror", "trv_launch_count", "trv_last_kernel_name",
-    "trv_allreduce_noalloc", "trv_noalloc_max_scratch_bytes",
+    "trv_allreduce_noalloc", "trv_noalloc_max_scratch_bytes", "trv_cost_model",
 ]
+
+
+class Cost(ctypes.Structure):
+    """trv_cost_t"""
+    _fields_ = [("steps", ctypes.c_int32), ("bytes_sent_per_node", ctypes.c_int64), ("tx_bytes", ctypes.c_int64),
+                ("latency_term", ctypes.c_double), ("tx_term", ctypes.c_double), ("total", ctypes.c_double),
+                ("lambda_", ctypes.c_double), ("delta", ctypes.c_double), ("theta", ctypes.c_double)]
 
 _lib = None
 
@@ -68,6 +75,7 @@ def lib():
         L.trv_allreduce_host.argtypes = [vp, vp, vp, sz, ctypes.c_int, ctypes.c_int, vp, sz, vp]
         L.trv_host_workspace_bytes.argtypes = [vp, sz, ctypes.POINTER(sz)]
         L.trv_link_loads.argtypes = [vp, sz, sz, vp, vp, vp, vp]
+        L.trv_cost_model.argtypes = [vp, sz, sz, ctypes.c_double, ctypes.c_double, ctypes.POINTER(Cost)]
         L.trv_strerror.argtypes = [ctypes.c_int]
         L.trv_strerror.restype = ctypes.c_char_p
         L.trv_launch_count.argtypes = []
@@ -215,6 +223,12 @@ class Plan:
         _check(lib().trv_link_loads(self._h, count, elem_size, _np_ptr(msgs), _np_ptr(byts), _np_ptr(mm), _np_ptr(mb)),
                "trv_link_loads")
         return {"msgs": msgs, "bytes": byts, "max_msgs": mm, "max_bytes": mb}
+
+
+    def cost_model(self, count, elem_size, alpha, beta):
+        c = Cost()
+        _check(lib().trv_cost_model(self._h, count, elem_size, float(alpha), float(beta), ctypes.byref(c)), "trv_cost_model")
+        return c
 
 
 # ---------------------------------------------------------------- torch conveniences (marshalling only)

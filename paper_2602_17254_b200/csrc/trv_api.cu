@@ -1,5 +1,6 @@
 // C ABI of the Trivance engine: argument checks, kernel-family choice, host-buffer variant.
 #include <algorithm>
+#include <cmath>
 #include <cstring>
 #include <vector>
 
@@ -247,6 +248,42 @@ trv_status_t trv_link_loads(trv_plan_t plan, size_t count, size_t elem_size, int
                             int32_t* max_msgs, int64_t* max_bytes) {
     if (!plan || elem_size == 0) return TRV_ERR_INVALID_ARG;
     return run_link_loads(plan->plan, count, elem_size, msgs, bytes, max_msgs, max_bytes);
+}
+
+trv_status_t trv_cost_model(trv_plan_t plan, size_t count, size_t elem_size, double alpha, double beta, trv_cost_t* out) {
+    if (!plan || !out || elem_size == 0 || !(alpha >= 0) || !(beta >= 0)) return TRV_ERR_INVALID_ARG;
+    const Plan& p = plan->plan;
+    const int T = p.rows(), n = p.n, D = p.ndims;
+    std::vector<int64_t> max_bytes((size_t)T), mb((size_t)n), sent((size_t)n, 0);
+    trv_status_t st = run_link_loads(p, count, elem_size, nullptr, nullptr, nullptr, max_bytes.data());
+    if (st != TRV_OK) return st;
+    // bytes every node sends: Reduce-Scatter / latency rows are indexed by destination, AllGather rows by source
+    for (int c = 0; c < D; ++c)
+        for (int row = 0; row < T; ++row) {
+            message_bytes(p, (int64_t)count, (int64_t)elem_size, c, row, mb.data());
+            const Step& s = p.steps[c][p.step_of_row(row)];
+            const bool by_source = p.variant == TRV_BANDWIDTH_OPTIMAL && row >= p.S;
+            for (int r = 0; r < n; ++r) {
+                int peer[2], dir[2], hops[2];
+                const int np = send_peers(p, r, s.dim, s.dist, peer, dir, hops);
+                for (int i = 0; i < np; ++i) sent[r] += by_source ? mb[r] : mb[peer[i]];
+            }
+        }
+    int64_t tx = 0, smax = 0;
+    for (int row = 0; row < T; ++row) tx += max_bytes[row];
+    for (int r = 0; r < n; ++r) smax = std::max(smax, sent[r]);
+    const double m = (double)count * (double)elem_size;
+    const double log3n = std::log((double)n) / std::log(3.0);
+    out->steps = T;
+    out->bytes_sent_per_node = smax;
+    out->tx_bytes = tx;
+    out->latency_term = T * alpha;
+    out->tx_term = beta * (double)tx;
+    out->total = out->latency_term + out->tx_term;
+    out->lambda = log3n > 0 ? T / log3n : 0;
+    out->delta = m > 0 ? (double)smax / (2.0 * m) : 0;
+    out->theta = m > 0 ? (double)tx / (m / D) : 0;
+    return TRV_OK;
 }
 
 const char* trv_strerror(trv_status_t status) {

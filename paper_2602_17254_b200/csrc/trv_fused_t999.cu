@@ -12,10 +12,11 @@
 // Between groups the tile stays in shared memory; inside a group every set is read and written by
 // one thread only, so the two barriers between the groups are the only synchronisation.
 // A thread owns V adjacent columns (V = 1: 288 threads; V = 2: packed adds, 144 threads) of one
-// ninth of the sets.  Measured on B200 (729 x 32 MiB): V = 1 with direct loads 9.96 ms, V = 2
-// 10.8 ms, V = 2 with asynchronous global->shared staging 10.8 ms, two groups with an 81-value
-// register set 13.8 ms, a warp-specialised persistent variant 13.1 ms: what counts is the number
-// of warps that have loads in flight, not the instruction count.
+// ninth of the sets.  Measured on B200 (729 x 32 MiB): V = 1 9.96 ms, V = 2 10.8 ms; staging the
+// plane with asynchronous global->shared copies, two groups with an 81-value register set,
+// persistent and warp-specialised variants were all slower (10.8 - 14 ms): what counts is the
+// number of warps that have loads in flight, not the instruction count.  With 288 threads the
+// register file allows two CTAs per SM only up to 96 registers per thread.
 #include "trv_dev.cuh"
 #include "trv_fused_lat.cuh"
 
@@ -28,16 +29,7 @@ struct Rot {
     static constexpr int sC = ROT == 0 ? 81 : (ROT == 1 ? 1 : 9);
 };
 
-__device__ __forceinline__ void cp_async_bytes(void* smem_dst, const void* gmem_src, int bytes) {
-    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
-    if (bytes == 8) asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(d), "l"(gmem_src) : "memory");
-    else asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() {
-    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
-}
-
-template <typename T, int ROT, int V, bool ASYNC, bool FULL, typename Addr>
+template <typename T, int ROT, int V, bool FULL, typename Addr>
 __device__ __forceinline__ void t999_body(const Addr& in, const Addr& out, const LatArgs& a, T* slab, long long t0) {
     using R = Rot<ROT>;
     using E = Elem<T, V>;
@@ -49,23 +41,9 @@ __device__ __forceinline__ void t999_body(const Addr& in, const Addr& out, const
     auto sl = [&](int r) -> E& { return *reinterpret_cast<E*>(mine + r * 32); };
     {   // ---- group 1: (A,1) (B,1) on the plane C = set
         const int r0 = set * R::sC;
-        constexpr bool STAGED = ASYNC && FULL;
-        if constexpr (STAGED) {
-            // asynchronous global -> shared copies of the thread's own plane: all 81 in flight at once,
-            // no registers held; only the issuing thread reads them back, so no barrier is needed
-#pragma unroll
-            for (int idx = 0; idx < 81; ++idx) {
-                const int r = r0 + (idx % 9) * R::sA + (idx / 9) * R::sB;
-                cp_async_bytes(&sl(r), in.ptr(r) + e * (long long)sizeof(T), V * 4);
-            }
-            cp_async_wait_all();
-        }
         auto load_row = [&](int j, E (&row)[9]) {
 #pragma unroll
-            for (int i = 0; i < 9; ++i) {
-                if constexpr (STAGED) row[i] = sl(r0 + i * R::sA + j * R::sB);
-                else row[i] = load_elem<T, V, FULL>(in.ptr(r0 + i * R::sA + j * R::sB), e, lo, hi);
-            }
+            for (int i = 0; i < 9; ++i) row[i] = load_elem<T, V, FULL>(in.ptr(r0 + i * R::sA + j * R::sB), e, lo, hi);
             reg_step<9, 1, 9, 1>(row);                                      // (A,1)
         };
         auto emit = [&](int j, const E (&p)[9], const E (&q)[9], const E (&r)[9]) {     // (B,1) for row j
@@ -119,7 +97,7 @@ __device__ __forceinline__ void t999_body(const Addr& in, const Addr& out, const
     }
 }
 
-template <typename T, int V, bool ASYNC, typename Addr>
+template <typename T, int V, typename Addr>
 __global__ void __launch_bounds__(288 / V, 2) k_lat_t999(Addr in, Addr out, LatArgs a) {
     pdl_trigger();
     extern __shared__ uint4 slab_raw[];
@@ -129,14 +107,14 @@ __global__ void __launch_bounds__(288 / V, 2) k_lat_t999(Addr in, Addr out, LatA
     if (t0 >= a.hi[c]) return;
     pdl_wait();
     const bool full = t0 >= a.lo[c] && t0 + 32 <= a.hi[c];
-    if (c == 0) { if (full) t999_body<T, 0, V, ASYNC, true>(in, out, a, slab, t0); else t999_body<T, 0, V, ASYNC, false>(in, out, a, slab, t0); }
-    else if (c == 1) { if (full) t999_body<T, 1, V, ASYNC, true>(in, out, a, slab, t0); else t999_body<T, 1, V, ASYNC, false>(in, out, a, slab, t0); }
-    else { if (full) t999_body<T, 2, V, ASYNC, true>(in, out, a, slab, t0); else t999_body<T, 2, V, ASYNC, false>(in, out, a, slab, t0); }
+    if (c == 0) { if (full) t999_body<T, 0, V, true>(in, out, a, slab, t0); else t999_body<T, 0, V, false>(in, out, a, slab, t0); }
+    else if (c == 1) { if (full) t999_body<T, 1, V, true>(in, out, a, slab, t0); else t999_body<T, 1, V, false>(in, out, a, slab, t0); }
+    else { if (full) t999_body<T, 2, V, true>(in, out, a, slab, t0); else t999_body<T, 2, V, false>(in, out, a, slab, t0); }
 }
 
-template <typename T, int V, bool ASYNC, typename Addr>
+template <typename T, int V, typename Addr>
 static trv_status_t launch_t999_v(const Call& c, const Addr& in, const Addr& out, const LatArgs& a, long long tiles_x) {
-    auto kfn = k_lat_t999<T, V, ASYNC, Addr>;
+    auto kfn = k_lat_t999<T, V, Addr>;
     constexpr size_t smem = 729 * 32 * sizeof(T);
     static const cudaError_t once = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (once != cudaSuccess) return TRV_ERR_CUDA;
@@ -156,7 +134,7 @@ static trv_status_t launch_t999(const Call& c, const Addr& in, const Addr& out, 
     if (tiles_x > (1LL << 30)) return TRV_ERR_UNSUPPORTED;
     // One column per thread and direct loads measured fastest on B200: 18 warps per SM matter more
     // than packed adds or asynchronous staging here.
-    return launch_t999_v<T, 1, false>(c, in, out, a, tiles_x);
+    return launch_t999_v<T, 1>(c, in, out, a, tiles_x);
 }
 
 trv_status_t run_fused_t999(const Call& c, const LatArgs& a) {

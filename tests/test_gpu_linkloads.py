@@ -72,3 +72,19 @@ def test_config1_and_config5_tables():
     with pytest.raises(binding.TrivanceError) as e:
         binding.Plan((243,), LAT, binding.ALGO_RECDOUB)
     assert e.value.status == binding.ERR_UNDEFINED_SCHEDULE
+
+
+@pytest.mark.parametrize("dims,algo", [((9,), binding.ALGO_TRIVANCE), ((243,), binding.ALGO_TRIVANCE), ((9, 9, 9), binding.ALGO_TRIVANCE),
+                                       ((3, 9), binding.ALGO_TRIVANCE), ((27,), binding.ALGO_BRUCK), ((64,), binding.ALGO_RECDOUB)])
+@pytest.mark.parametrize("variant", [LAT, BW])
+def test_cost_model_matches_oracle(dims, algo, variant):
+    """trv_cost_model (Sec. 2.1 cost, Table 1/2 factors) vs the oracle's: integers exact, doubles to rounding."""
+    alpha, beta = 1.5e-6, 1.0 / 100e9
+    for count in (100003, 8192):
+        got = binding.Plan(dims, variant, algo).cost_model(count, 4, alpha, beta)
+        want = oracle.cost_model(dims, variant, count, 4, alpha, beta, algo=algo)
+        assert got.steps == want["steps"] and got.bytes_sent_per_node == want["bytes_sent_per_node"]
+        assert got.tx_bytes == want["tx_bytes"]
+        for name, key in [("latency_term", "latency_term"), ("tx_term", "tx_term"), ("total", "total"), ("lambda_", "lambda"),
+                          ("delta", "delta"), ("theta", "theta")]:
+            assert np.isclose(getattr(got, name), want[key], rtol=1e-12, atol=0), name

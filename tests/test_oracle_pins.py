@@ -461,3 +461,50 @@ def test_slices_follow_different_step_orders():
     swapped = oracle.allreduce(dims, LAT, np.concatenate([x[:, 32:], x[:, :32]], axis=1))
     assert not np.array_equal(out[:, :32], swapped[:, 32:])
     assert np.allclose(out[:, :32], swapped[:, 32:], rtol=1e-4, atol=1e-4)
+
+
+# ------------------------------------------------------------------ cost model and optimality factors (Sec. 2.1, Tables 1 and 2)
+
+@pytest.mark.parametrize("n", [9, 27, 81, 243])
+def test_table1_factors_on_rings(n):
+    """Table 1: Trivance (B) = (2, 1, 2/3 log3 n), Trivance (L) = (1, log3 n, n/2),
+    Bruck (B) = (2, 1, 2 log3 n), Bruck (L) = (1, log3 n, 3n/2); 1 stands for 1 - 1/n and n/2 for (n-1)/2."""
+    s = round(np.log(n) / np.log(3))
+    E = 3 * n
+    tb = oracle.cost_model((n,), BW, E, 4, 0.0, 1.0)
+    tl = oracle.cost_model((n,), LAT, E, 4, 0.0, 1.0)
+    bb = oracle.cost_model((n,), BW, E, 4, 0.0, 1.0, algo=oracle.ALGO_BRUCK)
+    bl = oracle.cost_model((n,), LAT, E, 4, 0.0, 1.0, algo=oracle.ALGO_BRUCK)
+    assert np.isclose(tb["lambda"], 2) and np.isclose(tb["delta"], 1 - 1 / n) and np.isclose(tb["theta"], 2 * s / 3)
+    assert np.isclose(tl["lambda"], 1) and np.isclose(tl["delta"], s) and np.isclose(tl["theta"], (n - 1) / 2)
+    assert np.isclose(bb["lambda"], 2) and np.isclose(bb["delta"], 1 - 1 / n) and np.isclose(bb["theta"], 2 * s)
+    assert np.isclose(bl["lambda"], 1) and np.isclose(bl["delta"], s) and np.isclose(bl["theta"], 3 * (n - 1) / 2)
+
+
+@pytest.mark.parametrize("q", [3, 4, 6])
+def test_table1_recursive_doubling_latency_row(q):
+    """Table 1: Rec.Doub. (L) = (log2 3, log2 n / 2, n); n stands for n - 1 (App. B: sum of 2^k)."""
+    n = 2 ** q
+    c = oracle.cost_model((n,), LAT, 4 * n, 4, 0.0, 1.0, algo=oracle.ALGO_RECDOUB)
+    assert np.isclose(c["lambda"], np.log2(3)) and np.isclose(c["delta"], q / 2) and np.isclose(c["theta"], n - 1)
+
+
+def test_cost_is_steps_alpha_plus_beta_times_weighted_bytes():
+    """Sec. 2.1: C(m, A) = steps * alpha + sum_k beta * m_k * c_k, written out for the 9-ring:
+    latency form m_k = m, c_k = 1, 3; bandwidth form m_k = m/3, m/9 (and the mirror), c_k = 1, 3."""
+    m = 4 * 9 * 5
+    alpha, beta = 1.5e-6, 1.0 / 100e9
+    lat = oracle.cost_model((9,), LAT, 45, 4, alpha, beta)
+    bw = oracle.cost_model((9,), BW, 45, 4, alpha, beta)
+    assert np.isclose(lat["total"], 2 * alpha + beta * (m * 1 + m * 3))
+    assert np.isclose(bw["total"], 4 * alpha + beta * 2 * (m / 3 * 1 + m / 9 * 3))
+    assert lat["steps"] == 2 and bw["steps"] == 4
+
+
+def test_table2_latency_form_on_tori():
+    """Table 2: Trivance (L) = D/2 * n^(1/D) (exactly D (a-1)/2), Bruck (L) three times that."""
+    for dims in [(9, 9), (9, 9, 9), (27, 27)]:
+        D, a, n = len(dims), dims[0], int(np.prod(dims))
+        t = oracle.cost_model(dims, LAT, n * D, 4, 0.0, 1.0)
+        b = oracle.cost_model(dims, LAT, n * D, 4, 0.0, 1.0, algo=oracle.ALGO_BRUCK)
+        assert np.isclose(t["theta"], D * (a - 1) / 2) and np.isclose(b["theta"], 3 * D * (a - 1) / 2)
