@@ -210,7 +210,7 @@ def run_ours(args, w):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     dist = None
-    if world > 1:
+    if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:       # launched by torchrun: one rank per GPU over NCCL
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
