@@ -111,15 +111,17 @@ struct TabAddr {
 };
 struct StrideAddr {
     char* base;
-    long long stride;   // bytes
-    __device__ __forceinline__ char* ptr(int rank) const { return base + (long long)rank * stride; }
+    unsigned stride;    // bytes; 32-bit so that base + stride * rank is ONE 32x32->64 multiply-add
+    __device__ __forceinline__ char* ptr(int rank) const { return base + (unsigned long long)stride * (unsigned)rank; }
 };
-// true (and base/stride filled) iff p[r] == p[0] + r * stride for all r
+// true (and base/stride filled) iff p[r] == p[0] + r * stride for all r with 0 <= stride < 2^32
 inline bool uniform_stride(const void* const* p, int n, StrideAddr* out) {
     out->base = (char*)const_cast<void*>(p[0]);
-    out->stride = n > 1 ? (long long)((const char*)p[1] - (const char*)p[0]) : 0;
+    const long long st = n > 1 ? (long long)((const char*)p[1] - (const char*)p[0]) : 0;
+    if (st < 0 || st > 0xffffffffLL) return false;
+    out->stride = (unsigned)st;
     for (int r = 2; r < n; ++r)
-        if ((const char*)p[r] - (const char*)p[r - 1] != out->stride) return false;
+        if ((const char*)p[r] - (const char*)p[r - 1] != st) return false;
     return true;
 }
 
