@@ -244,14 +244,15 @@ def run_ours(args, w):
             ins[b].normal_(generator=g) if w.dist == "normal" else ins[b].uniform_(-1.0, 1.0, generator=g)
     in_ptrs = [binding.ptr_array([ins[b, r].data_ptr() for r in range(n)]) for b in range(batch)]
     out_ptrs = [binding.ptr_array([outs[b, r].data_ptr() for r in range(n)]) for b in range(batch)]
-    need = plan.scratch_bytes(count, binding.KERNEL_AUTO, in_place=False)
+    kfam = {"auto": binding.KERNEL_AUTO, "step": binding.KERNEL_STEP, "fused": binding.KERNEL_FUSED}[args.kernel]
+    need = plan.scratch_bytes(count, kfam, in_place=False)
     scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
     sh = stream.cuda_stream
 
     def step():
         for b in range(batch):
-            plan.allreduce_ex(in_ptrs[b], out_ptrs[b], count, dcode, kernel=binding.KERNEL_AUTO,
+            plan.allreduce_ex(in_ptrs[b], out_ptrs[b], count, dcode, kernel=kfam,
                               scratch_ptr=scratch.data_ptr() if need else 0, scratch_bytes=need,
                               stream=torch.cuda.current_stream().cuda_stream)
 
@@ -371,7 +372,7 @@ def run_ours(args, w):
                        "ranks": n, "bytes_per_rank": w.bytes_per_rank, "calls_per_step": batch,
                        "l2": "each step touches %d distinct buffer sets = %.0f MiB read + %.0f MiB written (L2 is 126 MiB): "
                              "inputs larger than L2, no flush" % (batch, batch * set_bytes / 2**20, batch * set_bytes / 2**20),
-                       "kernel": kernel_name, "call": "trv_allreduce_ex, separate output buffers, TRV_KERNEL_AUTO"
+                       "kernel": kernel_name, "call": "trv_allreduce_ex, separate output buffers, TRV_KERNEL_%s" % args.kernel.upper()
                        + (", one step captured in a CUDA graph and replayed" if args.graph else ""),
                        "parallelism": "replicas" if world > 1 else "single GPU"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -406,6 +407,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-check", action="store_true", help="skip the parity spot check")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--kernel", default="auto", choices=["auto", "step", "fused"],
+                    help="kernel family (step = one launch per schedule step, as the paper states the steps)")
     ap.add_argument("--graph", action="store_true", help="capture one step in a CUDA graph and time its replays")
     ap.add_argument("--count", type=int, default=0, help="override the workload's elements per rank")
     ap.add_argument("--profile", action="store_true",
