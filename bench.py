@@ -407,6 +407,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-check", action="store_true", help="skip the parity spot check")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--dims", default="", help="ad-hoc torus sides, e.g. 27,27 (overrides the workload's topology)")
+    ap.add_argument("--variant", default="latency", choices=["latency", "bandwidth"], help="form for --dims")
     ap.add_argument("--kernel", default="auto", choices=["auto", "step", "fused"],
                     help="kernel family (step = one launch per schedule step, as the paper states the steps)")
     ap.add_argument("--graph", action="store_true", help="capture one step in a CUDA graph and time its replays")
@@ -419,6 +421,10 @@ def main():
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     w = synth.CONFIGS[args.workload]
+    if args.dims:       # ad-hoc topology: same recipe (float32 N(0,1)), for shapes outside the named configurations
+        dims = tuple(int(v) for v in args.dims.split(","))
+        variant = synth.LATENCY if args.variant == "latency" else synth.BANDWIDTH
+        w = synth.Workload("adhoc_%s_%s" % ("x".join(map(str, dims)), args.variant), dims, variant, w.count, "normal", 9)
     if args.count:      # same topology and form, shorter vectors (small cases for ncu captures)
         w = synth.Workload(w.name + "@%d" % args.count, w.dims, w.variant, args.count, w.dist, w.seed)
     if args.impl == "reference":

@@ -138,14 +138,16 @@ __global__ void __launch_bounds__(288 / V) k_lat_ring(Addr in, Addr out, LatArgs
 
 // ------------------------------------------------------------------ host side
 
-enum class LatKind { None, Reg, Ring, T999 };
+enum class LatKind { None, Reg, Ring, T999, Lines };
 
 static LatKind classify(const Plan& p) {
-    if (p.algo != TRV_ALGO_TRIVANCE || p.variant != TRV_LATENCY_OPTIMAL || !p.equal_dims) return LatKind::None;
-    if (p.n <= 81 && p.ndims <= 4) return LatKind::Reg;
-    if (p.ndims == 1 && (p.n == 243 || p.n == 729)) return LatKind::Ring;
-    if (p.ndims == 3 && p.dims[0] == 9) return LatKind::T999;
-    return LatKind::None;
+    if (p.algo != TRV_ALGO_TRIVANCE || p.variant != TRV_LATENCY_OPTIMAL) return LatKind::None;
+    if (p.equal_dims) {
+        if (p.n <= 81 && p.ndims <= 4) return LatKind::Reg;
+        if (p.ndims == 1 && (p.n == 243 || p.n == 729)) return LatKind::Ring;
+        if (p.ndims == 3 && p.dims[0] == 9) return LatKind::T999;
+    }
+    return fused_lines_supported(p) ? LatKind::Lines : LatKind::None;     // 27x27, unequal sides, ...
 }
 
 bool fused_latency_supported(const Plan& p) { return classify(p) != LatKind::None; }
@@ -211,6 +213,9 @@ static trv_status_t lat_fused_launch(const Call& c, const Addr& in, const Addr& 
     } else if (kind == LatKind::T999) {
         g_last_kernel = "lat_t999";
         return run_fused_t999(c, a);
+    } else if (kind == LatKind::Lines) {
+        g_last_kernel = "lat_lines";
+        return run_fused_lines(c, a);
     } else {
         return TRV_ERR_UNSUPPORTED;
     }

@@ -58,5 +58,7 @@ struct LatArgs {
 };
 
 trv_status_t run_fused_t999(const Call& c, const LatArgs& a);
+bool fused_lines_supported(const Plan& p);
+trv_status_t run_fused_lines(const Call& c, const LatArgs& a);
 
 }  // namespace trv

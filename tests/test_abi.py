@@ -104,7 +104,8 @@ def test_scratch_and_support_queries(library):
     assert lat27.scratch_bytes(1000, binding.KERNEL_STEP, in_place=False) == 27 * 1024 * 4
     lat9 = binding.Plan([9], binding.LATENCY_OPTIMAL)
     assert lat9.scratch_bytes(64, binding.KERNEL_STEP) == 9 * 64 * 4
-    odd = binding.Plan([27, 9], binding.LATENCY_OPTIMAL)                # no fused kernel for unequal sides
+    assert binding.Plan([27, 9], binding.LATENCY_OPTIMAL).kernel_supported(binding.KERNEL_FUSED)     # generic line-group kernel
+    odd = binding.Plan([243, 3], binding.LATENCY_OPTIMAL)               # a side above 81 off a ring: no fused latency kernel
     assert not odd.kernel_supported(binding.KERNEL_FUSED)
     assert odd.scratch_bytes(64) == odd.scratch_bytes(64, binding.KERNEL_STEP) > 0
     with pytest.raises(binding.TrivanceError):

@@ -25,8 +25,9 @@ def _built():
     binding.lib()
 
 
-FUSED_LAT = [(3,), (9,), (27,), (81,), (243,), (729,), (3, 3), (9, 9), (3, 3, 3), (3, 3, 3, 3), (9, 9, 9)]
-ANY = FUSED_LAT + [(3, 9), (27, 3), (3, 3, 9), (27, 27)]
+FUSED_LAT = [(3,), (9,), (27,), (81,), (243,), (729,), (3, 3), (9, 9), (3, 3, 3), (3, 3, 3, 3), (9, 9, 9),
+             (3, 9), (27, 3), (3, 3, 9), (27, 27), (9, 81), (81, 9), (3, 81), (9, 3, 27), (3, 27, 9)]   # the last ones: line-group kernel
+ANY = FUSED_LAT + [(243, 3)]
 
 
 @pytest.mark.parametrize("dims", ANY)
@@ -120,7 +121,7 @@ def test_sharded_windows_equal_the_unsharded_run(dims, variant):
 
 def test_default_entry_point_and_plan_owned_scratch():
     """trv_allreduce (in place, AUTO) incl. the case where the plan has to allocate scratch itself."""
-    for dims, variant in [((27,), LAT), ((27, 3), LAT), ((81,), BW)]:
+    for dims, variant in [((27,), LAT), ((243, 3), LAT), ((81,), BW)]:
         plan = binding.Plan(dims, variant)
         n = plan.n
         x = synth.rank_matrix("normal", 51, n, 2048)
