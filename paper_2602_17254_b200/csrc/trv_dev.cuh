@@ -59,6 +59,14 @@ inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     g_launches.fetch_add(1, std::memory_order_relaxed);
 }
 
+// Kernels that need more than 48 KB of dynamic shared memory must opt in; the attribute belongs
+// to the current device's copy of the function, so it is set (a cheap host-side call) at every
+// launch rather than cached per process.
+template <typename K>
+inline bool allow_big_smem(K kernel, int bytes) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+
 // (a + b) + c, one rounding per add, never contracted or reassociated.
 __device__ __forceinline__ float add3(float a, float b, float c) { return __fadd_rn(__fadd_rn(a, b), c); }
 __device__ __forceinline__ uint32_t add3(uint32_t a, uint32_t b, uint32_t c) { return (a + b) + c; }

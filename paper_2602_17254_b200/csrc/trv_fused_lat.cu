@@ -205,8 +205,7 @@ static trv_status_t lat_fused_launch(const Call& c, const Addr& in, const Addr& 
             } else {
                 g_last_kernel = "lat_ring<729>";
                 auto kfn = k_lat_ring<T, 81, 1, Addr>;
-                static const cudaError_t once = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, 729 * 32 * 4);
-                (void)once;
+                if (!allow_big_smem(kfn, 729 * 32 * 4)) return TRV_ERR_CUDA;
                 launch_pdl(kfn, dim3((unsigned)tiles), dim3(288), 729 * 32 * 4, c.st, in, out, a);
             }
         }

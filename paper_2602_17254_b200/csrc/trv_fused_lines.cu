@@ -229,8 +229,7 @@ static trv_status_t launch_lines_cg(const Call& c, const Addr& in, const Addr& o
         }
     if (tiles == 0) return TRV_OK;
     auto kfn = k_lat_lines<T, CG, Addr>;
-    static const cudaError_t once = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, 729 * 32 * 4);
-    if (once != cudaSuccess) return TRV_ERR_CUDA;
+    if (!allow_big_smem(kfn, 729 * 32 * 4)) return TRV_ERR_CUDA;
     launch_pdl(kfn, dim3((unsigned)tiles, p.ndims, 1), dim3(32 * kLnSets), (size_t)p.n * 32 * CG * sizeof(T), c.st, in, out, a, prog);
     return TRV_OK;
 }

@@ -116,8 +116,7 @@ template <typename T, int V, typename Addr>
 static trv_status_t launch_t999_v(const Call& c, const Addr& in, const Addr& out, const LatArgs& a, long long tiles_x) {
     auto kfn = k_lat_t999<T, V, Addr>;
     constexpr size_t smem = 729 * 32 * sizeof(T);
-    static const cudaError_t once = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (once != cudaSuccess) return TRV_ERR_CUDA;
+    if (!allow_big_smem(kfn, (int)smem)) return TRV_ERR_CUDA;
     launch_pdl(kfn, dim3((unsigned)tiles_x, 3, 1), dim3(288 / V), smem, c.st, in, out, a);
     return TRV_OK;
 }
