@@ -28,7 +28,7 @@ typedef struct trv_plan_s *trv_plan_t;          /* opaque; owned by the library 
 typedef enum {
     TRV_OK = 0,
     TRV_ERR_INVALID_ARG = 1,        /* NULL pointer, bad enum, misaligned or aliasing buffers ... */
-    TRV_ERR_UNSUPPORTED = 2,        /* a side that is not a power of three, too many ranks, op != sum */
+    TRV_ERR_UNSUPPORTED = 2,        /* a side that is no power of three (other than a ring in the bandwidth form), too many ranks, op != sum */
     TRV_ERR_UNDEFINED_SCHEDULE = 3, /* the schedule does not exist for this n (Recursive Doubling, n != 2^q) */
     TRV_ERR_ALLOC = 4,
     TRV_ERR_CUDA = 5,               /* a CUDA runtime call failed; cudaGetLastError has the reason */
@@ -65,7 +65,20 @@ typedef enum { TRV_KERNEL_AUTO = 0, TRV_KERNEL_STEP = 1, TRV_KERNEL_FUSED = 2 } 
  * Host-only integer work; makes no CUDA call.  A plan is immutable: it may be used from
  * several threads and streams at once.
  * Errors: INVALID_ARG (NULL, ndims out of range, side < 2), UNSUPPORTED (side not a power
- * of three, more than TRV_MAX_RANKS ranks). */
+ * of three, more than TRV_MAX_RANKS ranks).
+ *
+ * Rings of any other size (Sec. 4.4): with ndims = 1 and the bandwidth-optimal variant, a side
+ * n >= 2 that is no power of three gives the schedule of ceil(log3 n) steps per phase: the
+ * regular distances 3^0 .. 3^(s-1), s = floor(log3 n), then one step at distance
+ * ceil((n - 3^s) / 2).  The paper fixes the steps, the distances, that no block is sent twice
+ * by a node in a phase and that a node sends at most m bytes per phase; which tree a block
+ * follows it leaves open.  This library's reading: the AllGather of a block runs the steps in
+ * reverse order; the nodes holding the block are kept in the order they got it; in a step
+ * every holder, in that order, offers it to its left peer (h - dist), then to its right peer
+ * (h + dist); a node that already holds it is skipped.  The Reduce-Scatter runs the same tree
+ * backwards, a receiver adding (from_left + own) + from_right and leaving out a side nothing
+ * comes from.  Such plans run through the STEP kernels only.  The latency-optimal variant is
+ * not defined for these sizes: UNSUPPORTED, as for tori with such a side. */
 trv_status_t trv_plan_create(const int32_t *dims, int32_t ndims, trv_variant_t variant, trv_plan_t *out);
 
 /* Same, for a comparator schedule (Sec. 2.4, Fig. 1).  TRV_ALGO_BRUCK: peers r + 3^k and
@@ -93,6 +106,9 @@ trv_status_t trv_plan_peers(trv_plan_t plan, int32_t c, int32_t row, int32_t *pe
 /* set: HOST array of n bytes; set[j] = 1 iff block j is part of the message sent to rank
  * `dst` in Reduce-Scatter step `step` of collective c (closed form Pi of Sec. 4.3: the
  * blocks that agree with dst modulo 3^(visits so far) in every dimension). */
+/* For a ring whose size is no power of three (Sec. 4.4) the two senders' sets differ:
+ * set[j] then has bit 0 set if dst receives a partial of block j from its left peer in that
+ * step and bit 1 if it receives one from its right peer. */
 trv_status_t trv_plan_send_set(trv_plan_t plan, int32_t c, int32_t step, int32_t dst, uint8_t *set);
 
 /* bounds: HOST array of n+1 global element indices: block j of collective c covers
@@ -200,8 +216,15 @@ trv_status_t trv_link_loads(trv_plan_t plan, size_t count, size_t elem_size, int
 /* bytes: HOST int64 [n].  Row < S (Reduce-Scatter or latency form): bytes of the message a
  * rank RECEIVES from each sender in that row, indexed by destination.  Row >= S (AllGather):
  * bytes of the message a rank SENDS to each of its peers, indexed by source.  Host-only. */
+/* UNSUPPORTED for a ring whose size is no power of three (its two messages differ): use the next call. */
 trv_status_t trv_plan_message_bytes(trv_plan_t plan, size_t count, size_t elem_size, int32_t c, int32_t row,
                                     int64_t *bytes);
+
+/* bytes: HOST array of n: bytes of the message every rank SENDS in that row to its peer number
+ * `side` (0: the first peer of trv_plan_peers -- Trivance: r - dist; 1: the second), always
+ * indexed by the sending rank; 0 where no message goes that way.  Every kind of plan.  Host-only. */
+trv_status_t trv_plan_message_bytes_side(trv_plan_t plan, size_t count, size_t elem_size, int32_t c, int32_t row,
+                                         int32_t side, int64_t *bytes);
 
 /* ---------------------------------------------------------------- cost model
  *

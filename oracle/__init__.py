@@ -7,5 +7,5 @@ imports it.
 from .oracle import (  # noqa: F401
     ALGO_BRUCK, ALGO_RECDOUB, ALGO_TRIVANCE, VARIANT_BANDWIDTH, VARIANT_LATENCY,
     OracleError, allreduce, block_bounds, bytes_sent, cost_model, block_propagation, build, link_loads,
-    naive_sum_f32, num_steps, peers, send_set, step_list,
+    gen_allreduce, gen_link_loads, gen_num_steps, gen_tree, naive_sum_f32, num_steps, peers, send_set, step_list,
 )

@@ -61,6 +61,17 @@ def _dims(dims):
     return a, a.ctypes.data_as(ctypes.c_void_p), ctypes.c_int(a.size)
 
 
+def _general_ring(dims, algo=ALGO_TRIVANCE):
+    """n if dims is a ring whose size is no power of three (Trivance, Sec. 4.4), else 0."""
+    a = np.atleast_1d(np.asarray(dims)).reshape(-1)
+    if algo != ALGO_TRIVANCE or a.size != 1 or a[0] < 2:
+        return 0
+    n = int(a[0])
+    while n % 3 == 0:
+        n //= 3
+    return int(a[0]) if n != 1 else 0
+
+
 def num_steps(dims, algo=ALGO_TRIVANCE):
     """(n, steps per phase) of the schedule on a torus with these dimensions."""
     _, p, nd = _dims(dims)
@@ -134,6 +145,10 @@ def allreduce(dims, variant, x, E=None, e0=0, max_steps=-1, counters=False):
     the whole vector).  Returns the [n][w] result, or (result, counters) with
     per-rank byte counters ``sent_rs``, ``sent_ag``, ``reduced``.
     """
+    if _general_ring(dims):
+        if variant != VARIANT_BANDWIDTH or max_steps >= 0:
+            raise OracleError(2)
+        return gen_allreduce(x, E=E, e0=e0, counters=counters)
     x = np.ascontiguousarray(x)
     if x.dtype not in _DTYPES or x.ndim != 2:
         raise TypeError("x must be a 2-D int32, float32 or float64 array")
@@ -157,6 +172,10 @@ def allreduce(dims, variant, x, E=None, e0=0, max_steps=-1, counters=False):
 
 def link_loads(dims, variant, E, elem_size=4, algo=ALGO_TRIVANCE):
     """Per-step link loads: dict with msgs/bytes [T][n][D][2] and max_msgs/max_bytes [T]."""
+    if _general_ring(dims, algo):
+        if variant != VARIANT_BANDWIDTH:
+            raise OracleError(2)
+        return gen_link_loads(_general_ring(dims, algo), E, elem_size)
     a, p, nd = _dims(dims)
     n, s = num_steps(dims, algo)
     T = 2 * s if variant == VARIANT_BANDWIDTH else s
@@ -174,6 +193,10 @@ def link_loads(dims, variant, E, elem_size=4, algo=ALGO_TRIVANCE):
 
 def bytes_sent(dims, variant, E, elem_size=4, algo=ALGO_TRIVANCE):
     """[n] int64: bytes every node sends over the whole AllReduce."""
+    if _general_ring(dims, algo):
+        if variant != VARIANT_BANDWIDTH:
+            raise OracleError(2)
+        return gen_link_loads(_general_ring(dims, algo), E, elem_size)["sent"]
     _, p, nd = _dims(dims)
     n, _ = num_steps(dims, algo)
     out = np.zeros(n, np.int64)
@@ -186,7 +209,7 @@ def cost_model(dims, variant, E, elem_size, alpha, beta, algo=ALGO_TRIVANCE):
     """Sec. 2.1: C = steps * alpha + sum_k beta * m_k * c_k, with m_k * c_k = bytes on the most loaded
     link of step k; plus the optimality factors of Tables 1 and 2 (lambda, delta, theta)."""
     ll = link_loads(dims, variant, E, elem_size, algo)
-    n, _ = num_steps(dims, algo)
+    n = _general_ring(dims, algo) or num_steps(dims, algo)[0]
     T = ll["max_bytes"].size
     tx = int(ll["max_bytes"].sum())
     sent = int(bytes_sent(dims, variant, E, elem_size, algo).max())
@@ -195,3 +218,56 @@ def cost_model(dims, variant, E, elem_size, alpha, beta, algo=ALGO_TRIVANCE):
     return {"steps": T, "bytes_sent_per_node": sent, "tx_bytes": tx, "latency_term": T * alpha, "tx_term": beta * tx,
             "total": T * alpha + beta * tx, "lambda": T / (np.log(n) / np.log(3.0)), "delta": sent / (2.0 * m),
             "theta": tx / (m / D)}
+
+
+# ------------------------------------------------------------------ rings of any size (Sec. 4.4)
+
+def gen_num_steps(n):
+    """(S, [dist_0 .. dist_{S-1}]) of the ring of n nodes: regular distances, then the final one."""
+    s = ctypes.c_int()
+    d = np.zeros(32, np.int32)
+    _check(_load().orc_gen_num_steps(ctypes.c_int(n), ctypes.byref(s), d.ctypes.data_as(ctypes.c_void_p)))
+    return s.value, [int(v) for v in d[:s.value]]
+
+
+def gen_tree(n):
+    """(par, stp), both [n][n]: par[b][v] = node v gets block b from (-1 for v = b), stp[b][v] = in which step."""
+    par = np.zeros((n, n), np.int32)
+    stp = np.zeros((n, n), np.int32)
+    _check(_load().orc_gen_tree(ctypes.c_int(n), par.ctypes.data_as(ctypes.c_void_p), stp.ctypes.data_as(ctypes.c_void_p)))
+    return par, stp
+
+
+def gen_allreduce(x, E=None, e0=0, counters=False):
+    """Bandwidth-optimal Trivance AllReduce on a ring of x.shape[0] nodes (any size >= 2); as ``allreduce``."""
+    x = np.ascontiguousarray(x)
+    if x.dtype not in _DTYPES or x.ndim != 2:
+        raise TypeError("x must be a 2-D int32, float32 or float64 array")
+    n, w = x.shape
+    if E is None:
+        E = w
+    out = np.empty_like(x)
+    ctr = [np.zeros(n, np.int64) for _ in range(3)] if counters else [None] * 3
+    ptr = [c.ctypes.data_as(ctypes.c_void_p) if c is not None else None for c in ctr]
+    _check(_load().orc_gen_allreduce(ctypes.c_int(n), ctypes.c_int(_DTYPES[x.dtype]), ctypes.c_int64(E), ctypes.c_int64(e0),
+                                     ctypes.c_int64(e0 + w), x.ctypes.data_as(ctypes.c_void_p),
+                                     out.ctypes.data_as(ctypes.c_void_p), *ptr))
+    if counters:
+        return out, {"sent_rs": ctr[0], "sent_ag": ctr[1], "reduced": ctr[2]}
+    return out
+
+
+def gen_link_loads(n, E, elem_size=4):
+    """Link loads of that schedule: msgs/bytes [2S][n][1][2], max_msgs/max_bytes [2S], sent [n]."""
+    S, _ = gen_num_steps(n)
+    T = 2 * S
+    msgs = np.zeros((T, n, 1, 2), np.int32)
+    byts = np.zeros((T, n, 1, 2), np.int64)
+    mm = np.zeros(T, np.int32)
+    mb = np.zeros(T, np.int64)
+    sent = np.zeros(n, np.int64)
+    _check(_load().orc_gen_link_loads(ctypes.c_int(n), ctypes.c_int64(E), ctypes.c_int64(elem_size),
+                                      msgs.ctypes.data_as(ctypes.c_void_p), byts.ctypes.data_as(ctypes.c_void_p),
+                                      mm.ctypes.data_as(ctypes.c_void_p), mb.ctypes.data_as(ctypes.c_void_p),
+                                      sent.ctypes.data_as(ctypes.c_void_p)))
+    return {"msgs": msgs, "bytes": byts, "max_msgs": mm, "max_bytes": mb, "sent": sent}

@@ -548,3 +548,213 @@ done:
     free(lm); free(lb); free(set); free(have); free(snap); free(blen);
     return rc;
 }
+
+/* ------------------------------------------------------------------ rings of any size (Sec. 4.4) */
+
+/*
+ * Bandwidth-optimal Trivance on a ring whose size n is NOT a power of three.
+ *
+ * What the paper fixes (Sec. 4.4): the first s' = floor(log3 n) steps are the regular ones
+ * (distances 3^0 .. 3^(s'-1)); one final step follows in which every node talks to both
+ * nodes at distance d = ceil((n - 3^s') / 2); ceil(log3 n) steps in all; blocks travel as in
+ * Algorithm 1 with every block forwarded at most once per phase, so a node sends at most m
+ * bytes per phase; the final step's congestion is d on every link; for n = 7 a node sends two
+ * blocks per direction in the first step and one block, at distance two, in the final one.
+ *
+ * Reading where the paper is silent (PARITY UNPINNED by the paper; also in the design notes):
+ * which tree a block follows.  The AllGather of block b runs the steps in reverse order (the
+ * distance-d step first).  The nodes that hold the block are kept in the order they got it;
+ * in a step every holder, in that order, offers the block first to its left peer (h - dist)
+ * and then to its right peer (h + dist); a node that holds the block already -- one that got
+ * it earlier in the same step included -- is skipped.  The Reduce-Scatter runs the same tree
+ * backwards: in step t every node that received block b in AllGather step t sends its
+ * partial of block b to the node it got the block from, and a receiver adds
+ * (from_left + own) + from_right, leaving out a side nothing came from.
+ * For n a power of three this rule gives the regular schedule (no node is ever skipped).
+ */
+static int gen_steps(int n, int *dist) {
+    int p = 1, s = 0;
+    while ((long long)p * 3 <= n) { p *= 3; dist[s++] = p / 3; }
+    if (p != n) dist[s++] = (n - p + 1) / 2;
+    return s;
+}
+
+/* par[b*n+v] = node v got block b from (-1 for v = b); stp[b*n+v] = the step it got it in */
+static int gen_build(int n, int S, const int *dist, int32_t *par, int32_t *stp) {
+    int *list = (int *)malloc(sizeof(int) * (size_t)n);
+    uint8_t *have = (uint8_t *)malloc((size_t)n);
+    int rc = ORC_OK;
+    if (!list || !have) { free(list); free(have); return ORC_NOMEM; }
+    for (int b = 0; b < n && rc == ORC_OK; ++b) {
+        int len = 1;
+        memset(have, 0, (size_t)n);
+        list[0] = b; have[b] = 1; par[(size_t)b * n + b] = -1; stp[(size_t)b * n + b] = -1;
+        for (int t = S - 1; t >= 0; --t) {
+            int len0 = len;
+            for (int i = 0; i < len0; ++i) {
+                int h = list[i];
+                for (int side = 0; side < 2; ++side) {
+                    int v = ((h + (side ? dist[t] : -dist[t])) % n + n) % n;
+                    if (have[v]) continue;
+                    have[v] = 1; par[(size_t)b * n + v] = h; stp[(size_t)b * n + v] = t; list[len++] = v;
+                }
+            }
+        }
+        if (len != n) rc = ORC_INTERNAL;
+    }
+    free(list); free(have);
+    return rc;
+}
+
+int orc_gen_num_steps(int n, int *S_out, int32_t *dist_out) {
+    if (n < 2 || n > 4096) return ORC_BAD_ARG;
+    int dist[32];
+    int S = gen_steps(n, dist);
+    if (S_out) *S_out = S;
+    if (dist_out) for (int t = 0; t < S; ++t) dist_out[t] = dist[t];
+    return ORC_OK;
+}
+
+int orc_gen_tree(int n, int32_t *par, int32_t *stp) {
+    if (n < 2 || n > 4096 || !par || !stp) return ORC_BAD_ARG;
+    int dist[32];
+    int S = gen_steps(n, dist);
+    return gen_build(n, S, dist, par, stp);
+}
+
+#define DEFINE_GEN(T, SUFFIX, ADD)                                                                         \
+static int gen_allreduce_##SUFFIX(int n, int S, const int *dist, const int32_t *par, const int32_t *stp,   \
+                                  int64_t E, int64_t e0, int64_t e1, const T *in, T *out,                  \
+                                  orc_counters *ctr) {                                                     \
+    int64_t w = e1 - e0;                                                                                   \
+    if (w <= 0) return ORC_OK;                                                                             \
+    int64_t *bs = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n + 1));                                    \
+    T *partial = (T *)malloc(sizeof(T) * (size_t)n * (size_t)w);                                           \
+    T *msg = (T *)malloc(sizeof(T) * (size_t)n * (size_t)w);     /* what every node puts on the wire */     \
+    if (!bs || !partial || !msg) { free(bs); free(partial); free(msg); return ORC_NOMEM; }                 \
+    for (int j = 0; j <= n; ++j) bs[j] = clampi(block_bound(0, E, n, j), e0, e1) - e0;                     \
+    memcpy(partial, in, sizeof(T) * (size_t)n * (size_t)w);                                                \
+    /* ---- Reduce-Scatter: the tree of every block, leaves first */                                      \
+    for (int t = 0; t < S; ++t) {                                                                          \
+        memcpy(msg, partial, sizeof(T) * (size_t)n * (size_t)w);                                           \
+        for (int b = 0; b < n; ++b) {                                                                      \
+            int64_t bl = bs[b + 1] - bs[b];                                                                \
+            for (int p = 0; p < n; ++p) {                                                                  \
+                int ql = ((p - dist[t]) % n + n) % n, qr = (p + dist[t]) % n;                              \
+                int hl = (stp[(size_t)b * n + ql] == t && par[(size_t)b * n + ql] == p);                   \
+                int hr = (qr != ql && stp[(size_t)b * n + qr] == t && par[(size_t)b * n + qr] == p);       \
+                T *own = partial + (size_t)p * w + bs[b];                                                  \
+                const T *ml = msg + (size_t)ql * w + bs[b], *mr = msg + (size_t)qr * w + bs[b];            \
+                if (!hl && !hr) continue;                                                                  \
+                for (int64_t e = 0; e < bl; ++e) {                                                         \
+                    T acc = own[e];                                                                        \
+                    if (hl) acc = ADD(ml[e], acc);                                                         \
+                    if (hr) acc = ADD(acc, mr[e]);                                                         \
+                    own[e] = acc;                                                                          \
+                }                                                                                          \
+                if (ctr && ctr->sent_rs) {                                                                 \
+                    if (hl) ctr->sent_rs[ql] += (int64_t)sizeof(T) * bl;                                   \
+                    if (hr) ctr->sent_rs[qr] += (int64_t)sizeof(T) * bl;                                   \
+                }                                                                                          \
+                if (ctr && ctr->reduced) ctr->reduced[p] += (int64_t)sizeof(T) * bl * (1 + hl + hr);       \
+            }                                                                                              \
+        }                                                                                                  \
+    }                                                                                                      \
+    /* ---- AllGather: the same trees, root first */                                                      \
+    for (int t = S - 1; t >= 0; --t) {                                                                     \
+        memcpy(msg, partial, sizeof(T) * (size_t)n * (size_t)w);                                           \
+        for (int b = 0; b < n; ++b)                                                                        \
+            for (int v = 0; v < n; ++v) if (stp[(size_t)b * n + v] == t) {                                 \
+                int q = par[(size_t)b * n + v]; int64_t bl = bs[b + 1] - bs[b];                            \
+                memcpy(partial + (size_t)v * w + bs[b], msg + (size_t)q * w + bs[b], sizeof(T) * (size_t)bl);\
+                if (ctr && ctr->sent_ag) ctr->sent_ag[q] += (int64_t)sizeof(T) * bl;                       \
+            }                                                                                              \
+    }                                                                                                      \
+    memcpy(out, partial, sizeof(T) * (size_t)n * (size_t)w);                                               \
+    free(bs); free(partial); free(msg);                                                                    \
+    return ORC_OK;                                                                                         \
+}
+DEFINE_GEN(uint32_t, i32, ADD_WRAP)
+DEFINE_GEN(float, f32, ADD_FP)
+DEFINE_GEN(double, f64, ADD_FP)
+
+/* AllReduce (bandwidth-optimal form) on a ring of any size n >= 2; arguments as orc_allreduce. */
+int orc_gen_allreduce(int n, int dtype, int64_t E, int64_t e0, int64_t e1, const void *in, void *out,
+                      int64_t *sent_rs, int64_t *sent_ag, int64_t *reduced) {
+    if (n < 2 || n > 4096 || E < 0 || e0 < 0 || e1 < e0 || e1 > E || !in || !out) return ORC_BAD_ARG;
+    if (dtype != ORC_I32 && dtype != ORC_F32 && dtype != ORC_F64) return ORC_BAD_ARG;
+    int dist[32];
+    int S = gen_steps(n, dist), rc;
+    int32_t *par = (int32_t *)malloc(sizeof(int32_t) * (size_t)n * n), *stp = (int32_t *)malloc(sizeof(int32_t) * (size_t)n * n);
+    orc_counters ctr = { sent_rs, sent_ag, reduced };
+    if (!par || !stp) { free(par); free(stp); return ORC_NOMEM; }
+    rc = gen_build(n, S, dist, par, stp);
+    if (rc == ORC_OK) {
+        if (dtype == ORC_I32) rc = gen_allreduce_i32(n, S, dist, par, stp, E, e0, e1, (const uint32_t *)in, (uint32_t *)out, &ctr);
+        else if (dtype == ORC_F32) rc = gen_allreduce_f32(n, S, dist, par, stp, E, e0, e1, (const float *)in, (float *)out, &ctr);
+        else rc = gen_allreduce_f64(n, S, dist, par, stp, E, e0, e1, (const double *)in, (double *)out, &ctr);
+    }
+    free(par); free(stp);
+    return rc;
+}
+
+/*
+ * Link loads of the same schedule (rows: S Reduce-Scatter steps, then the S AllGather steps in
+ * reverse order; arrays [2S][n][1][2] as in orc_link_loads).  All blocks a node sends to one
+ * peer in one step form ONE message; it walks dist links in its direction of travel.
+ * sent (optional, [n]): bytes every node sends over both phases.
+ */
+int orc_gen_link_loads(int n, int64_t E, int64_t elem_size, int32_t *msgs, int64_t *bytes,
+                       int32_t *max_msgs, int64_t *max_bytes, int64_t *sent) {
+    if (n < 2 || n > 4096 || E < 0 || elem_size < 1) return ORC_BAD_ARG;
+    int dist[32];
+    int S = gen_steps(n, dist), T = 2 * S, rc;
+    size_t links = (size_t)n * 2;
+    int32_t *par = (int32_t *)malloc(sizeof(int32_t) * (size_t)n * n), *stp = (int32_t *)malloc(sizeof(int32_t) * (size_t)n * n);
+    int32_t *lm = (int32_t *)calloc((size_t)T * links, sizeof(int32_t));
+    int64_t *lb = (int64_t *)calloc((size_t)T * links, sizeof(int64_t));
+    int64_t *mb = (int64_t *)malloc(sizeof(int64_t) * links);       /* [source][side]: bytes of its message */
+    int32_t *mc = (int32_t *)malloc(sizeof(int32_t) * links);       /* blocks in it */
+    if (!par || !stp || !lm || !lb || !mb || !mc) { rc = ORC_NOMEM; goto done; }
+    rc = gen_build(n, S, dist, par, stp);
+    if (rc) goto done;
+    if (sent) memset(sent, 0, sizeof(int64_t) * (size_t)n);
+    for (int row = 0; row < T; ++row) {
+        int t = row < S ? row : T - 1 - row;
+        memset(mb, 0, sizeof(int64_t) * links); memset(mc, 0, sizeof(int32_t) * links);
+        for (int b = 0; b < n; ++b)
+            for (int v = 0; v < n; ++v) if (stp[(size_t)b * n + v] == t) {
+                int q = par[(size_t)b * n + v];
+                /* v is its parent's left peer (tried first, so also when both peers coincide) or right peer */
+                int left_child = (v == ((q - dist[t]) % n + n) % n);
+                int src = row < S ? v : q;
+                int side = row < S ? left_child : !left_child;      /* 0: travels towards -, 1: towards + */
+                mb[(size_t)src * 2 + side] += (block_bound(0, E, n, b + 1) - block_bound(0, E, n, b)) * elem_size;
+                mc[(size_t)src * 2 + side] += 1;
+            }
+        for (int src = 0; src < n; ++src)
+            for (int side = 0; side < 2; ++side) if (mc[(size_t)src * 2 + side]) {
+                int cur = src;
+                if (sent) sent[src] += mb[(size_t)src * 2 + side];
+                for (int h = 0; h < dist[t]; ++h) {
+                    size_t li = ((size_t)row * n + cur) * 2 + (side ? 0 : 1);
+                    lm[li] += 1; lb[li] += mb[(size_t)src * 2 + side];
+                    cur = ((cur + (side ? 1 : -1)) % n + n) % n;
+                }
+            }
+    }
+    for (int row = 0; row < T; ++row) {
+        int32_t mm = 0; int64_t mx = 0;
+        for (size_t l = 0; l < links; ++l) {
+            if (lm[(size_t)row * links + l] > mm) mm = lm[(size_t)row * links + l];
+            if (lb[(size_t)row * links + l] > mx) mx = lb[(size_t)row * links + l];
+        }
+        if (max_msgs) max_msgs[row] = mm;
+        if (max_bytes) max_bytes[row] = mx;
+    }
+    if (msgs) memcpy(msgs, lm, sizeof(int32_t) * (size_t)T * links);
+    if (bytes) memcpy(bytes, lb, sizeof(int64_t) * (size_t)T * links);
+done:
+    free(par); free(stp); free(lm); free(lb); free(mb); free(mc);
+    return rc;
+}

@@ -26,7 +26,7 @@ SYMBOLS = [
     "trv_plan_create", "trv_plan_create_algo", "trv_plan_destroy", "trv_plan_info", "trv_plan_step",
     "trv_plan_peers", "trv_plan_send_set", "trv_plan_block_bounds", "trv_allreduce", "trv_scratch_bytes",
     "trv_kernel_supported", "trv_allreduce_ex", "trv_allreduce_host", "trv_host_workspace_bytes",
-    "trv_link_loads", "trv_plan_message_bytes", "trv_strerror", "trv_launch_count", "trv_last_kernel_name",
+    "trv_link_loads", "trv_plan_message_bytes", "trv_plan_message_bytes_side", "trv_strerror", "trv_launch_count", "trv_last_kernel_name",
     "trv_allreduce_noalloc", "trv_noalloc_max_scratch_bytes", "trv_cost_model",
 ]
 
@@ -64,6 +64,7 @@ def lib():
         L.trv_plan_send_set.argtypes = [vp, i32, i32, i32, vp]
         L.trv_plan_block_bounds.argtypes = [vp, sz, i32, vp]
         L.trv_plan_message_bytes.argtypes = [vp, sz, sz, i32, i32, vp]
+        L.trv_plan_message_bytes_side.argtypes = [vp, sz, sz, i32, i32, i32, vp]
         L.trv_allreduce.argtypes = [vp, vp, sz, ctypes.c_int, ctypes.c_int, vp]
         L.trv_scratch_bytes.argtypes = [vp, sz, ctypes.c_int, i32, ctypes.POINTER(sz)]
         L.trv_kernel_supported.argtypes = [vp, ctypes.c_int]
@@ -163,6 +164,12 @@ class Plan:
         _check(lib().trv_plan_send_set(self._h, c, step, dst, _np_ptr(out)), "trv_plan_send_set")
         return out.astype(bool)
 
+    def send_mask(self, c, step, dst):
+        """Raw bytes of trv_plan_send_set (rings of other sizes: bit 0 = from the left peer, bit 1 = from the right)."""
+        out = np.zeros(self.n, np.uint8)
+        _check(lib().trv_plan_send_set(self._h, c, step, dst, _np_ptr(out)), "trv_plan_send_set")
+        return out
+
     def block_bounds(self, count, c):
         out = np.zeros(self.n + 1, np.int64)
         _check(lib().trv_plan_block_bounds(self._h, count, c, _np_ptr(out)), "trv_plan_block_bounds")
@@ -171,6 +178,12 @@ class Plan:
     def message_bytes(self, count, elem_size, c, row):
         out = np.zeros(self.n, np.int64)
         _check(lib().trv_plan_message_bytes(self._h, count, elem_size, c, row, _np_ptr(out)), "trv_plan_message_bytes")
+        return out
+
+    def message_bytes_side(self, count, elem_size, c, row, side):
+        out = np.zeros(self.n, np.int64)
+        _check(lib().trv_plan_message_bytes_side(self._h, count, elem_size, c, row, side, _np_ptr(out)),
+               "trv_plan_message_bytes_side")
         return out
 
     def kernel_supported(self, kernel):

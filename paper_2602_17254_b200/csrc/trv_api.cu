@@ -11,6 +11,7 @@ std::atomic<uint64_t> g_launches{0};
 thread_local const char* g_last_kernel = "none";
 
 static bool fused_supported(const Plan& p) {
+    if (p.general) return false;
     return p.variant == TRV_LATENCY_OPTIMAL ? fused_latency_supported(p) : fused_bandwidth_supported(p);
 }
 
@@ -52,6 +53,7 @@ static trv_status_t dispatch(Call& c, trv_kernel_t kernel) {
     } else if (kernel == TRV_KERNEL_AUTO) {
         fused = fused_supported(p);
     }
+    if (p.general) return run_step_general(c);
     if (p.variant == TRV_LATENCY_OPTIMAL) return fused ? run_fused_latency(c) : run_step_latency(c);
     return fused ? run_fused_bandwidth(c) : run_step_bandwidth(c);
 }
@@ -116,7 +118,8 @@ trv_status_t trv_plan_send_set(trv_plan_t plan, int32_t c, int32_t step, int32_t
     if (!plan || !set) return TRV_ERR_INVALID_ARG;
     const Plan& p = plan->plan;
     if (c < 0 || c >= p.ndims || step < 0 || step >= p.S || dst < 0 || dst >= p.n) return TRV_ERR_INVALID_ARG;
-    for (int j = 0; j < p.n; ++j) set[j] = in_send_set(p, c, step, dst, j) ? 1 : 0;
+    for (int j = 0; j < p.n; ++j)
+        set[j] = p.general ? (uint8_t)general_recv_mask(p, step, dst, j) : (in_send_set(p, c, step, dst, j) ? 1 : 0);
     return TRV_OK;
 }
 
@@ -134,7 +137,17 @@ trv_status_t trv_plan_message_bytes(trv_plan_t plan, size_t count, size_t elem_s
     if (!plan || !bytes || elem_size == 0) return TRV_ERR_INVALID_ARG;
     const Plan& p = plan->plan;
     if (c < 0 || c >= p.ndims || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
+    if (p.general) return TRV_ERR_UNSUPPORTED;
     message_bytes(p, (int64_t)count, (int64_t)elem_size, c, row, bytes);
+    return TRV_OK;
+}
+
+trv_status_t trv_plan_message_bytes_side(trv_plan_t plan, size_t count, size_t elem_size, int32_t c, int32_t row,
+                                         int32_t side, int64_t* bytes) {
+    if (!plan || !bytes || elem_size == 0 || side < 0 || side > 1) return TRV_ERR_INVALID_ARG;
+    const Plan& p = plan->plan;
+    if (c < 0 || c >= p.ndims || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
+    message_bytes_side(p, (int64_t)count, (int64_t)elem_size, c, row, side, bytes);
     return TRV_OK;
 }
 
@@ -257,18 +270,13 @@ trv_status_t trv_cost_model(trv_plan_t plan, size_t count, size_t elem_size, dou
     std::vector<int64_t> max_bytes((size_t)T), mb((size_t)n), sent((size_t)n, 0);
     trv_status_t st = run_link_loads(p, count, elem_size, nullptr, nullptr, nullptr, max_bytes.data());
     if (st != TRV_OK) return st;
-    // bytes every node sends: Reduce-Scatter / latency rows are indexed by destination, AllGather rows by source
+    // bytes every node sends: both of its messages in every row of every collective
     for (int c = 0; c < D; ++c)
-        for (int row = 0; row < T; ++row) {
-            message_bytes(p, (int64_t)count, (int64_t)elem_size, c, row, mb.data());
-            const Step& s = p.steps[c][p.step_of_row(row)];
-            const bool by_source = p.variant == TRV_BANDWIDTH_OPTIMAL && row >= p.S;
-            for (int r = 0; r < n; ++r) {
-                int peer[2], dir[2], hops[2];
-                const int np = send_peers(p, r, s.dim, s.dist, peer, dir, hops);
-                for (int i = 0; i < np; ++i) sent[r] += by_source ? mb[r] : mb[peer[i]];
+        for (int row = 0; row < T; ++row)
+            for (int side = 0; side < 2; ++side) {
+                message_bytes_side(p, (int64_t)count, (int64_t)elem_size, c, row, side, mb.data());
+                for (int r = 0; r < n; ++r) sent[r] += mb[r];
             }
-        }
     int64_t tx = 0, smax = 0;
     for (int row = 0; row < T; ++row) tx += max_bytes[row];
     for (int r = 0; r < n; ++r) smax = std::max(smax, sent[r]);

@@ -148,6 +148,7 @@ __device__ __forceinline__ V add3v(const V& a, const V& b, const V& c) {
 // step-family launchers (trv_step.cu)
 trv_status_t run_step_latency(const Call& c);
 trv_status_t run_step_bandwidth(const Call& c);
+trv_status_t run_step_general(const Call& c);
 size_t step_scratch_bytes(const Plan& p, size_t count, bool in_place);
 
 // fused-family launchers (trv_fused_lat.cu / trv_fused_bw.cu)

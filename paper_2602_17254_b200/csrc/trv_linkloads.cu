@@ -20,10 +20,10 @@ struct MsgClass {
     int delta;      // destination = source + delta (ring positions, wraps)
     int filter;     // 0: every source sends; 1: sources with (pos & bit) == 0; 2: (pos & bit) != 0
     int bit;
+    int plane;      // which of the two per-source weight arrays: bytes sent to the first / second peer
 };
 struct RowSlice {
     int dim, stride, size;      // the ring's dimension
-    int by_source;              // weights indexed by source (AllGather rows) or by destination
     int nclass;
     MsgClass cls[2];
 };
@@ -51,10 +51,11 @@ __global__ void __launch_bounds__(32) k_link_tally(const RowSlice* __restrict__ 
     // ring number -> rank of its position 0
     const int q = blockIdx.x;
     const int base = (q % rs.stride) + (q / rs.stride) * rs.stride * a;
-    const long long* w = mbytes + ((size_t)row * D + c) * n;
+    const long long* w0 = mbytes + ((size_t)row * D + c) * 2 * n;
 
     for (int k = 0; k < rs.nclass; ++k) {
         const MsgClass mc = rs.cls[k];
+        const long long* w = w0 + (size_t)mc.plane * n;
         long long carry = 0;
         int ccarry = 0;
         for (int s0 = 0; s0 < a; s0 += 32) {
@@ -64,10 +65,7 @@ __global__ void __launch_bounds__(32) k_link_tally(const RowSlice* __restrict__ 
             if (s < a) {
                 const bool sends = mc.filter == 0 || (mc.filter == 1 ? (s & mc.bit) == 0 : (s & mc.bit) != 0);
                 if (sends) {
-                    int dpos = s + mc.delta;
-                    dpos %= a;
-                    if (dpos < 0) dpos += a;
-                    wt = w[base + (rs.by_source ? s : dpos) * rs.stride];
+                    wt = w[base + s * rs.stride];
                     cnt = 1;
                 }
             }
@@ -135,32 +133,42 @@ trv_status_t run_link_loads(const Plan& p, size_t count, size_t elem_size, int32
     const int n = p.n, D = p.ndims, T = p.rows();
     const size_t links = (size_t)n * D * 2;
     std::vector<RowSlice> desc((size_t)T * D);
-    std::vector<long long> mb((size_t)T * D * n);
+    std::vector<long long> mb((size_t)T * D * 2 * n);   // [row][slice][peer number][source rank]
     int max_rings = 1;
     for (int row = 0; row < T; ++row) {
         for (int c = 0; c < D; ++c) {
             const Step& st = p.steps[c][p.step_of_row(row)];
             RowSlice& rs = desc[(size_t)row * D + c];
             rs.dim = st.dim; rs.stride = p.stride[st.dim]; rs.size = p.dims[st.dim];
-            rs.by_source = (p.variant == TRV_BANDWIDTH_OPTIMAL && row >= p.S) ? 1 : 0;
             if (rs.size > kMaxRing) return TRV_ERR_UNSUPPORTED;
             if (n / rs.size > max_rings) max_rings = n / rs.size;
             const int d = st.dist;
-            if (p.algo == TRV_ALGO_TRIVANCE) {
+            if (p.general) {
+                // a direction in which no block travels in this step carries no message at all
+                const int t = p.step_of_row(row);
+                bool any[2] = {false, false};
+                for (int o = 1; o < n; ++o)
+                    if (p.gstep[o] == t) any[(row < p.S) == (p.gsgn[o] > 0) ? 1 : 0] = true;
+                rs.nclass = 0;
+                if (any[0]) rs.cls[rs.nclass++] = MsgClass{-1, d, -d, 0, 0, 0};
+                if (any[1]) rs.cls[rs.nclass++] = MsgClass{+1, d, +d, 0, 0, 1};
+            } else if (p.algo == TRV_ALGO_TRIVANCE) {
                 rs.nclass = 2;
-                rs.cls[0] = MsgClass{-1, d, -d, 0, 0};
-                rs.cls[1] = MsgClass{+1, d, +d, 0, 0};
+                rs.cls[0] = MsgClass{-1, d, -d, 0, 0, 0};
+                rs.cls[1] = MsgClass{+1, d, +d, 0, 0, 1};
             } else if (p.algo == TRV_ALGO_BRUCK) {
                 rs.nclass = 2;
-                rs.cls[0] = MsgClass{+1, d, d, 0, 0};
-                rs.cls[1] = MsgClass{+1, 2 * d, 2 * d, 0, 0};
+                rs.cls[0] = MsgClass{+1, d, d, 0, 0, 0};
+                rs.cls[1] = MsgClass{+1, 2 * d, 2 * d, 0, 0, 1};
             } else {
                 rs.nclass = 2;
-                rs.cls[0] = MsgClass{+1, d, +d, 1, d};
-                rs.cls[1] = MsgClass{-1, d, -d, 2, d};
+                rs.cls[0] = MsgClass{+1, d, +d, 1, d, 0};
+                rs.cls[1] = MsgClass{-1, d, -d, 2, d, 0};
             }
             static_assert(sizeof(long long) == sizeof(int64_t), "int64");
-            message_bytes(p, (int64_t)count, (int64_t)elem_size, c, row, (int64_t*)&mb[((size_t)row * D + c) * n]);
+            for (int side = 0; side < 2; ++side)
+                message_bytes_side(p, (int64_t)count, (int64_t)elem_size, c, row, side,
+                                   (int64_t*)&mb[(((size_t)row * D + c) * 2 + side) * n]);
         }
     }
 

@@ -17,6 +17,38 @@ static int exact_log(int a, int base) {
     return s;
 }
 
+// Sec. 4.4 with the reading stated in the header of the C interface: the AllGather of a block runs
+// the steps in reverse order (the extra distance first); holders are kept in the order they got
+// the block; in a step each holder, in that order, offers it to its left peer, then to its right
+// peer, and a node that holds it already is skipped.  Written in offsets from the block's owner.
+static void build_general_ring(Plan& p, int n) {
+    int pw = 1;
+    std::vector<Step> steps;
+    while ((long long)pw * 3 <= n) { steps.push_back(Step{0, pw}); pw *= 3; }
+    steps.push_back(Step{0, (n - pw + 1) / 2});
+    p.general = true;
+    p.S = (int)steps.size();
+    p.gstep.assign(n, -1);
+    p.gsgn.assign(n, 0);
+    std::vector<int> order(1, 0);
+    std::vector<char> held(n, 0);
+    held[0] = 1;
+    for (int t = p.S - 1; t >= 0; --t) {
+        const size_t cnt = order.size();
+        for (size_t i = 0; i < cnt; ++i)
+            for (int side = 0; side < 2; ++side) {
+                const int delta = side ? steps[t].dist : -steps[t].dist;
+                const int v = ((order[i] + delta) % n + n) % n;
+                if (held[v]) continue;
+                held[v] = 1;
+                p.gstep[v] = (int8_t)t;
+                p.gsgn[v] = (int8_t)(side ? -1 : +1);      // the child sends back the way the block came
+                order.push_back(v);
+            }
+    }
+    p.steps.assign(1, steps);
+}
+
 trv_status_t build_plan(const int32_t* dims, int32_t ndims, int variant, int algo, trv_plan_s** out) {
     if (!dims || !out || ndims < 1 || ndims > TRV_MAX_DIMS) return TRV_ERR_INVALID_ARG;
     if (variant != TRV_LATENCY_OPTIMAL && variant != TRV_BANDWIDTH_OPTIMAL) return TRV_ERR_INVALID_ARG;
@@ -30,6 +62,14 @@ trv_status_t build_plan(const int32_t* dims, int32_t ndims, int variant, int alg
     if (!holder) return TRV_ERR_ALLOC;
     Plan& p = holder->plan;
     p.algo = algo; p.variant = variant; p.ndims = ndims; p.base = base;
+    if (algo == TRV_ALGO_TRIVANCE && ndims == 1 && exact_log(dims[0], 3) < 0) {
+        // a ring of any other size: only the bandwidth-optimal form is defined (Sec. 4.4)
+        if (variant != TRV_BANDWIDTH_OPTIMAL || dims[0] > TRV_MAX_RANKS) { delete holder; return TRV_ERR_UNSUPPORTED; }
+        p.dims[0] = dims[0]; p.stride[0] = 1; p.n = dims[0];
+        build_general_ring(p, dims[0]);
+        *out = holder;
+        return TRV_OK;
+    }
     long long n = 1;
     for (int d = 0; d < ndims; ++d) {
         int s = exact_log(dims[d], base);
@@ -90,6 +130,47 @@ int send_peers(const Plan& p, int r, int dim, int dist, int peer[2], int dir[2],
             peer[1] = -1; dir[1] = 0; hops[1] = 0;
             return 1;
         }
+    }
+}
+
+int general_recv_mask(const Plan& p, int t, int dst, int j) {
+    const int n = p.n, dist = p.steps[0][t].dist;
+    const int o = ((dst - j) % n + n) % n;
+    const int ol = ((o - dist) % n + n) % n, orr = (o + dist) % n;
+    int mask = 0;
+    if (p.gstep[ol] == t && p.gsgn[ol] > 0) mask |= 1;
+    if (orr != ol && p.gstep[orr] == t && p.gsgn[orr] < 0) mask |= 2;
+    return mask;
+}
+
+void message_bytes_side(const Plan& p, int64_t E, int64_t elem_size, int c, int row, int side, int64_t* out) {
+    const int n = p.n;
+    if (p.general) {
+        // Reduce-Scatter row: the node at offset o sends block (node - o); AllGather row: the parent
+        // of the node at offset o, which sits at offset o + sgn * dist, sends it to that node.
+        const int t = p.step_of_row(row), dist = p.steps[0][t].dist;
+        const bool rs = row < p.S;
+        for (int r = 0; r < n; ++r) out[r] = 0;
+        for (int o = 1; o < n; ++o) {
+            if (p.gstep[o] != t) continue;
+            const int sends_right = rs ? (p.gsgn[o] > 0) : (p.gsgn[o] < 0);
+            if (sends_right != side) continue;
+            const int src_off = rs ? o : ((o + p.gsgn[o] * dist) % n + n) % n;
+            for (int r = 0; r < n; ++r) {
+                const int j = ((r - src_off) % n + n) % n;
+                out[r] += (block_lo(0, E, n, j + 1) - block_lo(0, E, n, j)) * elem_size;
+            }
+        }
+        return;
+    }
+    std::vector<int64_t> tmp((size_t)n);
+    message_bytes(p, E, elem_size, c, row, tmp.data());
+    const Step& st = p.steps[c][p.step_of_row(row)];
+    const bool by_source = p.variant == TRV_BANDWIDTH_OPTIMAL && row >= p.S;
+    for (int r = 0; r < n; ++r) {
+        int peer[2], dir[2], hops[2];
+        const int np = send_peers(p, r, st.dim, st.dist, peer, dir, hops);
+        out[r] = side < np ? (by_source ? tmp[r] : tmp[peer[side]]) : 0;
     }
 }
 

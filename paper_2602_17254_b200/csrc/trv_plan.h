@@ -26,6 +26,14 @@ struct Plan {
     // the message to p at step t iff j_d == p_d (mod mod[c][t][d]) for every d  (closed form Pi)
     std::vector<std::vector<std::vector<int>>> mod;
 
+    // Rings whose size is no power of three (Sec. 4.4), bandwidth-optimal form only.  The tree a
+    // block follows is the same for every block up to rotation, so it is stored once, by the
+    // OFFSET o = (node - block) mod n:  gstep[o] = Reduce-Scatter step in which the node at
+    // offset o sends its partial on (-1 for the owner, o = 0); gsgn[o] = +1 if it sends it to
+    // node + dist, -1 if to node - dist.
+    bool general = false;
+    std::vector<int8_t> gstep, gsgn;
+
     // plan-owned scratch for trv_allreduce (STEP family of the latency form), grown on demand
     void* scratch = nullptr;
     size_t scratch_bytes = 0;
@@ -53,7 +61,14 @@ bool in_send_set(const Plan& p, int c, int t, int dst, int j);
 // peers a rank sends to in step (dim, dist); returns how many; dir = +1 / -1, hops = links crossed
 int send_peers(const Plan& p, int r, int dim, int dist, int peer[2], int dir[2], int hops[2]);
 // message bytes of one row, indexed by destination (row < S) or by source (AllGather rows)
+// (not for general rings)
 void message_bytes(const Plan& p, int64_t E, int64_t elem_size, int c, int row, int64_t* out);
+// bytes of the message every rank SENDS to its peer number `side` (0: first peer -- Trivance: the
+// left one; 1: second peer) in one row; 0 where it sends none.  Every kind of plan.
+void message_bytes_side(const Plan& p, int64_t E, int64_t elem_size, int c, int row, int side, int64_t* out);
+// general rings: what `dst` receives for block j in Reduce-Scatter step t: bit 0 = a partial from
+// its left peer, bit 1 = one from its right peer
+int general_recv_mask(const Plan& p, int t, int dst, int j);
 
 }  // namespace trv
 
