@@ -11,7 +11,7 @@ std::atomic<uint64_t> g_launches{0};
 thread_local const char* g_last_kernel = "none";
 
 static bool fused_supported(const Plan& p) {
-    if (p.general) return false;
+    if (p.general) return fused_tree_supported(p);
     return p.variant == TRV_LATENCY_OPTIMAL ? fused_latency_supported(p) : fused_bandwidth_supported(p);
 }
 
@@ -53,7 +53,7 @@ static trv_status_t dispatch(Call& c, trv_kernel_t kernel) {
     } else if (kernel == TRV_KERNEL_AUTO) {
         fused = fused_supported(p);
     }
-    if (p.general) return run_step_general(c);
+    if (p.general) return fused ? run_fused_tree(c) : run_step_general(c);
     if (p.variant == TRV_LATENCY_OPTIMAL) return fused ? run_fused_latency(c) : run_step_latency(c);
     return fused ? run_fused_bandwidth(c) : run_step_bandwidth(c);
 }

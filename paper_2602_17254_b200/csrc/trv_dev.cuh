@@ -156,6 +156,9 @@ bool fused_latency_supported(const Plan& p);
 bool fused_bandwidth_supported(const Plan& p);
 trv_status_t run_fused_latency(const Call& c);
 trv_status_t run_fused_bandwidth(const Call& c);
+// rings of any other size (trv_fused_tree.cu)
+bool fused_tree_supported(const Plan& p);
+trv_status_t run_fused_tree(const Call& c);
 
 // link-load tally (trv_linkloads.cu)
 trv_status_t run_link_loads(const Plan& p, size_t count, size_t elem_size, int32_t* msgs, int64_t* bytes,

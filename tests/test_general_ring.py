@@ -211,7 +211,7 @@ def test_unsupported_forms():
             binding.Plan(dims, variant)
         assert e.value.status == binding.ERR_UNSUPPORTED
     plan = binding.Plan([10], binding.BANDWIDTH_OPTIMAL)
-    assert not plan.kernel_supported(binding.KERNEL_FUSED) and plan.kernel_supported(binding.KERNEL_STEP)
+    assert plan.kernel_supported(binding.KERNEL_FUSED) and plan.kernel_supported(binding.KERNEL_STEP)
     with pytest.raises(binding.TrivanceError) as e:
         plan.message_bytes(100, 4, 0, 0)
     assert e.value.status == binding.ERR_UNSUPPORTED

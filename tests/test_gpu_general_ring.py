@@ -26,9 +26,12 @@ def _built():
 @pytest.mark.parametrize("n", SIZES)
 def test_matches_oracle(n):
     count = 4099 if n <= 100 else 1531      # several blocks of ragged length, unaligned block starts
-    check_case((n,), BW, count, "normal", 21, AUTO)
+    check_case((n,), BW, count, "normal", 21, FUSED)
     check_case((n,), BW, count, "int32", 22, STEP, in_place=False)
+    check_case((n,), BW, count, "int32", 22, FUSED, in_place=False)
+    check_case((n,), BW, count, "normal", 21, STEP)
     check_scattered((n,), BW, count, "uniform", 23, AUTO)
+    check_scattered((n,), BW, count, "uniform", 23, STEP)
 
 
 @pytest.mark.parametrize("n", [7, 32, 100])
@@ -41,7 +44,17 @@ def test_short_vectors(n, count):
 
 @pytest.mark.parametrize("n", [10, 53])
 def test_larger_vector_spans_many_ctas(n):
-    check_case((n,), BW, 700001, "normal", 26, AUTO)
+    check_case((n,), BW, 700001, "normal", 26, STEP)
+    check_case((n,), BW, 700001, "normal", 26, FUSED)
+
+
+@pytest.mark.parametrize("n,count", [(4, 1 << 20), (10, (1 << 20) + 6), (100, (1 << 20) + 3)])
+def test_two_columns_per_thread_path(n, count):
+    """Long vectors take the kernel with two columns per thread; block boundaries fall inside some pairs."""
+    check_case((n,), BW, count, "normal", 32, FUSED)
+    assert binding.last_kernel_name() == "bw_tree<V=2>"
+    check_case((n,), BW, count, "int32", 33, FUSED, in_place=False)
+    check_scattered((n,), BW, count, "normal", 34, FUSED)
 
 
 @pytest.mark.parametrize("n", [7, 32, 244])
@@ -60,16 +73,17 @@ def test_largest_ring():
 
 def test_empty_and_kernel_choice():
     plan = binding.Plan((10,), BW)
-    assert plan.kernel_supported(STEP) and not plan.kernel_supported(FUSED)
+    assert plan.kernel_supported(STEP) and plan.kernel_supported(FUSED)
     x = torch.zeros((10, 64), dtype=torch.int32, device=DEV)
     ptrs = [x[r].data_ptr() for r in range(10)]
-    with pytest.raises(binding.TrivanceError) as e:
-        plan.allreduce_ex(ptrs, None, 64, binding.INT32, kernel=FUSED, stream=torch.cuda.current_stream().cuda_stream)
-    assert e.value.status == binding.ERR_UNSUPPORTED
     before = binding.launch_count()
     plan.allreduce_ex(ptrs, None, 0, binding.INT32, kernel=AUTO, stream=torch.cuda.current_stream().cuda_stream)
     assert binding.launch_count() == before
     plan.allreduce_ex(ptrs, None, 64, binding.INT32, kernel=AUTO, stream=torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert binding.last_kernel_name() == "bw_tree<V=1>" and binding.launch_count() - before == 1
+    before = binding.launch_count()
+    plan.allreduce_ex(ptrs, None, 64, binding.INT32, kernel=STEP, stream=torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
     assert binding.last_kernel_name() == "step_general"
     # one launch per row of the schedule, in place
