@@ -90,3 +90,7 @@ def rank_matrix(dist, seed, n, count):
 def workload_inputs(w: Workload, count=None):
     """All ranks' vectors of a workload (optionally only the first `count` elements)."""
     return rank_matrix(w.dist, w.seed, w.n, w.count if count is None else count)
+# Rings whose size is no power of three (Sec. 4.4; 32 is the paper's worked example), bandwidth form.
+for _n in (32, 100):
+    _name = "ring%d_bw_8MiB" % _n
+    CONFIGS[_name] = Workload(_name, (_n,), BANDWIDTH, 8 * MiB // 4, "normal", 5)

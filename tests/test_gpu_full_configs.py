@@ -54,7 +54,7 @@ def test_config_every_element(name):
 
 
 @pytest.mark.parametrize("name", ["ring243_lat_8MiB", "ring243_bw_8MiB", "ring243_lat_32MiB", "ring243_bw_32MiB",
-                                  "torus9x9x9_lat_32MiB", "torus9x9x9_bw_32MiB"])
+                                  "torus9x9x9_lat_32MiB", "torus9x9x9_bw_32MiB", "ring32_bw_8MiB", "ring100_bw_8MiB"])
 def test_config_sampled_windows(name):
     w = synth.CONFIGS[name]
     plan = binding.Plan(w.dims, w.variant)
