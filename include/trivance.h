@@ -33,7 +33,8 @@ typedef enum {
     TRV_ERR_ALLOC = 4,
     TRV_ERR_CUDA = 5,               /* a CUDA runtime call failed; cudaGetLastError has the reason */
     TRV_ERR_SCRATCH = 6,            /* caller-provided scratch/workspace too small or misaligned */
-    TRV_ERR_TOO_LARGE = 7           /* the call needs more than the fixed capacity of a no-allocation entry point */
+    TRV_ERR_TOO_LARGE = 7,          /* the call needs more than the fixed capacity of a no-allocation entry point */
+    TRV_ERR_TIMEOUT = 8             /* a bounded device-side wait of the PIPELINED kernel ran out (trv_pipeline_status) */
 } trv_status_t;
 
 typedef enum { TRV_LATENCY_OPTIMAL = 0, TRV_BANDWIDTH_OPTIMAL = 1 } trv_variant_t;
@@ -48,8 +49,14 @@ typedef enum { TRV_SUM = 0 } trv_op_t;
  *   FUSED: all steps of a column of elements on chip; one read and one write per element.
  *          Exists for the shapes trv_kernel_supported() reports.
  *   AUTO : FUSED where it exists, else STEP.
- * Both families give bit-identical results. */
-typedef enum { TRV_KERNEL_AUTO = 0, TRV_KERNEL_STEP = 1, TRV_KERNEL_FUSED = 2 } trv_kernel_t;
+ *   PIPELINED: the chunk-level readiness engine the paper sketches for a collective-library
+ *          backend (App. D): latency form only; one persistent kernel; a work item per (rank,
+ *          step, chunk) runs as soon as the chunks of both peers and the local partial of the
+ *          previous step are marked ready, with no barrier between steps.  Never chosen by AUTO.
+ *          Needs scratch (trv_scratch_bytes); all its device-side waits are bounded, see
+ *          trv_pipeline_status.
+ * All families give bit-identical results. */
+typedef enum { TRV_KERNEL_AUTO = 0, TRV_KERNEL_STEP = 1, TRV_KERNEL_FUSED = 2, TRV_KERNEL_PIPELINED = 3 } trv_kernel_t;
 
 #define TRV_MAX_DIMS 8
 #define TRV_MAX_RANKS 1024
@@ -196,6 +203,23 @@ trv_status_t trv_host_workspace_bytes(trv_plan_t plan, size_t count, size_t *byt
 trv_status_t trv_allreduce_noalloc(trv_plan_t plan, void *const *rank_buffers, size_t count, trv_dtype_t dtype,
                                    trv_op_t op, void *cuda_stream);
 size_t trv_noalloc_max_scratch_bytes(void);
+
+/* ---------------------------------------------------------------- PIPELINED family: status
+ *
+ * The PIPELINED kernel (App. D; Discussion, "Joint Reduction Overheads") waits on readiness entries
+ * inside the kernel.  Every such wait gives up after a fixed number of polls (about half a second),
+ * records TRV_ERR_TIMEOUT in the first bytes of the call's scratch and ends the kernel; the CUDA
+ * context stays usable and the output is then undefined.
+ *
+ * trv_pipeline_status: synchronises `cuda_stream`, reads that record from the DEVICE scratch of the
+ * last PIPELINED call and returns TRV_OK or TRV_ERR_TIMEOUT (TRV_ERR_CUDA if the copy fails).
+ *
+ * trv_pipeline_selftest_timeout: queues one tiny kernel whose single waiter waits, with a limit of
+ * 1000 polls, for an entry that nothing sets; a following trv_pipeline_status on the same scratch
+ * (at least 512 bytes, 256-byte aligned, DEVICE) returns TRV_ERR_TIMEOUT.  It exists so that the
+ * give-up path can be tested without making any real wait fail. */
+trv_status_t trv_pipeline_status(const void *scratch, void *cuda_stream);
+trv_status_t trv_pipeline_selftest_timeout(void *scratch, size_t scratch_bytes, void *cuda_stream);
 
 /* ---------------------------------------------------------------- link loads
  *

@@ -16,10 +16,11 @@ LATENCY_OPTIMAL, BANDWIDTH_OPTIMAL = 0, 1
 ALGO_TRIVANCE, ALGO_BRUCK, ALGO_RECDOUB = 0, 1, 2
 INT32, FLOAT32 = 0, 1
 SUM = 0
-KERNEL_AUTO, KERNEL_STEP, KERNEL_FUSED = 0, 1, 2
+KERNEL_AUTO, KERNEL_STEP, KERNEL_FUSED, KERNEL_PIPELINED = 0, 1, 2, 3
 MAX_RANKS = 1024
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_UNDEFINED_SCHEDULE, ERR_ALLOC, ERR_CUDA, ERR_SCRATCH, ERR_TOO_LARGE = range(8)
+(OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_UNDEFINED_SCHEDULE, ERR_ALLOC, ERR_CUDA, ERR_SCRATCH, ERR_TOO_LARGE,
+ ERR_TIMEOUT) = range(9)
 
 # every symbol include/trivance.h declares
 SYMBOLS = [
@@ -27,7 +28,8 @@ SYMBOLS = [
     "trv_plan_peers", "trv_plan_send_set", "trv_plan_block_bounds", "trv_allreduce", "trv_scratch_bytes",
     "trv_kernel_supported", "trv_allreduce_ex", "trv_allreduce_host", "trv_host_workspace_bytes",
     "trv_link_loads", "trv_plan_message_bytes", "trv_plan_message_bytes_side", "trv_strerror", "trv_launch_count", "trv_last_kernel_name",
-    "trv_allreduce_noalloc", "trv_noalloc_max_scratch_bytes", "trv_cost_model",
+    "trv_allreduce_noalloc", "trv_noalloc_max_scratch_bytes", "trv_cost_model", "trv_pipeline_status",
+    "trv_pipeline_selftest_timeout",
 ]
 
 
@@ -65,6 +67,8 @@ def lib():
         L.trv_plan_block_bounds.argtypes = [vp, sz, i32, vp]
         L.trv_plan_message_bytes.argtypes = [vp, sz, sz, i32, i32, vp]
         L.trv_plan_message_bytes_side.argtypes = [vp, sz, sz, i32, i32, i32, vp]
+        L.trv_pipeline_status.argtypes = [vp, vp]
+        L.trv_pipeline_selftest_timeout.argtypes = [vp, sz, vp]
         L.trv_allreduce.argtypes = [vp, vp, sz, ctypes.c_int, ctypes.c_int, vp]
         L.trv_scratch_bytes.argtypes = [vp, sz, ctypes.c_int, i32, ctypes.POINTER(sz)]
         L.trv_kernel_supported.argtypes = [vp, ctypes.c_int]
@@ -93,6 +97,15 @@ def strerror(status):
 
 def noalloc_max_scratch_bytes():
     return int(lib().trv_noalloc_max_scratch_bytes())
+
+
+def pipeline_status(scratch_ptr, stream=0):
+    """Status code (OK or ERR_TIMEOUT) recorded by the last PIPELINED call that used this device scratch."""
+    return int(lib().trv_pipeline_status(scratch_ptr, stream))
+
+
+def pipeline_selftest_timeout(scratch_ptr, scratch_bytes, stream=0):
+    _check(lib().trv_pipeline_selftest_timeout(scratch_ptr, scratch_bytes, stream), "trv_pipeline_selftest_timeout")
 
 
 def launch_count():

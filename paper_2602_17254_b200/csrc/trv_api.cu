@@ -47,6 +47,7 @@ static trv_status_t check_buffers(const Plan& p, const void* const* in, void* co
 static trv_status_t dispatch(Call& c, trv_kernel_t kernel) {
     const Plan& p = *c.plan;
     bool fused = false;
+    if (kernel == TRV_KERNEL_PIPELINED) return run_pipeline_latency(c);
     if (kernel == TRV_KERNEL_FUSED) {
         if (!fused_supported(p)) return TRV_ERR_UNSUPPORTED;
         fused = true;
@@ -154,6 +155,7 @@ trv_status_t trv_plan_message_bytes_side(trv_plan_t plan, size_t count, size_t e
 int32_t trv_kernel_supported(trv_plan_t plan, trv_kernel_t kernel) {
     if (!plan || plan->plan.algo != TRV_ALGO_TRIVANCE) return 0;
     if (kernel == TRV_KERNEL_FUSED) return fused_supported(plan->plan) ? 1 : 0;
+    if (kernel == TRV_KERNEL_PIPELINED) return pipeline_supported(plan->plan, false) ? 1 : 0;
     return (kernel == TRV_KERNEL_AUTO || kernel == TRV_KERNEL_STEP) ? 1 : 0;
 }
 
@@ -162,6 +164,11 @@ trv_status_t trv_scratch_bytes(trv_plan_t plan, size_t count, trv_kernel_t kerne
     const Plan& p = plan->plan;
     if (p.algo != TRV_ALGO_TRIVANCE) return TRV_ERR_UNSUPPORTED;
     bool fused = false;
+    if (kernel == TRV_KERNEL_PIPELINED) {
+        if (!pipeline_supported(p, in_place != 0)) return TRV_ERR_UNSUPPORTED;
+        *bytes = pipeline_scratch_bytes(p, count);
+        return TRV_OK;
+    }
     if (kernel == TRV_KERNEL_FUSED) {
         if (!fused_supported(p)) return TRV_ERR_UNSUPPORTED;
         fused = true;
@@ -182,7 +189,8 @@ trv_status_t trv_allreduce_ex(trv_plan_t plan, const void* const* in_buffers, vo
     if (p.algo != TRV_ALGO_TRIVANCE) return TRV_ERR_UNSUPPORTED;
     if (dtype != TRV_INT32 && dtype != TRV_FLOAT32) return TRV_ERR_INVALID_ARG;
     if (op != TRV_SUM) return TRV_ERR_UNSUPPORTED;
-    if (kernel != TRV_KERNEL_AUTO && kernel != TRV_KERNEL_STEP && kernel != TRV_KERNEL_FUSED) return TRV_ERR_INVALID_ARG;
+    if (kernel != TRV_KERNEL_AUTO && kernel != TRV_KERNEL_STEP && kernel != TRV_KERNEL_FUSED && kernel != TRV_KERNEL_PIPELINED)
+        return TRV_ERR_INVALID_ARG;
     if (global_offset > global_count || count > global_count - global_offset) return TRV_ERR_INVALID_ARG;
     if (count >= ((size_t)1 << 40)) return TRV_ERR_UNSUPPORTED;
     bool in_place = false;
@@ -257,6 +265,16 @@ trv_status_t trv_allreduce_host(trv_plan_t plan, const void* const* host_in, voi
     return TRV_OK;
 }
 
+trv_status_t trv_pipeline_status(const void* scratch, void* cuda_stream) {
+    if (!scratch) return TRV_ERR_INVALID_ARG;
+    return pipeline_status(scratch, (cudaStream_t)cuda_stream);
+}
+
+trv_status_t trv_pipeline_selftest_timeout(void* scratch, size_t scratch_bytes, void* cuda_stream) {
+    if (!scratch || ((uintptr_t)scratch & 255)) return TRV_ERR_SCRATCH;
+    return pipeline_selftest_timeout(scratch, scratch_bytes, (cudaStream_t)cuda_stream);
+}
+
 trv_status_t trv_link_loads(trv_plan_t plan, size_t count, size_t elem_size, int32_t* msgs, int64_t* bytes,
                             int32_t* max_msgs, int64_t* max_bytes) {
     if (!plan || elem_size == 0) return TRV_ERR_INVALID_ARG;
@@ -304,6 +322,7 @@ const char* trv_strerror(trv_status_t status) {
         case TRV_ERR_CUDA: return "CUDA runtime error";
         case TRV_ERR_SCRATCH: return "scratch or workspace too small or misaligned";
         case TRV_ERR_TOO_LARGE: return "size exceeds the fixed scratch capacity of the no-allocation entry point";
+        case TRV_ERR_TIMEOUT: return "a bounded device-side wait of the pipelined kernel ran out";
     }
     return "unknown status";
 }

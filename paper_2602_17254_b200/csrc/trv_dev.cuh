@@ -160,6 +160,13 @@ trv_status_t run_fused_bandwidth(const Call& c);
 bool fused_tree_supported(const Plan& p);
 trv_status_t run_fused_tree(const Call& c);
 
+// chunk-level readiness engine (trv_pipe.cu)
+bool pipeline_supported(const Plan& p, bool in_place);
+size_t pipeline_scratch_bytes(const Plan& p, size_t count);
+trv_status_t run_pipeline_latency(const Call& c);
+trv_status_t pipeline_status(const void* scratch, cudaStream_t st);
+trv_status_t pipeline_selftest_timeout(void* scratch, size_t scratch_bytes, cudaStream_t st);
+
 // link-load tally (trv_linkloads.cu)
 trv_status_t run_link_loads(const Plan& p, size_t count, size_t elem_size, int32_t* msgs, int64_t* bytes,
                             int32_t* max_msgs, int64_t* max_bytes);

@@ -32,11 +32,11 @@ def test_header_symbols_are_exported(library):
 
 def test_strerror_covers_every_status(library):
     seen = set()
-    for s in range(8):
+    for s in range(9):
         msg = binding.strerror(s)
         assert msg and msg != "unknown status"
         seen.add(msg)
-    assert len(seen) == 8
+    assert len(seen) == 9
     assert binding.strerror(99) == "unknown status"
 
 
