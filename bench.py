@@ -244,7 +244,8 @@ def run_ours(args, w):
             ins[b].normal_(generator=g) if w.dist == "normal" else ins[b].uniform_(-1.0, 1.0, generator=g)
     in_ptrs = [binding.ptr_array([ins[b, r].data_ptr() for r in range(n)]) for b in range(batch)]
     out_ptrs = [binding.ptr_array([outs[b, r].data_ptr() for r in range(n)]) for b in range(batch)]
-    kfam = {"auto": binding.KERNEL_AUTO, "step": binding.KERNEL_STEP, "fused": binding.KERNEL_FUSED}[args.kernel]
+    kfam = {"auto": binding.KERNEL_AUTO, "step": binding.KERNEL_STEP, "fused": binding.KERNEL_FUSED,
+            "pipelined": binding.KERNEL_PIPELINED}[args.kernel]
     need = plan.scratch_bytes(count, kfam, in_place=False)
     scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
@@ -409,8 +410,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--dims", default="", help="ad-hoc torus sides, e.g. 27,27 (overrides the workload's topology)")
     ap.add_argument("--variant", default="latency", choices=["latency", "bandwidth"], help="form for --dims")
-    ap.add_argument("--kernel", default="auto", choices=["auto", "step", "fused"],
-                    help="kernel family (step = one launch per schedule step, as the paper states the steps)")
+    ap.add_argument("--kernel", default="auto", choices=["auto", "step", "fused", "pipelined"],
+                    help="kernel family (step = one launch per schedule step, as the paper states the steps; "
+                         "pipelined = chunk-level readiness engine, latency form only)")
     ap.add_argument("--graph", action="store_true", help="capture one step in a CUDA graph and time its replays")
     ap.add_argument("--count", type=int, default=0, help="override the workload's elements per rank")
     ap.add_argument("--profile", action="store_true",

@@ -7,7 +7,7 @@
 // belongs to the current generation, reads the two incoming chunks where they were received, and
 // adds them to the local partial; chunks are taken in the same order on both sides.
 //
-// Here: ONE persistent kernel.  A work item is (chunk, step, rank).  All ranks share one address
+// Here: ONE persistent kernel whose warps are the workers.  A work item is (chunk, step, rank).  All ranks share one address
 // space, so the peer's partial of the previous step IS the receive slot: nothing is copied, and
 // "the left chunk has arrived" means "the left peer has finished this chunk's previous step".
 // The readiness entry of (chunk, rank) is a counter of finished steps, written with release
@@ -19,9 +19,9 @@
 //
 // Items are handed out by a ticket counter in a fixed total order in which every item comes after
 // the items it waits for (groups of K chunks; inside a group step by step, inside a step chunk by
-// chunk, rank by rank).  A CTA therefore only ever waits for items that were taken earlier, by CTAs
+// chunk, rank by rank).  A warp therefore only ever waits for items that were taken earlier, by warps
 // that are already running: no deadlock whatever the grid size, no cooperative launch needed.  K is
-// chosen so that one step of a group is about two grids' worth of items: when a CTA reaches step
+// chosen so that one step of a group is about two grids' worth of items: when a warp reaches step
 // t + 1 of a group, step t is almost always done, and a group's working set stays in L2 across all
 // steps, so the HBM traffic is close to one read and one write of the vectors although every step
 // re-reads its inputs.
@@ -91,17 +91,19 @@ __device__ __forceinline__ bool wait_entry(const int* entry, int need, PipeHeade
 template <typename T>
 __device__ __forceinline__ T ld_cg(const T* p) { return __ldcg(p); }
 
+// Every WARP is a worker of its own: it draws tickets, waits and publishes without involving the
+// rest of its CTA, so a CTA keeps eight items in flight.
 template <typename T, int CAP>
 __global__ void __launch_bounds__(kPipeThreads) k_lat_pipe(PtrTab<CAP> in, PtrTab<CAP> out, PipeArgs a) {
     using V = typename Vec4<T>::type;
-    __shared__ long long s_item;
-    const int tid = threadIdx.x;
+    constexpr unsigned kFull = 0xffffffffu;
+    const int lane = threadIdx.x & 31;
     const long long per_chunk = (long long)a.S * a.n;
     const long long total = (long long)a.nchunks * per_chunk;
     for (;;) {
-        if (tid == 0) s_item = (long long)atomicAdd(&a.hdr->ticket, 1ULL);
-        __syncthreads();
-        const long long item = s_item;
+        long long item = 0;
+        if (lane == 0) item = (long long)atomicAdd(&a.hdr->ticket, 1ULL);
+        item = __shfl_sync(kFull, item, 0);
         if (item >= total) break;
         // item -> (chunk c, step t, rank p): groups of K chunks, step-major inside a group
         const long long gsz = (long long)a.group * per_chunk;
@@ -120,20 +122,20 @@ __global__ void __launch_bounds__(kPipeThreads) k_lat_pipe(PtrTab<CAP> in, PtrTa
 
         // ---- readiness: both incoming chunks and the local partial; then the buffer to overwrite
         int ok = 1;
-        if (t > 0 && tid < 7) {
+        if (t > 0 && lane < 7) {
             int q = -1, need = t;
-            if (tid == 0) q = pl;
-            else if (tid == 1) q = pr;
-            else if (tid == 2) q = p;
-            else if (tid == 3) q = peer_of(p, a.stride[sl][t - 1], a.size[sl][t - 1], -a.dist[sl][t - 1]);
-            else if (tid == 4) q = peer_of(p, a.stride[sl][t - 1], a.size[sl][t - 1], +a.dist[sl][t - 1]);
+            if (lane == 0) q = pl;
+            else if (lane == 1) q = pr;
+            else if (lane == 2) q = p;
+            else if (lane == 3) q = peer_of(p, a.stride[sl][t - 1], a.size[sl][t - 1], -a.dist[sl][t - 1]);
+            else if (lane == 4) q = peer_of(p, a.stride[sl][t - 1], a.size[sl][t - 1], +a.dist[sl][t - 1]);
             else if (a.in_place && t == a.S - 1) {
-                q = peer_of(p, a.stride[sl][0], a.size[sl][0], tid == 5 ? -a.dist[sl][0] : +a.dist[sl][0]);
+                q = peer_of(p, a.stride[sl][0], a.size[sl][0], lane == 5 ? -a.dist[sl][0] : +a.dist[sl][0]);
                 need = 1;
             }
             if (q >= 0) ok = wait_entry(a.done + (size_t)c * a.n + q, need, a.hdr, a.spin_limit, item) ? 1 : 0;
         }
-        ok = __syncthreads_and(ok);
+        ok = __all_sync(kFull, ok);
         if (!ok) break;
 
         // ---- the joint reduction of this chunk: (from_left + own) + from_right
@@ -151,16 +153,17 @@ __global__ void __launch_bounds__(kPipeThreads) k_lat_pipe(PtrTab<CAP> in, PtrTa
         long long ahi = e1 & ~3LL;
         if (ahi < alo) ahi = alo;
         const long long head = alo - e0, tail = e1 - ahi;
-        if (tid < head) { const long long e = e0 + tid; O[e] = add3(ld_cg(L + e), ld_cg(M + e), ld_cg(R + e)); }
-        else if (tid < head + tail) { const long long e = ahi + (tid - head); O[e] = add3(ld_cg(L + e), ld_cg(M + e), ld_cg(R + e)); }
-        for (long long e = alo + 4LL * tid; e < ahi; e += 4LL * kPipeThreads) {
+        if (lane < head) { const long long e = e0 + lane; O[e] = add3(ld_cg(L + e), ld_cg(M + e), ld_cg(R + e)); }
+        else if (lane < head + tail) { const long long e = ahi + (lane - head); O[e] = add3(ld_cg(L + e), ld_cg(M + e), ld_cg(R + e)); }
+#pragma unroll 4
+        for (long long e = alo + 4LL * lane; e < ahi; e += 128) {
             const V l = ld_cg((const V*)(L + e)), m = ld_cg((const V*)(M + e)), r = ld_cg((const V*)(R + e));
             *(V*)(O + e) = add3v(l, m, r);
         }
         // ---- publish: this chunk of rank p has finished step t
         __threadfence();
-        __syncthreads();
-        if (tid == 0) st_release(a.done + (size_t)c * a.n + p, t + 1);
+        __syncwarp();
+        if (lane == 0) st_release(a.done + (size_t)c * a.n + p, t + 1);
     }
 }
 
@@ -173,7 +176,9 @@ __global__ void k_pipe_wait_never(PipeHeader* hdr, const int* entry, unsigned li
 
 static size_t pipe_padded(size_t count) { return (count + 63) & ~(size_t)63; }
 static int pipe_buffers(const Plan& p) { return p.S >= 3 ? 2 : (p.S == 2 ? 1 : 0); }
-static int pipe_chunk_elems(size_t count) { return count >= ((size_t)1 << 22) ? 2048 : 1024; }
+// Measured on B200 (ring 27 x 2 MiB / ring 243 x 8 MiB, us per call): 512 elements 135 / 5854, 1024: 112 / 4455,
+// 2048: 81 / 4126, 4096: 116 / 3961 (with groups of two grids' worth of items; one grid's worth: 104 / 4336).
+static int pipe_chunk_elems(size_t count) { return count >= ((size_t)1 << 16) ? 2048 : 1024; }
 
 static int pipe_chunks(const Call& c, int chunk_elems, int* cbase) {
     int total = 0;
@@ -216,8 +221,9 @@ static trv_status_t pipe_impl(const Call& c, PipeArgs& a) {
         return TRV_ERR_CUDA;
     const long long total = (long long)a.nchunks * a.S * a.n;
     long long grid = (long long)sms * per_sm;
-    if (grid > total) grid = total;
-    a.group = (int)((2 * grid + a.n - 1) / a.n);
+    if (grid > (total + 7) / 8) grid = (total + 7) / 8;
+    const long long workers = grid * (kPipeThreads / 32);
+    a.group = (int)((2 * workers + a.n - 1) / a.n);
     if (a.group < 1) a.group = 1;
     // the generation: ticket, error and all readiness entries start at zero
     const size_t entries = (size_t)a.nchunks * a.n * sizeof(int);

@@ -80,7 +80,7 @@ def test_short_vectors(dims, count):
 
 def test_many_groups():
     """More chunks than one group holds: several groups of chunks follow one another through all steps."""
-    _run((27,), 400003, "normal", 46)
+    _run((27,), 1500007, "normal", 46)
     _run((9, 9), 300007, "int32", 47, in_place=False)
 
 
