@@ -22,9 +22,12 @@
 // chunk, rank by rank).  A warp therefore only ever waits for items that were taken earlier, by warps
 // that are already running: no deadlock whatever the grid size, no cooperative launch needed.  K is
 // chosen so that one step of a group is about two grids' worth of items: when a warp reaches step
-// t + 1 of a group, step t is almost always done, and a group's working set stays in L2 across all
-// steps, so the HBM traffic is close to one read and one write of the vectors although every step
-// re-reads its inputs.
+// t + 1 of a group, step t is almost always done and nobody spins.  What bounds the engine is the
+// latency of an item (ticket, readiness loads, data round trip, fence, publish) times the items
+// per worker, so it runs with as many resident warps as fit; a group is then too large to stay in
+// L2 (2 x 5920 workers x 8 KB = 97 MB per buffer) and the DRAM traffic is 4.8x the one-read-one-
+// write minimum (ring 243: the STEP family moves 7x).  Smaller grids or chunks, which would keep a
+// group in L2, were 1.5 to 5x slower.
 //
 // Every wait is bounded: after kSpinLimit polls a waiter records TRV_ERR_TIMEOUT and the item in
 // the header, every other waiter sees that and leaves, and the kernel ends; trv_pipeline_status
