@@ -33,21 +33,12 @@
 // the header, every other waiter sees that and leaves, and the kernel ends; trv_pipeline_status
 // reports it.  Data written by other SMs is read with L1-bypassing loads.
 #include "trv_dev.cuh"
+#include "trv_wait.cuh"
 
 namespace trv {
 
 constexpr int kPipeThreads = 256;
 constexpr int kPipeMaxS = 8;
-constexpr unsigned kSpinLimit = 1u << 21;     // polls of >= 200 ns each: gives up after roughly half a second
-constexpr size_t kPipeHeaderBytes = 256;
-
-struct PipeHeader {
-    unsigned long long ticket;
-    int error;                  // 0, or TRV_ERR_TIMEOUT
-    int pad;
-    long long where;            // the item that gave up
-};
-
 struct PipeArgs {
     int n, S, nslices, in_place;
     int chunk_elems, nchunks, group;        // elements per chunk; chunks in all slices; chunks per group (K)
@@ -61,34 +52,12 @@ struct PipeArgs {
     PipeHeader* hdr;
 };
 
-__device__ __forceinline__ int ld_acquire(const int* p) {
-    int v;
-    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_release(int* p, int v) {
-    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
 __device__ __forceinline__ int peer_of(int p, int stride, int size, int delta) {
     const int x = (p / stride) % size;
     int y = x + delta;
     if (y < 0) y += size;
     if (y >= size) y -= size;
     return p + (y - x) * stride;
-}
-
-// Waits until *entry >= need.  false: gave up (limit reached or another waiter already gave up).
-__device__ __forceinline__ bool wait_entry(const int* entry, int need, PipeHeader* hdr, unsigned limit, long long item) {
-    unsigned spins = 0;
-    while (ld_acquire(entry) < need) {
-        if (ld_acquire(&hdr->error) != 0) return false;
-        if (++spins > limit) {
-            if (atomicCAS(&hdr->error, 0, (int)TRV_ERR_TIMEOUT) == 0) hdr->where = item;
-            return false;
-        }
-        __nanosleep(200);
-    }
-    return true;
 }
 
 template <typename T>
