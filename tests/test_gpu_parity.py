@@ -198,7 +198,9 @@ def test_launch_counter_and_kernel_names():
 def test_calls_can_be_captured_in_a_cuda_graph():
     """The AllReduce call is a pure launch sequence (no allocation, no synchronisation): it can be
     captured into a CUDA graph and replayed; replays give the oracle's bits."""
-    for dims, variant, kernel in [((27,), LAT, FUSED), ((243,), BW, FUSED), ((9, 9), LAT, STEP), ((9, 9, 9), LAT, FUSED)]:
+    for dims, variant, kernel in [((27,), LAT, FUSED), ((243,), BW, FUSED), ((9, 9), LAT, STEP), ((9, 9, 9), LAT, FUSED),
+                                  ((100,), BW, FUSED), ((32,), BW, STEP), ((27,), LAT, binding.KERNEL_PIPELINED),
+                                  ((3, 9), LAT, binding.KERNEL_PIPELINED)]:
         plan = binding.Plan(dims, variant)
         n, count = plan.n, 2048
         x = synth.rank_matrix("normal", 77, n, count)
