@@ -38,7 +38,8 @@ typedef enum {
 } trv_status_t;
 
 typedef enum { TRV_LATENCY_OPTIMAL = 0, TRV_BANDWIDTH_OPTIMAL = 1 } trv_variant_t;
-typedef enum { TRV_ALGO_TRIVANCE = 0, TRV_ALGO_BRUCK = 1, TRV_ALGO_RECDOUB = 2 } trv_algo_t;
+typedef enum { TRV_ALGO_TRIVANCE = 0, TRV_ALGO_BRUCK = 1, TRV_ALGO_RECDOUB = 2, TRV_ALGO_SWING = 3, TRV_ALGO_BUCKET = 4,
+               TRV_ALGO_MIRRORED = 16 /* flag, see trv_plan_create_algo */ } trv_algo_t;
 typedef enum { TRV_INT32 = 0, TRV_FLOAT32 = 1 } trv_dtype_t;
 typedef enum { TRV_SUM = 0 } trv_op_t;
 
@@ -91,8 +92,17 @@ trv_status_t trv_plan_create(const int32_t *dims, int32_t ndims, trv_variant_t v
 /* Same, for a comparator schedule (Sec. 2.4, Fig. 1).  TRV_ALGO_BRUCK: peers r + 3^k and
  * r + 2*3^k, both sent in the + direction.  TRV_ALGO_RECDOUB: peer r XOR 2^k on a ring of
  * 2^q ranks (ndims must be 1), the lower rank of a pair sending in the + direction;
- * UNDEFINED_SCHEDULE for other ring sizes.  Comparator plans serve trv_link_loads and the
- * schedule queries only; trv_allreduce returns UNSUPPORTED for them. */
+ * UNDEFINED_SCHEDULE for other ring sizes.  TRV_ALGO_SWING: peer r + rho(k) for even r and
+ * r - rho(k) for odd r, rho(k) = sum_{i<=k} (-2)^i = 1, -1, 3, -5, ... on a ring of 2^q ranks, each
+ * message the short way round; block sets by Algorithm 1.  TRV_ALGO_BUCKET: the ring algorithm,
+ * n - 1 steps per phase on a ring of any n >= 2, every step one block to the next node (bandwidth
+ * form only; rows 0..n-2 Reduce-Scatter, n-1..2n-3 AllGather, both counted forwards).
+ * `algo | TRV_ALGO_MIRRORED` (rings, not Trivance): the collective runs a second time with every
+ * direction reversed, the two sharing the vector half and half (the mirrored sub-collective by
+ * which these one-port schedules use both ports, Sec. 2.4); the plan then has two collectives
+ * (trv_plan_slices), the second one with negated distances.
+ * Comparator plans serve trv_link_loads, trv_cost_model and the schedule queries only;
+ * trv_allreduce returns UNSUPPORTED for them. */
 trv_status_t trv_plan_create_algo(const int32_t *dims, int32_t ndims, trv_variant_t variant, trv_algo_t algo,
                                   trv_plan_t *out);
 
@@ -102,6 +112,9 @@ trv_status_t trv_plan_destroy(trv_plan_t plan);
  * bandwidth form (Reduce-Scatter steps 0..S-1, then the AllGather steps, which mirror
  * S-1..0, Sec. 4.1).  Any output may be NULL. */
 trv_status_t trv_plan_info(trv_plan_t plan, int32_t *n, int32_t *ndims, int32_t *rows);
+
+/* Number of concurrent collectives (slices of the vector): ndims, or 2 * ndims for a mirrored comparator. */
+trv_status_t trv_plan_slices(trv_plan_t plan, int32_t *nslices);
 
 /* Row `row` of collective (slice) c: the dimension it runs along and the ring distance. */
 trv_status_t trv_plan_step(trv_plan_t plan, int32_t c, int32_t row, int32_t *dim, int32_t *dist);

@@ -52,13 +52,14 @@
 #define ORC_MAX_DIMS 8
 
 enum { ORC_OK = 0, ORC_BAD_ARG = 1, ORC_UNDEFINED = 2, ORC_NOMEM = 3, ORC_INTERNAL = 4 };
-enum { ORC_TRIVANCE = 0, ORC_BRUCK = 1, ORC_RECDOUB = 2 };
+enum { ORC_TRIVANCE = 0, ORC_BRUCK = 1, ORC_RECDOUB = 2, ORC_SWING = 3, ORC_BUCKET = 4, ORC_MIRROR = 16 };
 enum { ORC_LATENCY = 0, ORC_BANDWIDTH = 1 };
 enum { ORC_I32 = 0, ORC_F32 = 1, ORC_F64 = 2 };
 
 typedef struct {
     int algo, ndims, n, S;          /* S = steps per phase, summed over dimensions */
-    int base;                       /* 3 (Trivance, Bruck) or 2 (Recursive Doubling) */
+    int nsl;                        /* concurrent collectives (slices): ndims, or 2*ndims when mirrored */
+    int base;                       /* 3 (Trivance, Bruck) or 2 (Recursive Doubling, Swing) */
     int dims[ORC_MAX_DIMS];
     int stride[ORC_MAX_DIMS];       /* rank = sum x_d * stride_d */
     int sdim[ORC_MAX_DIMS];         /* steps spent in dimension d = log_base a_d */
@@ -71,11 +72,24 @@ static int ilog_exact(int a, int base) {       /* log_base a, or -1 if a is no p
     return s;
 }
 
+/* `algo` may carry the ORC_MIRROR flag (comparators on rings only): the collective then runs a
+ * second time with every direction reversed, the two sharing the vector half and half -- the
+ * "mirrored sub-collective" by which the one-port comparators use both ports (Sec. 2.4). */
 static int topo_init(orc_topo *tp, const int32_t *dims, int ndims, int algo) {
     if (!dims || ndims < 1 || ndims > ORC_MAX_DIMS) return ORC_BAD_ARG;
-    if (algo != ORC_TRIVANCE && algo != ORC_BRUCK && algo != ORC_RECDOUB) return ORC_BAD_ARG;
-    tp->algo = algo; tp->ndims = ndims; tp->base = (algo == ORC_RECDOUB) ? 2 : 3;
-    if (algo == ORC_RECDOUB && ndims != 1) return ORC_UNDEFINED;
+    int mirror = (algo & ORC_MIRROR) ? 1 : 0;
+    algo &= ~ORC_MIRROR;
+    if (algo < ORC_TRIVANCE || algo > ORC_BUCKET) return ORC_BAD_ARG;
+    if (mirror && (algo == ORC_TRIVANCE || ndims != 1)) return ORC_BAD_ARG;
+    tp->algo = algo; tp->ndims = ndims; tp->nsl = ndims * (mirror ? 2 : 1);
+    tp->base = (algo == ORC_RECDOUB || algo == ORC_SWING) ? 2 : 3;
+    if ((algo == ORC_RECDOUB || algo == ORC_SWING || algo == ORC_BUCKET) && ndims != 1) return ORC_UNDEFINED;
+    if (algo == ORC_BUCKET) {           /* ring algorithm: any n >= 2, n - 1 steps per phase (Sec. 2.4) */
+        if (dims[0] < 2 || dims[0] > 4096) return ORC_BAD_ARG;
+        tp->dims[0] = dims[0]; tp->stride[0] = 1; tp->sdim[0] = dims[0] - 1;
+        tp->n = dims[0]; tp->S = dims[0] - 1;
+        return ORC_OK;
+    }
     long long n = 1; tp->S = 0;
     for (int d = 0; d < ndims; ++d) {
         int s = ilog_exact(dims[d], tp->base);
@@ -93,14 +107,19 @@ static int ipow(int b, int e) { int r = 1; while (e-- > 0) r *= b; return r; }
 /* Step list of collective (slice) c (Sec. 5): round-robin over dimensions,
  * starting at dimension c, skipping dimensions whose steps are used up; the
  * distance in a dimension grows by the base each time it is revisited. */
+/* Swing's signed distance rho(k) = sum_{i<=k} (-2)^i = 1, -1, 3, -5, 11, ... (Sec. 2.4) */
+static int swing_rho(int k) { int r = 0, p = 1; for (int i = 0; i <= k; ++i) { r += p; p *= -2; } return r; }
+
+/* A mirrored slice (c >= ndims) gets negated distances: send_peers reverses everything for them. */
 static void step_list(const orc_topo *tp, int c, int *sdim_out, int *sdist_out) {
     int visits[ORC_MAX_DIMS] = {0};
+    int mir = (c >= tp->ndims) ? -1 : 1;
     int cur = c % tp->ndims;
     for (int t = 0; t < tp->S; ++t) {
         int d = cur;
         while (visits[d] >= tp->sdim[d]) d = (d + 1) % tp->ndims;
         sdim_out[t] = d;
-        sdist_out[t] = ipow(tp->base, visits[d]);
+        sdist_out[t] = mir * ((tp->algo == ORC_SWING) ? swing_rho(visits[d]) : ipow(tp->base, visits[d]));
         visits[d]++;
         cur = (d + 1) % tp->ndims;
     }
@@ -125,16 +144,35 @@ static int send_peers(const orc_topo *tp, int r, int d, int dist, int *peer, int
         peer[1] = shift_rank(tp, r, d, +dist); dir[1] = +1; hops[1] = dist;
         return 2;
     }
-    if (tp->algo == ORC_BRUCK) {
-        peer[0] = shift_rank(tp, r, d, dist);     dir[0] = +1; hops[0] = dist;
-        peer[1] = shift_rank(tp, r, d, 2 * dist); dir[1] = +1; hops[1] = 2 * dist;
-        return 2;
-    }
     {
-        int st = tp->stride[d], x = (r / st) % tp->dims[d];
-        int y = x ^ dist;
-        peer[0] = r + (y - x) * st; dir[0] = (y > x) ? +1 : -1; hops[0] = dist;
-        return 1;
+        /* comparators: a negative distance is the mirrored collective -- same pattern, every
+         * displacement and direction of travel reversed */
+        int sg = dist < 0 ? -1 : 1, a = dist < 0 ? -dist : dist;
+        if (tp->algo == ORC_BRUCK) {
+            peer[0] = shift_rank(tp, r, d, sg * a);     dir[0] = sg; hops[0] = a;
+            peer[1] = shift_rank(tp, r, d, sg * 2 * a); dir[1] = sg; hops[1] = 2 * a;
+            return 2;
+        }
+        if (tp->algo == ORC_SWING) {
+            /* pi(r,k) = r + rho(k) for even r, r - rho(k) for odd r (Sec. 2.4); here dist = +-rho(k), whose
+             * own sign is part of the pattern.  The message travels the short way round: |rho| < n/2. */
+            int st = tp->stride[d], x = (r / st) % tp->dims[d];
+            int delta = (x % 2 == 0) ? dist : -dist;
+            peer[0] = shift_rank(tp, r, d, delta); dir[0] = delta > 0 ? +1 : -1; hops[0] = delta > 0 ? delta : -delta;
+            return 1;
+        }
+        if (tp->algo == ORC_BUCKET) {       /* every step: one block to the next node of the ring */
+            peer[0] = shift_rank(tp, r, d, sg); dir[0] = sg; hops[0] = 1;
+            return 1;
+        }
+        {   /* Recursive Doubling: the pair (x, x XOR a); mirrored: the ring read backwards */
+            int st = tp->stride[d], x = (r / st) % tp->dims[d];
+            int xm = sg > 0 ? x : (tp->dims[d] - x) % tp->dims[d];
+            int ym = xm ^ a;
+            int y = sg > 0 ? ym : (tp->dims[d] - ym) % tp->dims[d];
+            peer[0] = r + (y - x) * st; dir[0] = (ym > xm) ? sg : -sg; hops[0] = a;
+            return 1;
+        }
     }
 }
 
@@ -182,7 +220,8 @@ int orc_num_steps(const int32_t *dims, int ndims, int algo, int *n_out, int *S_o
 int orc_step_list(const int32_t *dims, int ndims, int algo, int c, int32_t *dim_out, int32_t *dist_out) {
     orc_topo tp; int rc = topo_init(&tp, dims, ndims, algo);
     if (rc) return rc;
-    if (c < 0 || c >= ndims) return ORC_BAD_ARG;
+    if (tp.algo == ORC_BUCKET) return ORC_UNDEFINED;     /* n - 1 single-block steps: see orc_link_loads */
+    if (c < 0 || c >= tp.nsl) return ORC_BAD_ARG;
     int sd[64], sx[64];
     step_list(&tp, c, sd, sx);
     for (int t = 0; t < tp.S; ++t) { dim_out[t] = sd[t]; dist_out[t] = sx[t]; }
@@ -194,7 +233,8 @@ int orc_step_list(const int32_t *dims, int ndims, int algo, int c, int32_t *dim_
 int orc_peers(const int32_t *dims, int ndims, int algo, int c, int step, int32_t *peers_out) {
     orc_topo tp; int rc = topo_init(&tp, dims, ndims, algo);
     if (rc) return rc;
-    if (c < 0 || c >= ndims || step < 0 || step >= tp.S) return ORC_BAD_ARG;
+    if (tp.algo == ORC_BUCKET) return ORC_UNDEFINED;     /* n - 1 single-block steps: see orc_link_loads */
+    if (c < 0 || c >= tp.nsl || step < 0 || step >= tp.S) return ORC_BAD_ARG;
     int sd[64], sx[64];
     step_list(&tp, c, sd, sx);
     for (int r = 0; r < tp.n; ++r) {
@@ -209,7 +249,8 @@ int orc_peers(const int32_t *dims, int ndims, int algo, int c, int step, int32_t
 int orc_block_propagation(const int32_t *dims, int ndims, int algo, int c, int r, int step, uint8_t *marks) {
     orc_topo tp; int rc = topo_init(&tp, dims, ndims, algo);
     if (rc) return rc;
-    if (c < 0 || c >= ndims || r < 0 || r >= tp.n || step < 0) return ORC_BAD_ARG;
+    if (tp.algo == ORC_BUCKET) return ORC_UNDEFINED;     /* n - 1 single-block steps: see orc_link_loads */
+    if (c < 0 || c >= tp.nsl || r < 0 || r >= tp.n || step < 0) return ORC_BAD_ARG;
     int sd[64], sx[64];
     step_list(&tp, c, sd, sx);
     memset(marks, 0, (size_t)tp.n);
@@ -221,7 +262,8 @@ int orc_block_propagation(const int32_t *dims, int ndims, int algo, int c, int r
 int orc_send_set(const int32_t *dims, int ndims, int algo, int c, int p, int k, uint8_t *set) {
     orc_topo tp; int rc = topo_init(&tp, dims, ndims, algo);
     if (rc) return rc;
-    if (c < 0 || c >= ndims || p < 0 || p >= tp.n || k < 0 || k >= tp.S) return ORC_BAD_ARG;
+    if (tp.algo == ORC_BUCKET) return ORC_UNDEFINED;     /* n - 1 single-block steps: see orc_link_loads */
+    if (c < 0 || c >= tp.nsl || p < 0 || p >= tp.n || k < 0 || k >= tp.S) return ORC_BAD_ARG;
     int sd[64], sx[64];
     step_list(&tp, c, sd, sx);
     send_set(&tp, sd, sx, p, k, set);
@@ -425,7 +467,24 @@ int orc_bytes_sent(const int32_t *dims, int ndims, int variant, int algo, int64_
     if (rc) return rc;
     if (E < 0 || elem_size < 1 || !sent) return ORC_BAD_ARG;
     if (variant != ORC_LATENCY && variant != ORC_BANDWIDTH) return ORC_BAD_ARG;
-    int n = tp.n, D = tp.ndims, S = tp.S, T = (variant == ORC_BANDWIDTH) ? 2 * S : S;
+    int n = tp.n, D = tp.nsl, S = tp.S, T = (variant == ORC_BANDWIDTH) ? 2 * S : S;
+    if (tp.algo == ORC_BUCKET) {
+        /* Reduce-Scatter step t: node r sends block (r - t - 1) mod n on; AllGather step t: block (r - t) mod n
+         * (block j ends at node j); a mirrored collective runs the ring the other way round (Sec. 2.4). */
+        if (variant != ORC_BANDWIDTH) return ORC_UNDEFINED;
+        memset(sent, 0, sizeof(int64_t) * (size_t)n);
+        for (int c = 0; c < D; ++c) {
+            int64_t slo, shi; int sg = c >= tp.ndims ? -1 : 1;
+            slice_bounds(E, D, c, &slo, &shi);
+            for (int row = 0; row < T; ++row)
+                for (int r = 0; r < n; ++r) {
+                    int t = row < S ? row : row - S;
+                    int j = (((r - sg * (t + (row < S ? 1 : 0))) % n) + n) % n;
+                    sent[r] += (block_bound(slo, shi, n, j + 1) - block_bound(slo, shi, n, j)) * elem_size;
+                }
+        }
+        return ORC_OK;
+    }
     uint8_t *set = (uint8_t *)malloc((size_t)n);
     uint8_t *have = (uint8_t *)malloc((size_t)n * n), *snap = (uint8_t *)malloc((size_t)n * n);
     int64_t *blen = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);
@@ -485,7 +544,8 @@ int orc_link_loads(const int32_t *dims, int ndims, int variant, int algo, int64_
     if (rc) return rc;
     if (E < 0 || elem_size < 1) return ORC_BAD_ARG;
     if (variant != ORC_LATENCY && variant != ORC_BANDWIDTH) return ORC_BAD_ARG;
-    int n = tp.n, D = tp.ndims, S = tp.S, T = (variant == ORC_BANDWIDTH) ? 2 * S : S;
+    int n = tp.n, D = tp.ndims, NSL = tp.nsl, S = tp.S, T = (variant == ORC_BANDWIDTH) ? 2 * S : S;
+    if (tp.algo == ORC_BUCKET && variant != ORC_BANDWIDTH) return ORC_UNDEFINED;
     size_t links = (size_t)n * D * 2;
     int32_t *lm = (int32_t *)calloc((size_t)T * links, sizeof(int32_t));
     int64_t *lb = (int64_t *)calloc((size_t)T * links, sizeof(int64_t));
@@ -494,11 +554,25 @@ int orc_link_loads(const int32_t *dims, int ndims, int variant, int algo, int64_
     int64_t *blen = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);
     if (!lm || !lb || !set || !have || !snap || !blen) { rc = ORC_NOMEM; goto done; }
 
-    for (int c = 0; c < D; ++c) {
+    if (tp.algo == ORC_BUCKET) {        /* one block per node and step, one hop, always the same way round */
+        for (int c = 0; c < NSL; ++c) {
+            int64_t slo, shi; int sg = c >= tp.ndims ? -1 : 1;
+            slice_bounds(E, NSL, c, &slo, &shi);
+            for (int row = 0; row < T; ++row)
+                for (int r = 0; r < n; ++r) {
+                    int t = row < S ? row : row - S;
+                    int j = (((r - sg * (t + (row < S ? 1 : 0))) % n) + n) % n;
+                    size_t li = (((size_t)row * n + r) * D + 0) * 2 + (sg > 0 ? 0 : 1);
+                    lm[li] += 1;
+                    lb[li] += (block_bound(slo, shi, n, j + 1) - block_bound(slo, shi, n, j)) * elem_size;
+                }
+        }
+    } else
+    for (int c = 0; c < NSL; ++c) {
         int sd[64], sx[64];
         int64_t slo, shi;
         step_list(&tp, c, sd, sx);
-        slice_bounds(E, D, c, &slo, &shi);
+        slice_bounds(E, NSL, c, &slo, &shi);
         for (int j = 0; j < n; ++j) blen[j] = block_bound(slo, shi, n, j + 1) - block_bound(slo, shi, n, j);
         memset(have, 0, (size_t)n * n);
         for (int r = 0; r < n; ++r) have[(size_t)r * n + r] = 1;

@@ -13,7 +13,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libtrivance.so")
 
 LATENCY_OPTIMAL, BANDWIDTH_OPTIMAL = 0, 1
-ALGO_TRIVANCE, ALGO_BRUCK, ALGO_RECDOUB = 0, 1, 2
+ALGO_TRIVANCE, ALGO_BRUCK, ALGO_RECDOUB, ALGO_SWING, ALGO_BUCKET = 0, 1, 2, 3, 4
+ALGO_MIRRORED = 16
 INT32, FLOAT32 = 0, 1
 SUM = 0
 KERNEL_AUTO, KERNEL_STEP, KERNEL_FUSED, KERNEL_PIPELINED = 0, 1, 2, 3
@@ -24,7 +25,7 @@ MAX_RANKS = 1024
 
 # every symbol include/trivance.h declares
 SYMBOLS = [
-    "trv_plan_create", "trv_plan_create_algo", "trv_plan_destroy", "trv_plan_info", "trv_plan_step",
+    "trv_plan_create", "trv_plan_create_algo", "trv_plan_destroy", "trv_plan_info", "trv_plan_slices", "trv_plan_step",
     "trv_plan_peers", "trv_plan_send_set", "trv_plan_block_bounds", "trv_allreduce", "trv_scratch_bytes",
     "trv_kernel_supported", "trv_allreduce_ex", "trv_allreduce_host", "trv_host_workspace_bytes",
     "trv_link_loads", "trv_plan_message_bytes", "trv_plan_message_bytes_side", "trv_strerror", "trv_launch_count", "trv_last_kernel_name",
@@ -66,6 +67,7 @@ def lib():
         L.trv_plan_send_set.argtypes = [vp, i32, i32, i32, vp]
         L.trv_plan_block_bounds.argtypes = [vp, sz, i32, vp]
         L.trv_plan_message_bytes.argtypes = [vp, sz, sz, i32, i32, vp]
+        L.trv_plan_slices.argtypes = [vp, vp]
         L.trv_plan_message_bytes_side.argtypes = [vp, sz, sz, i32, i32, i32, vp]
         L.trv_pipeline_status.argtypes = [vp, vp]
         L.trv_pipeline_selftest_timeout.argtypes = [vp, sz, vp]
@@ -149,6 +151,9 @@ class Plan:
         n, nd, rows = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
         _check(lib().trv_plan_info(h, ctypes.byref(n), ctypes.byref(nd), ctypes.byref(rows)), "trv_plan_info")
         self.n, self.ndims, self.rows = n.value, nd.value, rows.value
+        ns = ctypes.c_int32()
+        _check(lib().trv_plan_slices(h, ctypes.byref(ns)), "trv_plan_slices")
+        self.nslices = ns.value
 
     def destroy(self):
         if getattr(self, "_h", None):

@@ -91,11 +91,17 @@ trv_status_t trv_plan_info(trv_plan_t plan, int32_t* n, int32_t* ndims, int32_t*
     return TRV_OK;
 }
 
+trv_status_t trv_plan_slices(trv_plan_t plan, int32_t* nslices) {
+    if (!plan || !nslices) return TRV_ERR_INVALID_ARG;
+    *nslices = plan->plan.nslices;
+    return TRV_OK;
+}
+
 trv_status_t trv_plan_step(trv_plan_t plan, int32_t c, int32_t row, int32_t* dim, int32_t* dist) {
     if (!plan) return TRV_ERR_INVALID_ARG;
     const Plan& p = plan->plan;
-    if (c < 0 || c >= p.ndims || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
-    const Step& s = p.steps[c][p.step_of_row(row)];
+    if (c < 0 || c >= p.nslices || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
+    const Step& s = p.steps[c][p.algo == TRV_ALGO_BUCKET ? 0 : p.step_of_row(row)];
     if (dim) *dim = s.dim;
     if (dist) *dist = s.dist;
     return TRV_OK;
@@ -104,8 +110,8 @@ trv_status_t trv_plan_step(trv_plan_t plan, int32_t c, int32_t row, int32_t* dim
 trv_status_t trv_plan_peers(trv_plan_t plan, int32_t c, int32_t row, int32_t* peers) {
     if (!plan || !peers) return TRV_ERR_INVALID_ARG;
     const Plan& p = plan->plan;
-    if (c < 0 || c >= p.ndims || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
-    const Step& s = p.steps[c][p.step_of_row(row)];
+    if (c < 0 || c >= p.nslices || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
+    const Step& s = p.steps[c][p.algo == TRV_ALGO_BUCKET ? 0 : p.step_of_row(row)];
     for (int r = 0; r < p.n; ++r) {
         int peer[2], dir[2], hops[2];
         send_peers(p, r, s.dim, s.dist, peer, dir, hops);
@@ -118,7 +124,7 @@ trv_status_t trv_plan_peers(trv_plan_t plan, int32_t c, int32_t row, int32_t* pe
 trv_status_t trv_plan_send_set(trv_plan_t plan, int32_t c, int32_t step, int32_t dst, uint8_t* set) {
     if (!plan || !set) return TRV_ERR_INVALID_ARG;
     const Plan& p = plan->plan;
-    if (c < 0 || c >= p.ndims || step < 0 || step >= p.S || dst < 0 || dst >= p.n) return TRV_ERR_INVALID_ARG;
+    if (c < 0 || c >= p.nslices || step < 0 || step >= p.S || dst < 0 || dst >= p.n) return TRV_ERR_INVALID_ARG;
     for (int j = 0; j < p.n; ++j)
         set[j] = p.general ? (uint8_t)general_recv_mask(p, step, dst, j) : (in_send_set(p, c, step, dst, j) ? 1 : 0);
     return TRV_OK;
@@ -127,8 +133,8 @@ trv_status_t trv_plan_send_set(trv_plan_t plan, int32_t c, int32_t step, int32_t
 trv_status_t trv_plan_block_bounds(trv_plan_t plan, size_t count, int32_t c, int64_t* bounds) {
     if (!plan || !bounds) return TRV_ERR_INVALID_ARG;
     const Plan& p = plan->plan;
-    if (c < 0 || c >= p.ndims) return TRV_ERR_INVALID_ARG;
-    const int64_t lo = slice_lo((int64_t)count, p.ndims, c), hi = slice_lo((int64_t)count, p.ndims, c + 1);
+    if (c < 0 || c >= p.nslices) return TRV_ERR_INVALID_ARG;
+    const int64_t lo = slice_lo((int64_t)count, p.nslices, c), hi = slice_lo((int64_t)count, p.nslices, c + 1);
     for (int j = 0; j <= p.n; ++j) bounds[j] = block_lo(lo, hi, p.n, j);
     return TRV_OK;
 }
@@ -137,7 +143,7 @@ trv_status_t trv_plan_message_bytes(trv_plan_t plan, size_t count, size_t elem_s
                                     int64_t* bytes) {
     if (!plan || !bytes || elem_size == 0) return TRV_ERR_INVALID_ARG;
     const Plan& p = plan->plan;
-    if (c < 0 || c >= p.ndims || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
+    if (c < 0 || c >= p.nslices || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
     if (p.general) return TRV_ERR_UNSUPPORTED;
     message_bytes(p, (int64_t)count, (int64_t)elem_size, c, row, bytes);
     return TRV_OK;
@@ -147,7 +153,7 @@ trv_status_t trv_plan_message_bytes_side(trv_plan_t plan, size_t count, size_t e
                                          int32_t side, int64_t* bytes) {
     if (!plan || !bytes || elem_size == 0 || side < 0 || side > 1) return TRV_ERR_INVALID_ARG;
     const Plan& p = plan->plan;
-    if (c < 0 || c >= p.ndims || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
+    if (c < 0 || c >= p.nslices || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
     message_bytes_side(p, (int64_t)count, (int64_t)elem_size, c, row, side, bytes);
     return TRV_OK;
 }
@@ -289,7 +295,7 @@ trv_status_t trv_cost_model(trv_plan_t plan, size_t count, size_t elem_size, dou
     trv_status_t st = run_link_loads(p, count, elem_size, nullptr, nullptr, nullptr, max_bytes.data());
     if (st != TRV_OK) return st;
     // bytes every node sends: both of its messages in every row of every collective
-    for (int c = 0; c < D; ++c)
+    for (int c = 0; c < p.nslices; ++c)
         for (int row = 0; row < T; ++row)
             for (int side = 0; side < 2; ++side) {
                 message_bytes_side(p, (int64_t)count, (int64_t)elem_size, c, row, side, mb.data());

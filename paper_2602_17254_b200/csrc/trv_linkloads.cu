@@ -18,8 +18,9 @@ struct MsgClass {
     int dir;        // +1 / -1
     int hops;       // links crossed
     int delta;      // destination = source + delta (ring positions, wraps)
-    int filter;     // 0: every source sends; 1: sources with (pos & bit) == 0; 2: (pos & bit) != 0
-    int bit;
+    int filter;     // 0: every source sends; 1: sources with (q & bit) == 0; 2: (q & bit) != 0, where q = pos,
+    int bit;        //    or q = (size - pos) % size when `backwards` is set (a mirrored Recursive Doubling)
+    int backwards;
     int plane;      // which of the two per-source weight arrays: bytes sent to the first / second peer
 };
 struct RowSlice {
@@ -41,17 +42,17 @@ __device__ __forceinline__ long long warp_scan_incl(long long v, int lane) {
 
 // grid: (rings of the row's dimension, slices, rows); block: one warp
 __global__ void __launch_bounds__(32) k_link_tally(const RowSlice* __restrict__ desc, const long long* __restrict__ mbytes,
-                                                   int n, int D, int* __restrict__ msgs, long long* __restrict__ bytes) {
+                                                   int n, int D, int NS, int* __restrict__ msgs, long long* __restrict__ bytes) {
     __shared__ long long P[kMaxRing];   // inclusive prefix of bytes by source position
     __shared__ int C[kMaxRing];         // inclusive prefix of message counts
     const int lane = threadIdx.x, c = blockIdx.y, row = blockIdx.z;
-    const RowSlice rs = desc[row * D + c];
+    const RowSlice rs = desc[row * NS + c];
     const int a = rs.size;
     if ((int)blockIdx.x >= n / a) return;
     // ring number -> rank of its position 0
     const int q = blockIdx.x;
     const int base = (q % rs.stride) + (q / rs.stride) * rs.stride * a;
-    const long long* w0 = mbytes + ((size_t)row * D + c) * 2 * n;
+    const long long* w0 = mbytes + ((size_t)row * NS + c) * 2 * n;
 
     for (int k = 0; k < rs.nclass; ++k) {
         const MsgClass mc = rs.cls[k];
@@ -63,7 +64,8 @@ __global__ void __launch_bounds__(32) k_link_tally(const RowSlice* __restrict__ 
             long long wt = 0;
             int cnt = 0;
             if (s < a) {
-                const bool sends = mc.filter == 0 || (mc.filter == 1 ? (s & mc.bit) == 0 : (s & mc.bit) != 0);
+                const int q = mc.backwards ? (a - s) % a : s;
+                const bool sends = mc.filter == 0 || (mc.filter == 1 ? (q & mc.bit) == 0 : (q & mc.bit) != 0);
                 if (sends) {
                     wt = w[base + s * rs.stride];
                     cnt = 1;
@@ -130,19 +132,20 @@ __global__ void __launch_bounds__(256) k_link_max(const int* __restrict__ msgs, 
 
 trv_status_t run_link_loads(const Plan& p, size_t count, size_t elem_size, int32_t* msgs, int64_t* bytes,
                             int32_t* max_msgs, int64_t* max_bytes) {
-    const int n = p.n, D = p.ndims, T = p.rows();
+    const int n = p.n, D = p.ndims, NS = p.nslices, T = p.rows();
     const size_t links = (size_t)n * D * 2;
-    std::vector<RowSlice> desc((size_t)T * D);
-    std::vector<long long> mb((size_t)T * D * 2 * n);   // [row][slice][peer number][source rank]
+    std::vector<RowSlice> desc((size_t)T * NS);
+    std::vector<long long> mb((size_t)T * NS * 2 * n);  // [row][slice][peer number][source rank]
     int max_rings = 1;
     for (int row = 0; row < T; ++row) {
-        for (int c = 0; c < D; ++c) {
-            const Step& st = p.steps[c][p.step_of_row(row)];
-            RowSlice& rs = desc[(size_t)row * D + c];
+        for (int c = 0; c < NS; ++c) {
+            const Step& st = p.steps[c][p.algo == TRV_ALGO_BUCKET ? 0 : p.step_of_row(row)];
+            RowSlice& rs = desc[(size_t)row * NS + c];
             rs.dim = st.dim; rs.stride = p.stride[st.dim]; rs.size = p.dims[st.dim];
             if (rs.size > kMaxRing) return TRV_ERR_UNSUPPORTED;
             if (n / rs.size > max_rings) max_rings = n / rs.size;
             const int d = st.dist;
+            const int sg = d < 0 ? -1 : 1, ad = d < 0 ? -d : d;       // comparators: negative = mirrored collective
             if (p.general) {
                 // a direction in which no block travels in this step carries no message at all
                 const int t = p.step_of_row(row);
@@ -150,25 +153,33 @@ trv_status_t run_link_loads(const Plan& p, size_t count, size_t elem_size, int32
                 for (int o = 1; o < n; ++o)
                     if (p.gstep[o] == t) any[(row < p.S) == (p.gsgn[o] > 0) ? 1 : 0] = true;
                 rs.nclass = 0;
-                if (any[0]) rs.cls[rs.nclass++] = MsgClass{-1, d, -d, 0, 0, 0};
-                if (any[1]) rs.cls[rs.nclass++] = MsgClass{+1, d, +d, 0, 0, 1};
+                if (any[0]) rs.cls[rs.nclass++] = MsgClass{-1, d, -d, 0, 0, 0, 0};
+                if (any[1]) rs.cls[rs.nclass++] = MsgClass{+1, d, +d, 0, 0, 0, 1};
             } else if (p.algo == TRV_ALGO_TRIVANCE) {
                 rs.nclass = 2;
-                rs.cls[0] = MsgClass{-1, d, -d, 0, 0, 0};
-                rs.cls[1] = MsgClass{+1, d, +d, 0, 0, 1};
+                rs.cls[0] = MsgClass{-1, d, -d, 0, 0, 0, 0};
+                rs.cls[1] = MsgClass{+1, d, +d, 0, 0, 0, 1};
             } else if (p.algo == TRV_ALGO_BRUCK) {
                 rs.nclass = 2;
-                rs.cls[0] = MsgClass{+1, d, d, 0, 0, 0};
-                rs.cls[1] = MsgClass{+1, 2 * d, 2 * d, 0, 0, 1};
+                rs.cls[0] = MsgClass{sg, ad, d, 0, 0, 0, 0};
+                rs.cls[1] = MsgClass{sg, 2 * ad, 2 * d, 0, 0, 0, 1};
+            } else if (p.algo == TRV_ALGO_SWING) {
+                // even positions send to pos + d, odd ones to pos - d, each the short way round
+                rs.nclass = 2;
+                rs.cls[0] = MsgClass{sg, ad, d, 1, 1, 0, 0};
+                rs.cls[1] = MsgClass{-sg, ad, -d, 2, 1, 0, 0};
+            } else if (p.algo == TRV_ALGO_BUCKET) {
+                rs.nclass = 1;
+                rs.cls[0] = MsgClass{sg, 1, sg, 0, 0, 0, 0};
             } else {
                 rs.nclass = 2;
-                rs.cls[0] = MsgClass{+1, d, +d, 1, d, 0};
-                rs.cls[1] = MsgClass{-1, d, -d, 2, d, 0};
+                rs.cls[0] = MsgClass{sg, ad, d, 1, ad, sg < 0 ? 1 : 0, 0};
+                rs.cls[1] = MsgClass{-sg, ad, -d, 2, ad, sg < 0 ? 1 : 0, 0};
             }
             static_assert(sizeof(long long) == sizeof(int64_t), "int64");
             for (int side = 0; side < 2; ++side)
                 message_bytes_side(p, (int64_t)count, (int64_t)elem_size, c, row, side,
-                                   (int64_t*)&mb[(((size_t)row * D + c) * 2 + side) * n]);
+                                   (int64_t*)&mb[(((size_t)row * NS + c) * 2 + side) * n]);
         }
     }
 
@@ -193,8 +204,8 @@ trv_status_t run_link_loads(const Plan& p, size_t count, size_t elem_size, int32
         ok(cudaMemset(d_bytes, 0, (size_t)T * links * sizeof(long long)));
     }
     if (st == TRV_OK) {
-        dim3 grid(max_rings, D, T);
-        TRV_LAUNCH(k_link_tally, grid, 32, 0, 0, d_desc, d_mb, n, D, d_msgs, d_bytes);
+        dim3 grid(max_rings, NS, T);
+        TRV_LAUNCH(k_link_tally, grid, 32, 0, 0, d_desc, d_mb, n, D, NS, d_msgs, d_bytes);
         TRV_LAUNCH(k_link_max, T, 256, 0, 0, d_msgs, d_bytes, (int)links, d_maxm, d_maxb);
         ok(cudaGetLastError());
         if (msgs) ok(cudaMemcpy(msgs, d_msgs, (size_t)T * links * sizeof(int), cudaMemcpyDeviceToHost));

@@ -16,6 +16,9 @@ struct Step {
 // What a fused kernel needs to know about one collective (slice).
 struct Plan {
     int algo = 0, variant = 0, ndims = 0, n = 0, S = 0, base = 3;
+    // concurrent collectives: ndims, or 2 * ndims for a comparator with its mirrored sub-collective
+    // (Sec. 2.4); the steps of a mirrored slice carry negated distances
+    int nslices = 0;
     int dims[TRV_MAX_DIMS] = {0};
     int stride[TRV_MAX_DIMS] = {0};     // rank = sum_d x_d * stride[d]
     int sdim[TRV_MAX_DIMS] = {0};       // steps in dimension d = log_base a_d
@@ -25,6 +28,11 @@ struct Plan {
     // mod[c][t][d] = base^(number of steps <= t of collective c that ran along d): block j is in
     // the message to p at step t iff j_d == p_d (mod mod[c][t][d]) for every d  (closed form Pi)
     std::vector<std::vector<std::vector<int>>> mod;
+
+    // Swing (Sec. 2.4) has no congruence form: reach[c][t][p] = bitset of the blocks rank p still
+    // answers for after Reduce-Scatter step t - 1 (its own and all it will forward), t = 0 .. S
+    std::vector<std::vector<std::vector<uint64_t>>> reach;
+    int words = 0;      // 64-bit words per bitset
 
     // Rings whose size is no power of three (Sec. 4.4), bandwidth-optimal form only.  The tree a
     // block follows is the same for every block up to rotation, so it is stored once, by the

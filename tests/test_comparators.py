@@ -1,0 +1,166 @@
+"""Comparator schedules of Sec. 2.4 as link-load models: Swing, Bucket (ring), and the mirrored
+sub-collectives.  Pins of the oracle against Sec. 2.4, Table 1 and App. B; the library's host-side
+tables against the oracle.  No GPU needed."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2602_17254_b200 import binding
+
+LAT, BW = oracle.VARIANT_LATENCY, oracle.VARIANT_BANDWIDTH
+M = oracle.ALGO_MIRROR
+
+
+def rho(k):
+    return (1 - (-2) ** (k + 1)) // 3
+
+
+def test_golden_per_step_congestion():
+    """tests/golden/table1_ring_comparators.txt: the per-step congestion App. B derives for each comparator."""
+    import os
+    algo = {"swing_latency": (oracle.ALGO_SWING, LAT), "swing_bandwidth_mirrored": (oracle.ALGO_SWING | M, BW),
+            "recursive_doubling_latency": (oracle.ALGO_RECDOUB, LAT)}
+    path = os.path.join(os.path.dirname(__file__), "golden", "table1_ring_comparators.txt")
+    rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 6
+    for name, n, *want in rows:
+        a, variant = algo[name]
+        ll = oracle.link_loads([int(n)], variant, 64 * int(n), 4, algo=a)
+        assert ll["max_msgs"][:len(want)].tolist() == [int(v) for v in want]
+
+
+def test_swing_distances_and_pairs():
+    """rho(k) = sum_{i<=k} (-2)^i = 1, -1, 3, -5, 11, ...; even ranks go to r + rho, odd ones to r - rho; the
+    exchange is pairwise (Sec. 2.4)."""
+    assert [rho(k) for k in range(6)] == [1, -1, 3, -5, 11, -21]
+    for n in (2, 8, 64, 256):
+        q = int(math.log2(n))
+        assert oracle.step_list([n], 0, oracle.ALGO_SWING) == [(0, rho(k)) for k in range(q)]
+        for k in range(q):
+            pe = oracle.peers([n], k, 0, oracle.ALGO_SWING)[:, 0]
+            for r in range(n):
+                assert pe[r] == (r + rho(k) if r % 2 == 0 else r - rho(k)) % n
+                assert pe[pe[r]] == r
+
+
+@pytest.mark.parametrize("n", [8, 16, 64, 256, 1024])
+def test_swing_congestion_matches_appendix_b(n):
+    """App. B: latency-optimal Swing has congestion ceil(|rho(k)| / 2) in step k; with the mirrored collective
+    the bandwidth-optimal one has |rho(k)| at message size m / 2^(k+2) per collective."""
+    q = int(math.log2(n))
+    ll = oracle.link_loads([n], LAT, 1024, 4, algo=oracle.ALGO_SWING)
+    assert ll["max_msgs"].tolist() == [math.ceil(abs(rho(k)) / 2) for k in range(q)]
+    E = 64 * n
+    ll = oracle.link_loads([n], BW, E, 4, algo=oracle.ALGO_SWING | M)
+    want = [abs(rho(k)) for k in range(q)]
+    assert ll["max_msgs"].tolist() == want + want[::-1]
+    m = 4 * E
+    assert ll["max_bytes"].tolist() == [abs(rho(k)) * (m // 2) // 2 ** (k + 1) for k in range(q)] + \
+        [abs(rho(k)) * (m // 2) // 2 ** (k + 1) for k in reversed(range(q))]
+    cm = oracle.cost_model([n], BW, E, 4, 0.0, 1.0, algo=oracle.ALGO_SWING | M)
+    theta = sum(abs(rho(k)) / 2 ** (k + 1) for k in range(q))
+    assert np.isclose(cm["theta"], theta, rtol=1e-12)
+    assert abs(theta - q / 3) < 0.45                      # Table 1: (1/3) log2 n, up to the constant the sum converges with
+    assert np.isclose(cm["delta"], (n - 1) / n) and np.isclose(cm["lambda"], 2 * q / (math.log(n) / math.log(3)))
+
+
+@pytest.mark.parametrize("n", [8, 64])
+def test_swing_block_sets_partition(n):
+    """Algorithm 1 on Swing's peers: n / 2^(k+1) blocks go out in step k and what a rank sends over all
+    steps plus its own block is everything, each block once (bandwidth optimality, Sec. 2.3)."""
+    q = int(math.log2(n))
+    for r in (0, 1, n // 2 + 1):
+        seen = np.zeros(n, int)
+        seen[r] += 1
+        for k in range(q):
+            p = oracle.peers([n], k, 0, oracle.ALGO_SWING)[r, 0]
+            s = oracle.send_set([n], p, k, 0, oracle.ALGO_SWING)
+            assert s.sum() == n // 2 ** (k + 1)
+            seen += s
+        assert (seen == 1).all()
+
+
+@pytest.mark.parametrize("n", [2, 7, 9, 32, 100])
+def test_bucket_ring_matches_table_1(n):
+    """The ring algorithm with both ports (Table 1, App. B): 2(n-1) steps, no two messages share a link,
+    every message one block of one half: Delta = Theta = (n-1)/n -> 1, Lambda = 2(n-1)/log3 n."""
+    E = 6 * n
+    ll = oracle.link_loads([n], BW, E, 4, algo=oracle.ALGO_BUCKET | M)
+    assert ll["msgs"].shape == (2 * (n - 1), n, 1, 2)
+    assert (ll["msgs"] == 1).all() and (ll["bytes"] == 4 * 3).all()
+    cm = oracle.cost_model([n], BW, E, 4, 0.0, 1.0, algo=oracle.ALGO_BUCKET | M)
+    assert cm["steps"] == 2 * (n - 1)
+    assert np.isclose(cm["theta"], (n - 1) / n) and np.isclose(cm["delta"], (n - 1) / n)
+    assert np.isclose(cm["lambda"], 2 * (n - 1) / (math.log(n) / math.log(3)))
+    one = oracle.link_loads([n], BW, E, 4, algo=oracle.ALGO_BUCKET)      # one port only: + links carry it all
+    assert (one["msgs"][..., 0] == 1).all() and (one["msgs"][..., 1] == 0).all()
+    with pytest.raises(oracle.OracleError):
+        oracle.link_loads([n], LAT, E, 4, algo=oracle.ALGO_BUCKET)
+
+
+@pytest.mark.parametrize("n", [8, 64, 256])
+def test_recursive_doubling_mirrored(n):
+    """Both ports through a mirrored collective (Sec. 2.4): the bytes per node halve per collective
+    (Delta = (n-1)/n).  On the links the two collectives overlap: the literal tally finds 2^(k+1) - 1
+    half-size messages on the worst link of step k, where Table 1 / App. B count one collective's 2^k
+    (the table's (1/2) log2 n) -- recorded here as it is tallied."""
+    q = int(math.log2(n))
+    E = 64 * n
+    ll = oracle.link_loads([n], BW, E, 4, algo=oracle.ALGO_RECDOUB | M)
+    want = [2 ** (k + 1) - 1 for k in range(q)]
+    assert ll["max_msgs"].tolist() == want + want[::-1]
+    cm = oracle.cost_model([n], BW, E, 4, 0.0, 1.0, algo=oracle.ALGO_RECDOUB | M)
+    assert np.isclose(cm["delta"], (n - 1) / n)
+    single = oracle.cost_model([n], BW, E, 4, 0.0, 1.0, algo=oracle.ALGO_RECDOUB)
+    assert np.isclose(single["theta"], q)                 # one collective on the whole vector: 2 * q * 2^k / 2^(k+1)
+    assert q / 2 < cm["theta"] < q
+
+
+# ------------------------------------------------------------------ the library's host-side tables
+
+CASES = [((8,), oracle.ALGO_SWING), ((64,), oracle.ALGO_SWING), ((64,), oracle.ALGO_SWING | M), ((16,), oracle.ALGO_RECDOUB | M),
+         ((27,), oracle.ALGO_BRUCK | M), ((9,), oracle.ALGO_BUCKET), ((10,), oracle.ALGO_BUCKET | M)]
+
+
+@pytest.mark.parametrize("dims,algo", CASES)
+@pytest.mark.parametrize("variant", [LAT, BW])
+def test_plan_tables_match_oracle(dims, algo, variant):
+    base = algo & ~M
+    if base == oracle.ALGO_BUCKET and variant == LAT:
+        with pytest.raises(binding.TrivanceError) as e:
+            binding.Plan(dims, variant, algo)
+        assert e.value.status == binding.ERR_UNSUPPORTED
+        return
+    plan = binding.Plan(dims, variant, algo)
+    n = plan.n
+    assert plan.nslices == (2 if algo & M else 1)
+    E = 37 * n + 5
+    sent = np.zeros(n, np.int64)
+    for c in range(plan.nslices):
+        for row in range(plan.rows):
+            for side in (0, 1):
+                sent += plan.message_bytes_side(E, 4, c, row, side)
+    assert np.array_equal(sent, oracle.bytes_sent(dims, variant, E, 4, algo=algo))
+    if base != oracle.ALGO_BUCKET:
+        _, S = oracle.num_steps(dims, algo)
+        for c in range(plan.nslices):
+            steps = oracle.step_list(dims, c, algo)
+            for t in range(S):
+                assert plan.step(c, t) == steps[t]
+                assert np.array_equal(plan.peers(c, t), oracle.peers(dims, t, c, algo))
+                if variant == BW:
+                    for dst in (0, 1, n - 1):
+                        assert np.array_equal(plan.send_set(c, t, dst), oracle.send_set(dims, dst, t, c, algo))
+    plan.destroy()
+
+
+def test_mirror_flag_is_for_ring_comparators_only():
+    for dims, algo in (((9,), oracle.ALGO_TRIVANCE | M), ((9, 9), oracle.ALGO_BRUCK | M)):
+        with pytest.raises(binding.TrivanceError) as e:
+            binding.Plan(dims, BW, algo)
+        assert e.value.status == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.TrivanceError) as e:
+        binding.Plan((12,), BW, oracle.ALGO_SWING)
+    assert e.value.status == binding.ERR_UNDEFINED_SCHEDULE

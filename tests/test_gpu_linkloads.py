@@ -88,3 +88,30 @@ def test_cost_model_matches_oracle(dims, algo, variant):
         for name, key in [("latency_term", "latency_term"), ("tx_term", "tx_term"), ("total", "total"), ("lambda_", "lambda"),
                           ("delta", "delta"), ("theta", "theta")]:
             assert np.isclose(getattr(got, name), want[key], rtol=1e-12, atol=0), name
+
+
+M = binding.ALGO_MIRRORED
+NEW = [((8,), binding.ALGO_SWING), ((64,), binding.ALGO_SWING), ((1024,), binding.ALGO_SWING), ((64,), binding.ALGO_SWING | M),
+       ((256,), binding.ALGO_SWING | M), ((16,), binding.ALGO_RECDOUB | M), ((512,), binding.ALGO_RECDOUB | M),
+       ((27,), binding.ALGO_BRUCK | M), ((9,), binding.ALGO_BUCKET), ((10,), binding.ALGO_BUCKET | M),
+       ((100,), binding.ALGO_BUCKET | M), ((2,), binding.ALGO_BUCKET | M)]
+
+
+@pytest.mark.parametrize("dims,algo", NEW)
+@pytest.mark.parametrize("variant", [LAT, BW])
+def test_swing_bucket_and_mirrored_link_loads(dims, algo, variant):
+    """Swing, the ring algorithm and the mirrored sub-collectives (Sec. 2.4): tally vs the oracle's walk."""
+    if (algo & ~M) == binding.ALGO_BUCKET and variant == LAT:     # the ring algorithm has no latency-optimal form
+        with pytest.raises(binding.TrivanceError) as e:
+            binding.Plan(dims, variant, algo)
+        assert e.value.status == binding.ERR_UNSUPPORTED
+        return
+    for count in (100003, 7):
+        got = binding.Plan(dims, variant, algo).link_loads(count, 4)
+        _same(got, oracle.link_loads(dims, variant, count, 4, algo=algo))
+    alpha, beta = 1.5e-6, 1.0 / 100e9
+    got = binding.Plan(dims, variant, algo).cost_model(100003, 4, alpha, beta)
+    want = oracle.cost_model(dims, variant, 100003, 4, alpha, beta, algo=algo)
+    assert got.steps == want["steps"] and got.bytes_sent_per_node == want["bytes_sent_per_node"] and got.tx_bytes == want["tx_bytes"]
+    for name, key in [("total", "total"), ("lambda_", "lambda"), ("delta", "delta"), ("theta", "theta")]:
+        assert np.isclose(getattr(got, name), want[key], rtol=1e-12, atol=0), name
