@@ -19,8 +19,11 @@
  *     collective on a different dimension in every step (Sec. 5);
  *   - congestion c_k = number of messages sharing a link in a step under
  *     deterministic shortest-path routing inside one dimension (Sec. 2.1,
- *     Fig. 1, App. E); Bruck-style and Recursive-Doubling schedules only as
- *     link-load comparators (Sec. 2.4, Fig. 1).
+ *     Fig. 1, App. E); Bruck-style, Recursive-Doubling, Swing and ring (Bucket)
+ *     schedules, each optionally with its mirrored sub-collective, only as
+ *     link-load comparators (Sec. 2.4, Fig. 1, Table 1, App. B);
+ *   - rings whose size is no power of three, bandwidth-optimal form (Sec. 4.4):
+ *     see the block of comments in front of gen_steps().
  *
  * Readings where the paper is silent (each also listed in the design notes):
  *   - a joint reduction adds as (from_left + own) + from_right, where "left"
@@ -36,6 +39,14 @@
  *     the paper beyond "collective 0 starts horizontal, collective 1 vertical
  *     and they swap every step" (Sec. 5).
  *   - int32 addition wraps modulo 2^32.
+ *   - the mirrored sub-collective of a comparator (Sec. 2.4) is the same pattern with every
+ *     displacement and direction of travel reversed, on the second half of the vector; for
+ *     Recursive Doubling that is the XOR pattern on the ring counted backwards (r -> -r mod n).
+ *     PARITY UNPINNED by the paper for Recursive Doubling (App. B counts one collective's
+ *     congestion there); for Swing and the ring algorithm App. B's per-step congestion pins it.
+ *   - the ring (Bucket) algorithm sends block (r - t - 1) mod n in Reduce-Scatter step t and block
+ *     (r - t) mod n in AllGather step t, always to r + 1: block j ends at node j.  Any such
+ *     numbering gives the same loads when the blocks have equal length.
  *
  * Floating point: binary32 (or binary64 for the error-bound checks), one add
  * at a time, no contraction, no reassociation.  Compile with
