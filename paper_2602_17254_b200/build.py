@@ -12,7 +12,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtrivance.so")
 OBJ = os.path.join(HERE, "build")
 
-SOURCES = ["trv_plan.cc", "trv_api.cu", "trv_step.cu", "trv_step_gen.cu", "trv_fused_lat.cu", "trv_fused_t999.cu", "trv_fused_lines.cu", "trv_fused_bw.cu", "trv_fused_tree.cu", "trv_pipe.cu", "trv_linkloads.cu", "trv_noalloc.cu"]
+SOURCES = ["trv_plan.cc", "trv_api.cu", "trv_step.cu", "trv_step_gen.cu", "trv_fused_lat.cu", "trv_fused_t999.cu", "trv_fused_t999_tma.cu", "trv_fused_lines.cu", "trv_fused_bw.cu", "trv_fused_tree.cu", "trv_pipe.cu", "trv_linkloads.cu", "trv_noalloc.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

@@ -210,6 +210,9 @@ static trv_status_t lat_fused_launch(const Call& c, const Addr& in, const Addr& 
             }
         }
     } else if (kind == LatKind::T999) {
+        // equally spaced rank buffers: the tile arrives by TMA; else per-thread loads
+        trv_status_t st = TRV_OK;
+        if (run_fused_t999_tma(c, a, &st)) return st;
         g_last_kernel = "lat_t999";
         return run_fused_t999(c, a);
     } else if (kind == LatKind::Lines) {
