@@ -234,6 +234,12 @@ size_t trv_noalloc_max_scratch_bytes(void);
 trv_status_t trv_pipeline_status(const void *scratch, void *cuda_stream);
 trv_status_t trv_pipeline_selftest_timeout(void *scratch, size_t scratch_bytes, void *cuda_stream);
 
+/* Some fused kernels fetch their tile by TMA and wait for it on an mbarrier; that wait is bounded.
+ * A thread block whose wait runs out stores nothing and adds one to a per-device counter.
+ * trv_tma_giveups reads that counter for the current device (a synchronous copy): 0 in every correct
+ * run; anything else means outputs of earlier calls are incomplete.  TRV_ERR_CUDA if it cannot be read. */
+trv_status_t trv_tma_giveups(uint32_t *count);
+
 /* ---------------------------------------------------------------- link loads
  *
  * Per-step, per-directed-link load of the plan's schedule (Sec. 2.1: c_k = number of

@@ -30,7 +30,7 @@ SYMBOLS = [
     "trv_kernel_supported", "trv_allreduce_ex", "trv_allreduce_host", "trv_host_workspace_bytes",
     "trv_link_loads", "trv_plan_message_bytes", "trv_plan_message_bytes_side", "trv_strerror", "trv_launch_count", "trv_last_kernel_name",
     "trv_allreduce_noalloc", "trv_noalloc_max_scratch_bytes", "trv_cost_model", "trv_pipeline_status",
-    "trv_pipeline_selftest_timeout",
+    "trv_pipeline_selftest_timeout", "trv_tma_giveups",
 ]
 
 
@@ -108,6 +108,13 @@ def pipeline_status(scratch_ptr, stream=0):
 
 def pipeline_selftest_timeout(scratch_ptr, scratch_bytes, stream=0):
     _check(lib().trv_pipeline_selftest_timeout(scratch_ptr, scratch_bytes, stream), "trv_pipeline_selftest_timeout")
+
+
+def tma_giveups():
+    """Thread blocks of TMA-fed kernels that gave up waiting for their tile on the current device (0 in a correct run)."""
+    v = ctypes.c_uint32()
+    _check(lib().trv_tma_giveups(ctypes.byref(v)), "trv_tma_giveups")
+    return v.value
 
 
 def launch_count():

@@ -5,6 +5,7 @@
 #include <vector>
 
 #include "trv_dev.cuh"
+#include "trv_tma.cuh"
 
 namespace trv {
 std::atomic<uint64_t> g_launches{0};
@@ -268,6 +269,14 @@ trv_status_t trv_allreduce_host(trv_plan_t plan, const void* const* host_in, voi
     if (st != TRV_OK) return st;
     for (int r = 0; r < p.n; ++r)
         if (cudaMemcpyAsync(host_out[r], dev[r], count * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return TRV_ERR_CUDA;
+    return TRV_OK;
+}
+
+trv_status_t trv_tma_giveups(uint32_t* count) {
+    if (!count) return TRV_ERR_INVALID_ARG;
+    const unsigned v = tma_giveups();
+    if (v == ~0u) return TRV_ERR_CUDA;
+    *count = v;
     return TRV_OK;
 }
 

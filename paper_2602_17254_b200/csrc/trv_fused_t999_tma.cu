@@ -6,11 +6,10 @@
 // at a time, and group 1 runs on shared memory like the other two.  Needs equally spaced rank buffers
 // (one tensor map describes them as a [729][count] matrix); other callers keep k_lat_t999.
 // The wait on the copy's mbarrier is bounded; a waiter that gives up counts it in a device-side
-// counter (t999_tma_giveups) and the CTA leaves without storing.
-#include <cuda.h>
-
+// counter (trv_tma.cuh) and the CTA leaves without storing.
 #include "trv_dev.cuh"
 #include "trv_fused_lat.cuh"
+#include "trv_tma.cuh"
 
 namespace trv {
 
@@ -22,8 +21,6 @@ struct RotT {
     static constexpr int sB = ROT == 0 ? 9 : (ROT == 1 ? 81 : 1);
     static constexpr int sC = ROT == 0 ? 81 : (ROT == 1 ? 1 : 9);
 };
-
-__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
 
 template <typename T, int ROT, bool FULL, typename Addr>
 __device__ __forceinline__ void t999_tma_body(const Addr& out, const LatArgs& a, T* slab, long long t0) {
@@ -92,44 +89,17 @@ __device__ __forceinline__ void t999_tma_body(const Addr& out, const LatArgs& a,
 }
 
 constexpr unsigned kTmaTileBytes = 729 * 32 * 4;
-constexpr unsigned kTmaWaitLimit = 1u << 22;    // try_wait polls (each suspends for a while): far beyond any real copy
 
 template <typename T>
-__global__ void __launch_bounds__(288, 2) k_lat_t999_tma(const __grid_constant__ CUtensorMap tmap, StrideAddr out, LatArgs a) {
+__global__ void __launch_bounds__(288, 2) k_lat_t999_tma(const __grid_constant__ CUtensorMap tmap, StrideAddr out, LatArgs a,
+                                                         unsigned* giveups) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     T* slab = reinterpret_cast<T*>(smem_raw);                           // [729][32]
     unsigned long long* bar = reinterpret_cast<unsigned long long*>(smem_raw + kTmaTileBytes);
     const int c = blockIdx.y;                                           // everything below is CTA-uniform
     const long long t0 = (a.lo[c] & ~31LL) + (long long)blockIdx.x * 32;
     if (t0 >= a.hi[c]) return;
-    const unsigned bar_s = smem_u32(bar), slab_s = smem_u32(slab);
-    if (threadIdx.x == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_s), "r"(1) : "memory");
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s), "r"(kTmaTileBytes) : "memory");
-#pragma unroll
-        for (int b = 0; b < 3; ++b)
-            asm volatile(
-                "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-                    slab_s + b * (243 * 32 * 4)),
-                "l"(&tmap), "r"((int)t0), "r"(243 * b), "r"(bar_s)
-                : "memory");
-    }
-    __syncthreads();                    // the barrier is initialised before anybody polls it
-    unsigned done = 0;
-    for (unsigned spins = 0; spins < kTmaWaitLimit; ++spins) {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(bar_s), "r"(0)
-            : "memory");
-        if (done) break;
-    }
-    if (!__syncthreads_and((int)done)) {        // gave up: count it, leave without storing
-        if (threadIdx.x == 0) atomicAdd(&g_tma_giveups, 1u);
-        return;
-    }
+    if (!tma_fetch_tile(&tmap, slab, bar, (int)t0, 3, 243, giveups)) return;     // gave up: counted, nothing stored
     const bool full = t0 >= a.lo[c] && t0 + 32 <= a.hi[c];
     if (c == 0) { if (full) t999_tma_body<T, 0, true>(out, a, slab, t0); else t999_tma_body<T, 0, false>(out, a, slab, t0); }
     else if (c == 1) { if (full) t999_tma_body<T, 1, true>(out, a, slab, t0); else t999_tma_body<T, 1, false>(out, a, slab, t0); }
@@ -155,21 +125,28 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
+bool tma_encode_ranks(const StrideAddr& in, int n, size_t count, int box_rows, CUtensorMap* out) {
+    if ((in.stride & 15) || ((uintptr_t)in.base & 15) || count == 0 || count >= ((size_t)1 << 31)) return false;
+    if (n > 1 && (size_t)in.stride < count * 4) return false;
+    if (box_rows < 1 || box_rows > 256 || n % box_rows) return false;
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint64_t gdim[2] = {(cuuint64_t)count, (cuuint64_t)n};
+    const cuuint64_t gstride[1] = {(cuuint64_t)(n > 1 ? in.stride : ((count * 4 + 15) & ~(size_t)15))};
+    const cuuint32_t box[2] = {32, (cuuint32_t)box_rows};
+    const cuuint32_t estride[2] = {1, 1};
+    return enc(out, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, in.base, gdim, gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // false: this call cannot use the TMA kernel (the caller falls back to k_lat_t999)
 bool run_fused_t999_tma(const Call& c, const LatArgs& a, trv_status_t* status) {
     StrideAddr sin, sout;
     if (!uniform_stride(c.in, 729, &sin) || !uniform_stride((const void* const*)c.out, 729, &sout)) return false;
-    if ((sin.stride & 15) || sin.stride < c.count * 4 || c.count >= ((size_t)1 << 31)) return false;
-    EncodeTiledFn enc = encode_tiled_fn();
-    if (!enc) return false;
     CUtensorMap tmap;
-    const cuuint64_t gdim[2] = {(cuuint64_t)c.count, 729};
-    const cuuint64_t gstride[1] = {(cuuint64_t)sin.stride};
-    const cuuint32_t box[2] = {32, 243};
-    const cuuint32_t estride[2] = {1, 1};
-    if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, sin.base, gdim, gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return false;
+    if (!tma_encode_ranks(sin, 729, c.count, 243, &tmap)) return false;
+    unsigned* giveups = tma_giveup_counter();
+    if (!giveups) return false;
     long long tiles_x = 0;
     for (int sl = 0; sl < 3; ++sl)
         if (a.hi[sl] > a.lo[sl]) {
@@ -183,16 +160,22 @@ bool run_fused_t999_tma(const Call& c, const LatArgs& a, trv_status_t* status) {
     g_last_kernel = "lat_t999_tma";
     if (c.dtype == TRV_FLOAT32) {
         if (!allow_big_smem(k_lat_t999_tma<float>, smem)) { *status = TRV_ERR_CUDA; return true; }
-        TRV_LAUNCH((k_lat_t999_tma<float>), dim3((unsigned)tiles_x, 3, 1), 288, smem, c.st, tmap, sout, a);
+        TRV_LAUNCH((k_lat_t999_tma<float>), dim3((unsigned)tiles_x, 3, 1), 288, smem, c.st, tmap, sout, a, giveups);
     } else {
         if (!allow_big_smem(k_lat_t999_tma<uint32_t>, smem)) { *status = TRV_ERR_CUDA; return true; }
-        TRV_LAUNCH((k_lat_t999_tma<uint32_t>), dim3((unsigned)tiles_x, 3, 1), 288, smem, c.st, tmap, sout, a);
+        TRV_LAUNCH((k_lat_t999_tma<uint32_t>), dim3((unsigned)tiles_x, 3, 1), 288, smem, c.st, tmap, sout, a, giveups);
     }
     if (cudaGetLastError() != cudaSuccess) *status = TRV_ERR_CUDA;
     return true;
 }
 
-unsigned t999_tma_giveups() {
+unsigned* tma_giveup_counter() {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_tma_giveups) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    return (unsigned*)p;
+}
+
+unsigned tma_giveups() {
     unsigned v = 0;
     if (cudaMemcpyFromSymbol(&v, g_tma_giveups, sizeof(v)) != cudaSuccess) return ~0u;
     return v;
