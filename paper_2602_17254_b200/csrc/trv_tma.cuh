@@ -1,7 +1,7 @@
 // Tile fetch by TMA for the fused latency kernels whose tile is 32 element columns x n ranks in
 // shared memory.  When the caller's rank buffers are equally spaced, one tensor map describes them as
 // an [n][count] matrix of 4-byte words; one thread of a CTA issues n / rows_per_box bulk tensor copies
-// (cp.async.bulk.tensor.2d, boxes of 32 columns x at most 243 ranks, no multicast) that complete on
+// (cp.async.bulk.tensor.2d, boxes of 32 columns x at most 243 ranks, each to this CTA alone) that complete on
 // an mbarrier, so the whole tile is in flight at once.  Columns beyond `count` arrive as zeros.
 // It pays where a thread would otherwise have few loads in flight (9x9x9: nine per thread, 10.1 -> 8.4 ms);
 // the line-group kernel, whose threads issue 27 or 81 loads at once, got slower with it (27x27: 0.60 -> 0.39
