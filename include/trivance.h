@@ -237,7 +237,10 @@ trv_status_t trv_pipeline_selftest_timeout(void *scratch, size_t scratch_bytes, 
 /* Some fused kernels fetch their tile by TMA and wait for it on an mbarrier; that wait is bounded.
  * A thread block whose wait runs out stores nothing and adds one to a per-device counter.
  * trv_tma_giveups reads that counter for the current device (a synchronous copy): 0 in every correct
- * run; anything else means outputs of earlier calls are incomplete.  TRV_ERR_CUDA if it cannot be read. */
+ * run; anything else means outputs of earlier calls are incomplete.  TRV_ERR_CUDA if it cannot be read.
+ * A call that uses such a kernel looks up the counter's device address (cudaGetSymbolAddress) and encodes a
+ * tensor map on the host; like the first call of trv_allreduce_noalloc, make the first such call on a device
+ * outside any stream capture.  If either step fails the call silently uses the kernel without TMA. */
 trv_status_t trv_tma_giveups(uint32_t *count);
 
 /* ---------------------------------------------------------------- link loads
