@@ -12,9 +12,9 @@
  *   - peers pi(r,k,n) = (r - 3^k, r + 3^k) mod n (Sec. 4.1);
  *   - latency-optimal form: log3 n steps, whole vector to both peers, joint
  *     reduction of the two received vectors with the local partial (Sec. 4.2);
- *   - bandwidth-optimal form: Reduce-Scatter over n blocks, block sets from
- *     the recursive BlockPropagation procedure (Algorithm 1, Sec. 4.3), then
- *     AllGather in reverse order (Sec. 4.1);
+ *   - bandwidth-optimal form: Reduce-Scatter over n blocks, block sets = the
+ *     sets BlockPropagation defines (Algorithm 1, Sec. 4.3), grown step by step
+ *     from the peers of each step, then AllGather in reverse order (Sec. 4.1);
  *   - D-dimensional tori: D collectives on 1/D of the vector each, every
  *     collective on a different dimension in every step (Sec. 5);
  *   - congestion c_k = number of messages sharing a link in a step under
@@ -25,7 +25,7 @@
  *   - rings whose size is no power of three, bandwidth-optimal form (Sec. 4.4):
  *     see the block of comments in front of gen_steps().
  *
- * Readings where the paper is silent (each also listed in the design notes):
+ * Readings where the paper is silent:
  *   - a joint reduction adds as (from_left + own) + from_right, where "left"
  *     is the peer r - 3^k.  PARITY UNPINNED by the paper: any fixed order
  *     satisfies every published fact; the tests pin it to this reading with an
@@ -187,18 +187,31 @@ static int send_peers(const orc_topo *tp, int r, int d, int dist, int *peer, int
     }
 }
 
-/* Algorithm 1 (BlockPropagation), generalised from the ring's pi(r,k,n) to the
- * step list of one collective: marks every rank reachable from r through the
- * steps step..S-1. */
+/* The set Algorithm 1 (BlockPropagation, Sec. 4.3) defines, computed in the oracle's own form:
+ * a block that rank r answers for at step `step` reaches, one step at a time, every rank that can
+ * be got to from r by hops taken in steps of strictly increasing number step <= k_1 < k_2 < ... < S.
+ * So the set grows step by step: the ranks known BEFORE step k (r itself and everything reached in
+ * steps step..k-1) each add their peers of step k.  blocks[] gets a 1 for every rank reached; r
+ * itself is a source only.  Generalised from the ring's pi(r,k,n) to one collective's step list. */
 static void block_propagation(const orc_topo *tp, const int *sdim, const int *sdist,
                               int r, int step, uint8_t *blocks) {
-    if (step >= tp->S) return;
+    int n = tp->n, nsrc = 1;
+    int *src = (int *)malloc(sizeof(int) * (size_t)n * 2);   /* sources so far, in the order they were reached */
+    uint8_t *seen = (uint8_t *)calloc((size_t)n, 1);
+    if (!src || !seen) { free(src); free(seen); return; }
+    src[0] = r; seen[r] = 1;
     for (int k = step; k < tp->S; ++k) {
-        int peer[2], dir[2], hops[2];
-        int np = send_peers(tp, r, sdim[k], sdist[k], peer, dir, hops);
-        for (int i = 0; i < np; ++i) blocks[peer[i]] = 1;
-        for (int i = 0; i < np; ++i) block_propagation(tp, sdim, sdist, peer[i], k + 1, blocks);
+        int before = nsrc;                                   /* ranks reached in step k do not send again in step k */
+        for (int i = 0; i < before; ++i) {
+            int peer[2], dir[2], hops[2];
+            int np = send_peers(tp, src[i], sdim[k], sdist[k], peer, dir, hops);
+            for (int j = 0; j < np; ++j) {
+                blocks[peer[j]] = 1;
+                if (!seen[peer[j]] && nsrc < 2 * n) { seen[peer[j]] = 1; src[nsrc++] = peer[j]; }
+            }
+        }
     }
+    free(src); free(seen);
 }
 
 /* Blocks a rank sends to peer p in Reduce-Scatter step k: p's own block plus
@@ -646,7 +659,7 @@ done:
  * bytes per phase; the final step's congestion is d on every link; for n = 7 a node sends two
  * blocks per direction in the first step and one block, at distance two, in the final one.
  *
- * Reading where the paper is silent (PARITY UNPINNED by the paper; also in the design notes):
+ * Reading where the paper is silent (PARITY UNPINNED by the paper):
  * which tree a block follows.  The AllGather of block b runs the steps in reverse order (the
  * distance-d step first).  The nodes that hold the block are kept in the order they got it;
  * in a step every holder, in that order, offers the block first to its left peer (h - dist)

@@ -1,6 +1,7 @@
 """Rings whose size is no power of three (Sec. 4.4): pins of the oracle against what the paper and
 the arithmetic fix, and the library's host-side schedule against the oracle.  No GPU needed."""
 import math
+import os
 
 import numpy as np
 import pytest
@@ -54,6 +55,33 @@ def test_figure_seven_nodes():
     assert (ll["msgs"][1] == 2).all() and (ll["bytes"][1] == 2 * blk).all()      # two messages of one block each
     # the AllGather mirrors it
     assert np.array_equal(ll["bytes"][2], ll["bytes"][1]) and np.array_equal(ll["bytes"][3], ll["bytes"][0])
+
+
+def _golden_trees():
+    path = os.path.join(os.path.dirname(__file__), "golden", "general_ring_trees.txt")
+    trees = {}
+    with open(path) as f:
+        for line in f:
+            line = line.split("#")[0].split()
+            if line:
+                n, v, q, t = map(int, line)
+                trees.setdefault(n, {})[v] = (q, t)
+    return trees
+
+
+@pytest.mark.parametrize("n", [5, 7, 8, 10])
+def test_tree_equals_the_hand_worked_one(n):
+    """tests/golden/general_ring_trees.txt: parent and step of every node for block 0, worked by hand from the
+    stated rule (Sec. 4.4 fixes steps and distances; holder order and left-before-right are the reading).  Every
+    other block's tree is that one rotated."""
+    gold = _golden_trees()[n]
+    assert sorted(gold) == list(range(n))
+    par, stp = oracle.gen_tree(n)
+    for b in range(n):
+        for v in range(n):
+            q, t = gold[(v - b) % n]
+            assert stp[b, v] == t, (b, v)
+            assert par[b, v] == (-1 if q < 0 else (q + b) % n), (b, v)
 
 
 @pytest.mark.parametrize("n", SIZES)

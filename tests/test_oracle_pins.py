@@ -194,6 +194,28 @@ def test_block_propagation_from_step0_reaches_everyone_else():
             assert m.sum() >= n - 1 and all(m[q] for q in range(n) if q != r)
 
 
+@pytest.mark.parametrize("dims", [(9,), (27,), (3, 3), (9, 3), (3, 3, 3)])
+def test_block_propagation_is_every_increasing_path(dims):
+    """Algorithm 1 (Sec. 4.3) reaches exactly the ranks at the end of a non-empty path whose hops are taken in
+    steps of strictly increasing number >= step, each hop to one of the two peers of its step.  Brute force over
+    all subsets of steps and all left/right choices."""
+    n, S = oracle.num_steps(dims)
+    for c in range(len(dims)):
+        peers = [oracle.peers(dims, t, c) for t in range(S)]
+        for step in range(S + 1):
+            for r in range(0, n, 2):
+                want = set()
+                for mask in range(1, 1 << (S - step)):
+                    used = [step + i for i in range(S - step) if mask >> i & 1]
+                    for choice in itertools.product((0, 1), repeat=len(used)):
+                        q = r
+                        for t, side in zip(used, choice):
+                            q = int(peers[t][q, side])
+                        want.add(q)
+                got = set(np.nonzero(oracle.block_propagation(dims, r, step, c))[0].tolist())
+                assert got == want, (dims, c, step, r)
+
+
 def test_ring9_send_sets_worked_by_hand():
     """n = 9: in step 0 rank 0 sends {1,4,7} to rank 1 and {8,2,5} to rank 8; in step 1 one block each."""
     f = lambda p, k: sorted(np.nonzero(oracle.send_set((9,), p, k))[0].tolist())
