@@ -70,8 +70,9 @@ typedef enum { TRV_KERNEL_AUTO = 0, TRV_KERNEL_STEP = 1, TRV_KERNEL_FUSED = 2, T
  * round-robin order starting at c, that still has steps left (Sec. 5).
  *   dims  : HOST array of ndims sides (1 <= ndims <= TRV_MAX_DIMS), each 3^k, k >= 1
  *   out   : receives the plan; release with trv_plan_destroy
- * Host-only integer work; makes no CUDA call.  A plan is immutable: it may be used from
- * several threads and streams at once.
+ * Host-only integer work; makes no CUDA call.  A plan's schedule is immutable: it may be used
+ * from several threads and streams at once (the one mutable part, the scratch trv_allreduce may
+ * allocate for a few shapes, is described there).
  * Errors: INVALID_ARG (NULL, ndims out of range, side < 2), UNSUPPORTED (side not a power
  * of three, more than TRV_MAX_RANKS ranks).
  *
@@ -85,7 +86,8 @@ typedef enum { TRV_KERNEL_AUTO = 0, TRV_KERNEL_STEP = 1, TRV_KERNEL_FUSED = 2, T
  * every holder, in that order, offers it to its left peer (h - dist), then to its right peer
  * (h + dist); a node that already holds it is skipped.  The Reduce-Scatter runs the same tree
  * backwards, a receiver adding (from_left + own) + from_right and leaving out a side nothing
- * comes from.  Such plans run through the STEP kernels only.  The latency-optimal variant is
+ * comes from.  Such plans have a STEP family (one launch per step) and, up to TRV_MAX_RANKS ranks, a
+ * FUSED kernel that walks the block's tree as a stack machine.  The latency-optimal variant is
  * not defined for these sizes: UNSUPPORTED, as for tori with such a side. */
 trv_status_t trv_plan_create(const int32_t *dims, int32_t ndims, trv_variant_t variant, trv_plan_t *out);
 
@@ -150,12 +152,25 @@ trv_status_t trv_plan_block_bounds(trv_plan_t plan, size_t count, int32_t c, int
  *                 nearest even, no flush to zero
  *   op          : TRV_SUM only
  *   cuda_stream : a cudaStream_t (NULL = the legacy default stream)
- * Asynchronous; never synchronises.  If the chosen kernel family needs scratch memory (the
- * STEP family of the latency form does), the plan allocates it with cudaMalloc on first
- * need, keeps it, and frees it in trv_plan_destroy; such calls on ONE plan must then not
- * overlap on the device.  Use trv_allreduce_ex to pass your own scratch instead. */
+ * Asynchronous.  For every shape the FUSED family serves (trv_kernel_supported) the call is a pure launch:
+ * it allocates nothing, never synchronises and writes nothing into the plan, so any number of threads and
+ * streams may use one plan at once.
+ * Shapes that fall to the STEP family of the latency form (e.g. a 243 x 3 torus) need ping-pong scratch.  The
+ * plan then allocates it with cudaMalloc on first need -- on the device that is current in that call -- keeps it,
+ * grows it when a later call needs more (cudaFree + cudaMalloc: this WAITS FOR THE DEVICE) and frees it in
+ * trv_plan_destroy.  That scratch binds the plan to its device: a later such call with another device current
+ * returns INVALID_ARG.  The grow path is serialised by a lock inside the plan, so concurrent calls are safe on
+ * the host; but all such calls on ONE plan share the one scratch and must not overlap on the device (order them
+ * on one stream or by events).  To keep trv_allreduce launch-only for these shapes too, call
+ * trv_plan_reserve_scratch once beforehand; to use your own scratch, call trv_allreduce_ex. */
 trv_status_t trv_allreduce(trv_plan_t plan, void *const *rank_buffers, size_t count, trv_dtype_t dtype, trv_op_t op,
                            void *cuda_stream);
+
+/* Allocates (or grows) the plan-owned scratch that trv_allreduce needs for vectors of up to `count` elements, on
+ * the current device; a no-op for shapes that need none.  May wait for the device (it frees a smaller scratch
+ * first).  After it, trv_allreduce calls with count' <= count on this plan allocate and synchronise nothing.
+ * Errors: INVALID_ARG (the plan's scratch lives on another device), ALLOC, CUDA, UNSUPPORTED (comparator plan). */
+trv_status_t trv_plan_reserve_scratch(trv_plan_t plan, size_t count);
 
 /* Bytes of scratch trv_allreduce_ex needs for this call shape (0 if none). */
 trv_status_t trv_scratch_bytes(trv_plan_t plan, size_t count, trv_kernel_t kernel, int32_t in_place, size_t *bytes);
@@ -180,12 +195,21 @@ trv_status_t trv_allreduce_ex(trv_plan_t plan, const void *const *in_buffers, vo
                               size_t global_count, size_t global_offset, trv_dtype_t dtype, trv_op_t op,
                               trv_kernel_t kernel, void *scratch, size_t scratch_bytes, void *cuda_stream);
 
-/* AllReduce of HOST vectors: copies the n host vectors into `workspace`, runs the AllReduce
- * there and copies the n results back, all queued on `cuda_stream`; returns without
- * synchronising (the host buffers must stay valid, and should be pinned, until the stream
- * reaches the end of this work).
- *   host_in / host_out: HOST arrays of n HOST pointers to count*4 bytes each (may be equal)
- *   workspace   : DEVICE pointer, 256-byte aligned, >= trv_host_workspace_bytes(...) bytes */
+/* AllReduce of HOST vectors, pipelined over element-range windows (columns of elements are independent, Sec. 2.2):
+ * window k + 1 is copied to the device while window k is reduced there (trv_allreduce_ex with the global element
+ * index) and window k - 1 is copied back; three window slots rotate through `workspace`, so the device holds a few
+ * windows, never the whole n x count matrix, and both directions of the host link are busy at once.
+ *   host_in / host_out: HOST arrays of n HOST pointers to count*4 bytes each; they may be equal (in place).
+ *                 Pinned memory is needed for the copies to overlap; equally spaced rows (rows of one matrix)
+ *                 are moved by one 2-D copy per window and direction instead of n copies.
+ *   workspace   : DEVICE pointer, 256-byte aligned.  trv_host_workspace_bytes(...) is the size for the preferred
+ *                 window (an eighth of the vector, between 64 KiB per rank and 128 MiB over all ranks); a smaller
+ *                 workspace is accepted and gives shorter windows; SCRATCH if not even windows of 64 elements fit.
+ * Uploads and downloads run on two internal streams that the library creates on the first call on a device (make
+ * that call outside any stream capture); kernels run on `cuda_stream`.  The internal streams wait for the work
+ * queued on `cuda_stream` before the call, and `cuda_stream` ends up waiting for the last download: to the caller
+ * the call is work queued on `cuda_stream`.  It returns without synchronising; the host buffers must stay valid
+ * until the stream reaches the end of this work.  Calls that share a workspace must be ordered by the caller. */
 trv_status_t trv_allreduce_host(trv_plan_t plan, const void *const *host_in, void *const *host_out, size_t count,
                                 trv_dtype_t dtype, trv_op_t op, void *workspace, size_t workspace_bytes,
                                 void *cuda_stream);

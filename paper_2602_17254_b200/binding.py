@@ -30,7 +30,7 @@ SYMBOLS = [
     "trv_kernel_supported", "trv_allreduce_ex", "trv_allreduce_host", "trv_host_workspace_bytes",
     "trv_link_loads", "trv_plan_message_bytes", "trv_plan_message_bytes_side", "trv_strerror", "trv_launch_count", "trv_last_kernel_name",
     "trv_allreduce_noalloc", "trv_noalloc_max_scratch_bytes", "trv_cost_model", "trv_pipeline_status",
-    "trv_pipeline_selftest_timeout", "trv_tma_giveups",
+    "trv_pipeline_selftest_timeout", "trv_tma_giveups", "trv_plan_reserve_scratch",
 ]
 
 
@@ -72,6 +72,7 @@ def lib():
         L.trv_pipeline_status.argtypes = [vp, vp]
         L.trv_pipeline_selftest_timeout.argtypes = [vp, sz, vp]
         L.trv_allreduce.argtypes = [vp, vp, sz, ctypes.c_int, ctypes.c_int, vp]
+        L.trv_plan_reserve_scratch.argtypes = [vp, sz]
         L.trv_scratch_bytes.argtypes = [vp, sz, ctypes.c_int, i32, ctypes.POINTER(sz)]
         L.trv_kernel_supported.argtypes = [vp, ctypes.c_int]
         L.trv_kernel_supported.restype = i32
@@ -218,6 +219,11 @@ class Plan:
         b = ctypes.c_size_t()
         _check(lib().trv_scratch_bytes(self._h, count, int(kernel), 1 if in_place else 0, ctypes.byref(b)), "trv_scratch_bytes")
         return b.value
+
+    def reserve_scratch(self, count):
+        """trv_plan_reserve_scratch: allocate the plan-owned scratch trv_allreduce needs up to this count (may wait for
+        the device); afterwards trv_allreduce is launch-only for every shape."""
+        _check(lib().trv_plan_reserve_scratch(self._h, count), "trv_plan_reserve_scratch")
 
     def host_workspace_bytes(self, count):
         b = ctypes.c_size_t()

@@ -55,9 +55,14 @@ static trv_status_t dispatch(Call& c, trv_kernel_t kernel) {
     } else if (kernel == TRV_KERNEL_AUTO) {
         fused = fused_supported(p);
     }
-    if (p.general) return fused ? run_fused_tree(c) : run_step_general(c);
-    if (p.variant == TRV_LATENCY_OPTIMAL) return fused ? run_fused_latency(c) : run_step_latency(c);
-    return fused ? run_fused_bandwidth(c) : run_step_bandwidth(c);
+    if (fused) {
+        const trv_status_t st = p.general ? run_fused_tree(c)
+                                : (p.variant == TRV_LATENCY_OPTIMAL ? run_fused_latency(c) : run_fused_bandwidth(c));
+        // a fused launcher that cannot serve this call shape: AUTO goes on to the STEP family (which checks the scratch)
+        if (st != TRV_ERR_UNSUPPORTED || kernel != TRV_KERNEL_AUTO) return st;
+    }
+    if (p.general) return run_step_general(c);
+    return p.variant == TRV_LATENCY_OPTIMAL ? run_step_latency(c) : run_step_bandwidth(c);
 }
 }  // namespace trv
 
@@ -210,6 +215,30 @@ trv_status_t trv_allreduce_ex(trv_plan_t plan, const void* const* in_buffers, vo
     return dispatch(c, kernel);
 }
 
+// Grows the plan-owned scratch to `need` bytes on the current device.  Caller holds scratch_mu.
+static trv_status_t grow_plan_scratch(Plan& p, size_t need) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return TRV_ERR_CUDA;
+    if (p.scratch && p.scratch_device != dev) return TRV_ERR_INVALID_ARG;   // the scratch lives on another GPU
+    if (need <= p.scratch_bytes) return TRV_OK;
+    // cudaFree waits for the device: kernels of earlier calls that still use the old scratch finish first
+    if (p.scratch) { cudaFree(p.scratch); p.scratch = nullptr; p.scratch_bytes = 0; p.scratch_device = -1; }
+    if (cudaMalloc(&p.scratch, need) != cudaSuccess) { (void)cudaGetLastError(); return TRV_ERR_ALLOC; }
+    p.scratch_bytes = need;
+    p.scratch_device = dev;
+    return TRV_OK;
+}
+
+trv_status_t trv_plan_reserve_scratch(trv_plan_t plan, size_t count) {
+    if (!plan) return TRV_ERR_INVALID_ARG;
+    size_t need = 0;
+    trv_status_t st = trv_scratch_bytes(plan, count, TRV_KERNEL_AUTO, 1, &need);
+    if (st != TRV_OK) return st;
+    std::lock_guard<std::mutex> lock(plan->scratch_mu);
+    if (need == 0 && !plan->plan.scratch) return TRV_OK;
+    return grow_plan_scratch(plan->plan, need);
+}
+
 trv_status_t trv_allreduce(trv_plan_t plan, void* const* rank_buffers, size_t count, trv_dtype_t dtype, trv_op_t op,
                            void* cuda_stream) {
     if (!plan) return TRV_ERR_INVALID_ARG;
@@ -217,59 +246,23 @@ trv_status_t trv_allreduce(trv_plan_t plan, void* const* rank_buffers, size_t co
     size_t need = 0;
     trv_status_t st = trv_scratch_bytes(plan, count, TRV_KERNEL_AUTO, 1, &need);
     if (st != TRV_OK) return st;
-    if (need > p.scratch_bytes) {
-        // validate before allocating anything
-        bool ip;
+    if (need == 0)      // the fused kernels: a pure launch, nothing of the plan is written
+        return trv_allreduce_ex(plan, (const void* const*)rank_buffers, rank_buffers, count, count, 0, dtype, op,
+                                TRV_KERNEL_AUTO, nullptr, 0, cuda_stream);
+    // STEP family of the latency form: the plan's own scratch.  The lock is held until the launches are queued, so
+    // that a concurrent call which has to grow (and free) the scratch cannot pull it away in between.
+    std::lock_guard<std::mutex> lock(plan->scratch_mu);
+    if (need > p.scratch_bytes || !p.scratch) {
+        bool ip;        // validate before allocating anything
         if (dtype != TRV_INT32 && dtype != TRV_FLOAT32) return TRV_ERR_INVALID_ARG;
         if (op != TRV_SUM) return TRV_ERR_UNSUPPORTED;
         st = check_buffers(p, (const void* const*)rank_buffers, rank_buffers, count, &ip);
         if (st != TRV_OK) return st;
-        if (p.scratch) { cudaFree(p.scratch); p.scratch = nullptr; p.scratch_bytes = 0; }
-        if (cudaMalloc(&p.scratch, need) != cudaSuccess) { (void)cudaGetLastError(); return TRV_ERR_ALLOC; }
-        p.scratch_bytes = need;
     }
+    st = grow_plan_scratch(p, need);
+    if (st != TRV_OK) return st;
     return trv_allreduce_ex(plan, (const void* const*)rank_buffers, rank_buffers, count, count, 0, dtype, op,
                             TRV_KERNEL_AUTO, p.scratch, p.scratch_bytes, cuda_stream);
-}
-
-static size_t host_row_bytes(size_t count) { return ((count * 4) + 255) & ~(size_t)255; }
-
-trv_status_t trv_host_workspace_bytes(trv_plan_t plan, size_t count, size_t* bytes) {
-    if (!plan || !bytes) return TRV_ERR_INVALID_ARG;
-    size_t scratch = 0;
-    trv_status_t st = trv_scratch_bytes(plan, count, TRV_KERNEL_AUTO, 1, &scratch);
-    if (st != TRV_OK) return st;
-    *bytes = (size_t)plan->plan.n * host_row_bytes(count) + scratch;
-    return TRV_OK;
-}
-
-trv_status_t trv_allreduce_host(trv_plan_t plan, const void* const* host_in, void* const* host_out, size_t count,
-                                trv_dtype_t dtype, trv_op_t op, void* workspace, size_t workspace_bytes,
-                                void* cuda_stream) {
-    if (!plan || !host_in || !host_out) return TRV_ERR_INVALID_ARG;
-    const Plan& p = plan->plan;
-    if (p.algo != TRV_ALGO_TRIVANCE) return TRV_ERR_UNSUPPORTED;
-    size_t need = 0;
-    trv_status_t st = trv_host_workspace_bytes(plan, count, &need);
-    if (st != TRV_OK) return st;
-    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return TRV_ERR_SCRATCH;
-    for (int r = 0; r < p.n; ++r)
-        if (!host_in[r] || !host_out[r]) return TRV_ERR_INVALID_ARG;
-    if (count == 0) return TRV_OK;
-    cudaStream_t s = (cudaStream_t)cuda_stream;
-    const size_t row = host_row_bytes(count);
-    std::vector<void*> dev(p.n);
-    for (int r = 0; r < p.n; ++r) {
-        dev[r] = (char*)workspace + (size_t)r * row;
-        if (cudaMemcpyAsync(dev[r], host_in[r], count * 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return TRV_ERR_CUDA;
-    }
-    void* scratch = (char*)workspace + (size_t)p.n * row;
-    st = trv_allreduce_ex(plan, (const void* const*)dev.data(), dev.data(), count, count, 0, dtype, op, TRV_KERNEL_AUTO,
-                          need > (size_t)p.n * row ? scratch : nullptr, need - (size_t)p.n * row, s);
-    if (st != TRV_OK) return st;
-    for (int r = 0; r < p.n; ++r)
-        if (cudaMemcpyAsync(host_out[r], dev[r], count * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return TRV_ERR_CUDA;
-    return TRV_OK;
 }
 
 trv_status_t trv_tma_giveups(uint32_t* count) {

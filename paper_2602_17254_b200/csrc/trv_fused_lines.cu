@@ -11,8 +11,15 @@
 // reads global memory directly and the last one writes it directly: 2 (groups - 1) shared-memory
 // passes per tile.  The host builds the group list and the base rank r0 of every set (integer work)
 // and passes both by value.
+//
+// The file is compiled five times (build.py): TRV_LN_PART = 0 gives the host side, 1..4 the kernels of one
+// (element type, tile width) pair each, so that the long straight-line bodies compile in parallel.
 #include "trv_dev.cuh"
 #include "trv_fused_lat.cuh"
+
+#ifndef TRV_LN_PART
+#error "compile with -DTRV_LN_PART=0..4 (see build.py)"
+#endif
 
 namespace trv {
 
@@ -35,6 +42,7 @@ struct LnProgram {
     short bases[kLnMaxD][kLnMaxBases];
 };
 
+#if TRV_LN_PART > 0
 template <typename T, int N, bool FULL, typename Addr, typename RankOf>
 __device__ __forceinline__ void ln_load(Elem<T, 1> (&v)[N], bool from_global, const Addr& in, const T* mine, int pitch, long long e,
                                         long long lo, long long hi, RankOf rank_of) {
@@ -153,8 +161,27 @@ __global__ void __launch_bounds__(32 * kLnSets, 2) k_lat_lines(Addr in, Addr out
     else ln_tile<T, CG, false>(p, c, in, out, slab, t0, lo, hi);
 }
 
+template <typename T, int CG, typename Addr>
+static trv_status_t launch_lines_cg(const Call& c, const Addr& in, const Addr& out, const LatArgs& a, const LnProgram& prog) {
+    const Plan& p = *c.plan;
+    long long tiles = 0;
+    for (int sl = 0; sl < p.ndims; ++sl)
+        if (a.hi[sl] > a.lo[sl]) {
+            const long long tw = 32 * CG;
+            const long long t = (a.hi[sl] - (a.lo[sl] & ~31LL) + tw - 1) / tw;
+            if (t > tiles) tiles = t;
+        }
+    if (tiles == 0) return TRV_OK;
+    auto kfn = k_lat_lines<T, CG, Addr>;
+    if (!allow_big_smem(kfn, 729 * 32 * 4)) return TRV_ERR_CUDA;
+    launch_pdl(kfn, dim3((unsigned)tiles, p.ndims, 1), dim3(32 * kLnSets), (size_t)p.n * 32 * CG * sizeof(T), c.st, in, out, a, prog);
+    return TRV_OK;
+}
+#endif  // TRV_LN_PART > 0
+
 // ------------------------------------------------------------------ host side
 
+#if TRV_LN_PART == 0
 bool fused_lines_supported(const Plan& p) {
     if (p.algo != TRV_ALGO_TRIVANCE || p.variant != TRV_LATENCY_OPTIMAL) return false;
     if (p.n > 729 || p.ndims > kLnMaxD) return false;
@@ -216,47 +243,46 @@ static bool build_program(const Plan& p, LnProgram* prog) {
     }
     return true;
 }
+#endif  // TRV_LN_PART == 0
 
-template <typename T, int CG, typename Addr>
-static trv_status_t launch_lines_cg(const Call& c, const Addr& in, const Addr& out, const LatArgs& a, const LnProgram& prog) {
+// one (element type, tile width) pair per translation unit
+template <typename T, int CG>
+trv_status_t launch_lines_part(const Call& c, const LatArgs& a, const LnProgram& prog);
+
+#if TRV_LN_PART > 0
+template <typename T, int CG>
+trv_status_t launch_lines_part(const Call& c, const LatArgs& a, const LnProgram& prog) {
     const Plan& p = *c.plan;
-    long long tiles = 0;
-    for (int sl = 0; sl < p.ndims; ++sl)
-        if (a.hi[sl] > a.lo[sl]) {
-            const long long tw = 32 * CG;
-            const long long t = (a.hi[sl] - (a.lo[sl] & ~31LL) + tw - 1) / tw;
-            if (t > tiles) tiles = t;
-        }
-    if (tiles == 0) return TRV_OK;
-    auto kfn = k_lat_lines<T, CG, Addr>;
-    if (!allow_big_smem(kfn, 729 * 32 * 4)) return TRV_ERR_CUDA;
-    launch_pdl(kfn, dim3((unsigned)tiles, p.ndims, 1), dim3(32 * kLnSets), (size_t)p.n * 32 * CG * sizeof(T), c.st, in, out, a, prog);
-    return TRV_OK;
+    StrideAddr sin, sout;
+    if (uniform_stride(c.in, p.n, &sin) && uniform_stride((const void* const*)c.out, p.n, &sout))
+        return launch_lines_cg<T, CG>(c, sin, sout, a, prog);
+    TabAddr<729> in, out;
+    for (int r = 0; r < p.n; ++r) { in.t.p[r] = const_cast<void*>(c.in[r]); out.t.p[r] = c.out[r]; }
+    return launch_lines_cg<T, CG>(c, in, out, a, prog);
 }
+#if TRV_LN_PART == 1
+template trv_status_t launch_lines_part<float, 9>(const Call&, const LatArgs&, const LnProgram&);
+#elif TRV_LN_PART == 2
+template trv_status_t launch_lines_part<float, 1>(const Call&, const LatArgs&, const LnProgram&);
+#elif TRV_LN_PART == 3
+template trv_status_t launch_lines_part<uint32_t, 9>(const Call&, const LatArgs&, const LnProgram&);
+#else
+template trv_status_t launch_lines_part<uint32_t, 1>(const Call&, const LatArgs&, const LnProgram&);
+#endif
+#endif  // TRV_LN_PART > 0
 
-template <typename T, typename Addr>
-static trv_status_t launch_lines(const Call& c, const Addr& in, const Addr& out, const LatArgs& a, const LnProgram& prog) {
-    if (prog.cg == 9) return launch_lines_cg<T, 9>(c, in, out, a, prog);
-    if (prog.cg == 3) return launch_lines_cg<T, 3>(c, in, out, a, prog);
-    return launch_lines_cg<T, 1>(c, in, out, a, prog);
-}
-
+#if TRV_LN_PART == 0
 trv_status_t run_fused_lines(const Call& c, const LatArgs& a) {
     const Plan& p = *c.plan;
     if (!fused_lines_supported(p)) return TRV_ERR_UNSUPPORTED;
     static thread_local LnProgram prog;       // 13 KB: kept off the stack
     if (!build_program(p, &prog)) return TRV_ERR_UNSUPPORTED;
-    StrideAddr sin, sout;
     trv_status_t st;
-    if (uniform_stride(c.in, p.n, &sin) && uniform_stride((const void* const*)c.out, p.n, &sout)) {
-        st = c.dtype == TRV_FLOAT32 ? launch_lines<float>(c, sin, sout, a, prog) : launch_lines<uint32_t>(c, sin, sout, a, prog);
-    } else {
-        TabAddr<729> in, out;
-        for (int r = 0; r < p.n; ++r) { in.t.p[r] = const_cast<void*>(c.in[r]); out.t.p[r] = c.out[r]; }
-        st = c.dtype == TRV_FLOAT32 ? launch_lines<float>(c, in, out, a, prog) : launch_lines<uint32_t>(c, in, out, a, prog);
-    }
+    if (c.dtype == TRV_FLOAT32) st = prog.cg == 9 ? launch_lines_part<float, 9>(c, a, prog) : launch_lines_part<float, 1>(c, a, prog);
+    else st = prog.cg == 9 ? launch_lines_part<uint32_t, 9>(c, a, prog) : launch_lines_part<uint32_t, 1>(c, a, prog);
     if (st != TRV_OK) return st;
     return cudaGetLastError() == cudaSuccess ? TRV_OK : TRV_ERR_CUDA;
 }
+#endif
 
 }  // namespace trv

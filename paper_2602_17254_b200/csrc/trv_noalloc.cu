@@ -1,7 +1,9 @@
 // trv_allreduce_noalloc: the step-by-step latency-form AllReduce for callers that must not
 // allocate device memory.  Its ping-pong scratch is a fixed array that is part of the library
 // image, so the call needs no cudaMalloc, no cudaFree and no memory pool.
+#include <algorithm>
 #include <mutex>
+#include <vector>
 
 #include "trv_dev.cuh"
 
@@ -47,14 +49,16 @@ trv_status_t trv_allreduce_noalloc(trv_plan_t plan, void* const* rank_buffers, s
     if (p.algo != TRV_ALGO_TRIVANCE || p.variant != TRV_LATENCY_OPTIMAL) return TRV_ERR_UNSUPPORTED;
     if (dtype != TRV_INT32 && dtype != TRV_FLOAT32) return TRV_ERR_INVALID_ARG;
     if (op != TRV_SUM) return TRV_ERR_UNSUPPORTED;
+    if (count >= ((size_t)1 << 40)) return TRV_ERR_TOO_LARGE;     // before any count * 4 below
+    // 16-byte aligned, pairwise disjoint: sort the start addresses (host stack/heap only, no device memory)
+    std::vector<uintptr_t> starts((size_t)p.n);
     for (int r = 0; r < p.n; ++r) {
         if (!rank_buffers[r] || ((uintptr_t)rank_buffers[r] & 15)) return TRV_ERR_INVALID_ARG;
-        for (int q = 0; q < r; ++q) {
-            const uintptr_t a = (uintptr_t)rank_buffers[q], b = (uintptr_t)rank_buffers[r];
-            if (a < b + count * 4 && b < a + count * 4) return TRV_ERR_INVALID_ARG;
-        }
+        starts[r] = (uintptr_t)rank_buffers[r];
     }
-    if (count >= ((size_t)1 << 40)) return TRV_ERR_TOO_LARGE;
+    std::sort(starts.begin(), starts.end());
+    for (int r = 1; r < p.n; ++r)
+        if (starts[r] - starts[r - 1] < count * 4) return TRV_ERR_INVALID_ARG;
     const size_t need = step_scratch_bytes(p, count, /*in_place=*/true);
     if (need > TRV_NOALLOC_SCRATCH_BYTES) return TRV_ERR_TOO_LARGE;
     if (count == 0) return TRV_OK;

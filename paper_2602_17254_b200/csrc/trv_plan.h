@@ -2,6 +2,7 @@
 #pragma once
 #include <cstddef>
 #include <cstdint>
+#include <mutex>
 #include <vector>
 
 #include "../../include/trivance.h"
@@ -42,9 +43,11 @@ struct Plan {
     bool general = false;
     std::vector<int8_t> gstep, gsgn;
 
-    // plan-owned scratch for trv_allreduce (STEP family of the latency form), grown on demand
+    // plan-owned scratch for trv_allreduce (STEP family of the latency form), grown on demand under
+    // trv_plan_s::scratch_mu; scratch_device = ordinal of the GPU it was allocated on (-1: none yet)
     void* scratch = nullptr;
     size_t scratch_bytes = 0;
+    int scratch_device = -1;
 
     int rows() const { return variant == TRV_BANDWIDTH_OPTIMAL ? 2 * S : S; }
     // schedule step behind a row: AllGather rows mirror the Reduce-Scatter steps
@@ -82,6 +85,7 @@ int general_recv_mask(const Plan& p, int t, int dst, int j);
 
 struct trv_plan_s {
     trv::Plan plan;
+    std::mutex scratch_mu;      // guards plan.scratch* (the only mutable part of a plan)
 };
 
 namespace trv {

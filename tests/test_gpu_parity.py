@@ -165,6 +165,62 @@ def test_host_buffer_entry_point():
     assert e.value.status == binding.ERR_SCRATCH
 
 
+@pytest.mark.parametrize("dims,variant,count,dist", [
+    ((27,), LAT, 200003, "normal"),         # 8 windows of 25024 elements + a ragged last one
+    ((9, 9), BW, 150001, "int32"),          # block and slice bounds must follow the global element index
+    ((9, 9, 9), LAT, 50021, "normal"),      # the TMA-fed kernel on windows of a longer vector
+    ((100,), BW, 140000, "normal"),         # ring of another size
+    ((243, 3), LAT, 70001, "normal"),       # STEP family: every window slot carries its own scratch
+])
+def test_host_buffer_entry_point_runs_windows_of_the_vector(dims, variant, count, dist):
+    """trv_allreduce_host pipelines element-range windows; the result is the oracle's for the whole vector."""
+    plan = binding.Plan(dims, variant)
+    n = plan.n
+    x = synth.rank_matrix(dist, 72, n, count)
+    hin = torch.from_numpy(x.copy()).pin_memory()
+    hout = torch.empty_like(hin).pin_memory()
+    need = plan.host_workspace_bytes(count)
+    assert need < n * count * 4 or count < 8 * 16384        # a few windows, not the whole matrix
+    ws = torch.empty(need, dtype=torch.uint8, device=DEV)
+    dcode = binding.INT32 if dist == "int32" else binding.FLOAT32
+    stream = torch.cuda.current_stream().cuda_stream
+    before = binding.launch_count()
+    plan.allreduce_host([hin[r].data_ptr() for r in range(n)], [hout[r].data_ptr() for r in range(n)], count, dcode,
+                        ws.data_ptr(), ws.numel(), stream)
+    torch.cuda.synchronize()
+    assert binding.launch_count() - before >= min(8, -(-count // 16384))      # one AllReduce per window
+    compare(dims, variant, x, hout.numpy())
+    assert np.array_equal(hin.numpy(), x)
+    # in place on the host, rows NOT equally spaced (one copy per row), and a workspace a fifth of the preferred size
+    rows = [torch.empty(count + 64 * (r % 3), dtype=hin.dtype).pin_memory() for r in range(n)]
+    for r in range(n):
+        rows[r][:count].copy_(torch.from_numpy(x[r]))
+    small = torch.empty(need // 5 // 256 * 256, dtype=torch.uint8, device=DEV)
+    plan.allreduce_host([t.data_ptr() for t in rows], None, count, dcode, small.data_ptr(), small.numel(), stream)
+    torch.cuda.synchronize()
+    got = np.stack([t[:count].numpy() for t in rows])
+    assert np.array_equal(got.view(np.uint32), hout.numpy().view(np.uint32))
+
+
+def test_plan_owned_scratch_is_bound_to_its_device_and_can_be_reserved():
+    """trv_allreduce on a shape that needs the STEP family's scratch: reserve first, then the call launches only."""
+    dims, count = (243, 3), 777
+    plan = binding.Plan(dims, LAT)
+    assert plan.scratch_bytes(count) > 0
+    plan.reserve_scratch(4 * count)
+    x = synth.rank_matrix("normal", 73, plan.n, count)
+    xd = torch.zeros((plan.n, 780), device=DEV)[:, :count]
+    xd.copy_(torch.from_numpy(x))
+    for _ in range(2):
+        xd.copy_(torch.from_numpy(x))
+        plan.allreduce([xd[r].data_ptr() for r in range(plan.n)], count, binding.FLOAT32, torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        compare(dims, LAT, x, xd.cpu().numpy())
+    plan.destroy()
+    fused = binding.Plan((27,), LAT)        # nothing to reserve for a fused shape
+    fused.reserve_scratch(10 ** 6)
+
+
 def test_fp32_tolerance_against_naive_and_exact_sums():
     """|err| <= 2e-6 * sum|x| against the naive sequential binary32 sum (and the fp64 sum)."""
     for dims, variant, dist in [((27,), LAT, "normal"), ((81,), BW, "normal"), ((9, 9, 9), LAT, "uniform"),

@@ -2,7 +2,8 @@
 running under stream capture, inside a framework that owns all device memory, or with a fixed
 memory budget).  Its scratch is a fixed 16 MiB array inside the library instead of a cudaMalloc'd
 buffer.  The test calls it through the C ABI twice in a row and compares every output bit with
-the ordinary entry point's (trv_allreduce_ex), then checks that oversized calls are refused.
+the ordinary entry point's (trv_allreduce_ex) and with the CPU oracle's, then checks that oversized
+calls are refused.
 
 Collected last on purpose (file name), so a run that stops at the first failure has already run
 every other test; it passes on its own in a fresh process as well."""
@@ -10,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2602_17254_b200 import binding, build, synth
 
 pytestmark = pytest.mark.gpu
@@ -49,6 +51,8 @@ def test_noalloc_matches_the_ordinary_entry_point_twice_in_a_row(dims, count, di
         torch.cuda.synchronize()
         got = xd.cpu().numpy()
         assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), "call %d differs" % call
+        exact = oracle.allreduce(dims, binding.LATENCY_OPTIMAL, x)
+        assert np.array_equal(got.view(np.uint32), exact.view(np.uint32)), "call %d differs from the oracle" % call
         assert binding.last_kernel_name() == "step_latency"
 
 
