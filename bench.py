@@ -3,11 +3,17 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
-One "step" is one pass of the hot path over a batch of independent synthetic buffer sets of the
-chosen workload: for every set one trv_allreduce_ex call (plan built once, outside the timed
-region).  The batch is sized so that the sets of one step exceed several times the L2 capacity:
-every call reads cold data from HBM.  Metric: effective AllReduce GB/s = n * S_bytes / t, where
-S_bytes is the per-rank vector size.  Rank 0 prints ONE JSON line.
+Default workload: torus9x9x9_lat_32MiB, the largest single-GPU configuration (729 ranks x 32 MiB).
+One "step" is `calls_per_step` passes of the whole hot path, each one trv_allreduce_ex call on one of
+`buffer_sets` independent synthetic buffer sets of the workload (plan built once, outside the timed
+region); consecutive calls rotate over sets that together exceed several times the L2 capacity, so
+every call reads cold data from HBM.  calls_per_step is chosen after the warm-up so that the timed
+region lasts at least 0.55 s (clock samples then fall inside it).  Metric: effective AllReduce GB/s =
+n * S_bytes / t, S_bytes = per-rank vector size.  Rank 0 prints ONE JSON line; besides the contract's
+keys it carries `roofline` (dominant kernel against the measured copy bandwidth), `e2e` (host buffers
+through trv_allreduce_host, with the plain pinned-copy rate of the same bytes as ceiling),
+`in_place_trv_allreduce_us` (the in-place call), `cpu_baseline` (the oracle on the host cores) and
+`per_workload`: the device-resident leg of every other configuration with >= 2 MiB per rank.
 
 With --gpus N > 1 (launched under torchrun) every GPU runs its own batch (element columns are
 independent, so a longer vector sharded by element range behaves the same): no collective on the
@@ -32,7 +38,7 @@ if ROOT not in sys.path:
 
 from paper_2602_17254_b200 import synth  # noqa: E402
 
-DEFAULT_WORKLOAD = "ring27_lat_2MiB"
+DEFAULT_WORKLOAD = "torus9x9x9_lat_32MiB"
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
 
@@ -197,6 +203,191 @@ class ClockSampler:
 
 # ------------------------------------------------------------------ GPU legs
 
+MIN_REGION_S = 0.55     # every timed region lasts at least this long, so that NVML samples fall inside it
+PER_WORKLOAD = ["ring27_lat_2MiB", "ring81_bw_8MiB", "torus9x9x9_lat_32MiB", "torus9x9x9_bw_32MiB", "ring243_lat_8MiB",
+                "ring243_bw_8MiB", "ring243_lat_32MiB", "ring243_bw_32MiB"]      # the configurations with >= 2 MiB per rank
+
+
+class Leg:
+    """Device buffers and call arguments of one workload: `batch` independent buffer sets."""
+
+    def __init__(self, torch, binding, w, dev, rank, batch, kfam):
+        self.torch, self.binding, self.w, self.kfam = torch, binding, w, kfam
+        n, count = w.n, w.count
+        self.set_bytes = n * count * 4
+        self.batch = batch or max(1, min(64, max(16, -(-4 * L2_BYTES // self.set_bytes)), (24 * 2**30) // self.set_bytes))
+        self.tdt = torch.int32 if w.dist == "int32" else torch.float32
+        self.dcode = binding.INT32 if w.dist == "int32" else binding.FLOAT32
+        self.plan = binding.Plan(w.dims, w.variant)
+        # Set 0 carries the workload's seeded vectors in its first columns (all of them when the set is small):
+        # they feed the parity spot check.  Everything else is drawn on the device with the same distribution
+        # (values do not influence the run time: the path has no data-dependent control flow).
+        self.check_cols = count if self.set_bytes <= 2**28 else min(count, 4096)
+        self.x0 = np.stack([synth.rank_vector(w.dist, w.seed, r, self.check_cols) for r in range(n)])
+        self.ins = torch.empty((self.batch, n, count), dtype=self.tdt, device=dev)
+        self.outs = torch.empty((self.batch, n, count), dtype=self.tdt, device=dev)
+        g = torch.Generator(device=dev)
+        g.manual_seed(1000 * w.seed + rank)
+        for b in range(self.batch):
+            if w.dist == "int32":
+                self.ins[b].copy_(torch.randint(-1000, 1001, (n, count), generator=g, device=dev, dtype=self.tdt))
+            elif w.dist == "normal":
+                self.ins[b].normal_(generator=g)
+            else:
+                self.ins[b].uniform_(-1.0, 1.0, generator=g)
+        self.ins[0][:, :self.check_cols].copy_(torch.from_numpy(self.x0))
+        self.in_ptrs = [binding.ptr_array([self.ins[b, r].data_ptr() for r in range(n)]) for b in range(self.batch)]
+        self.out_ptrs = [binding.ptr_array([self.outs[b, r].data_ptr() for r in range(n)]) for b in range(self.batch)]
+        self.need = self.plan.scratch_bytes(count, kfam, in_place=False)
+        self.scratch = torch.empty(max(self.need, 256), dtype=torch.uint8, device=dev)
+        self.plan.reserve_scratch(count)            # trv_allreduce (in place) then only launches
+
+    def call(self, b):
+        self.plan.allreduce_ex(self.in_ptrs[b], self.out_ptrs[b], self.w.count, self.dcode, kernel=self.kfam,
+                               scratch_ptr=self.scratch.data_ptr() if self.need else 0, scratch_bytes=self.need,
+                               stream=self.torch.cuda.current_stream().cuda_stream)
+
+    def call_in_place(self, b):     # the call the engine is named for: trv_allreduce on the output buffers of set b
+        self.plan.allreduce(self.out_ptrs[b], self.w.count, self.dcode, self.torch.cuda.current_stream().cuda_stream)
+
+    def parity(self):
+        """Set 0's output of the timed calls against the oracle, on the seeded columns."""
+        import oracle
+        want = oracle.allreduce(self.w.dims, self.w.variant, self.x0, E=self.w.count, e0=0)
+        got = self.outs[0, :, :self.check_cols].cpu().numpy()
+        return bool(np.array_equal(got.view(np.uint32), want.view(np.uint32)))
+
+    def free(self):
+        self.plan.destroy()
+        for name in ("ins", "outs", "scratch"):
+            setattr(self, name, None)
+        self.torch.cuda.empty_cache()
+
+
+def _timed(torch, stream, fn, reps, sampler=None):
+    """Milliseconds (CUDA events on the launching stream) of `reps` calls of fn(i)."""
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.start()
+    ev0.record(stream)
+    for i in range(reps):
+        fn(i)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.stop()
+    return ev0.elapsed_time(ev1)
+
+
+def _calls_per_step(torch, stream, leg, steps, fixed):
+    """Calls per step: a whole number of passes over the batch, enough for a timed region of MIN_REGION_S."""
+    if fixed:
+        return leg.batch
+    ms = _timed(torch, stream, lambda i: leg.call(i % leg.batch), 2 * leg.batch) / (2 * leg.batch)
+    passes = max(1, int(np.ceil(MIN_REGION_S * 1e3 / (ms * steps * leg.batch))))
+    return passes * leg.batch
+
+
+def _roofline(set_bytes, launches, calls, ms, kernel_name, workload):
+    per_launch_ms = ms / launches
+    algo_bytes = 2 * set_bytes / (launches / calls)         # per launch of the dominant kernel
+    peak, peak_src = _peak()
+    achieved = algo_bytes / (per_launch_ms * 1e-3) / 1e9
+    return {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "traffic": _traffic(kernel_name, workload), "peak_source": peak_src, "algorithmic_bytes_per_launch": algo_bytes,
+            "avg_launch_us": per_launch_ms * 1e3, "frac_of_nominal_8000": achieved / 8000.0}
+
+
+def _side_leg(torch, binding, name, dev, local, steps, kfam):
+    """One entry of `per_workload`: the device-resident leg of another configuration."""
+    w = synth.CONFIGS[name]
+    leg = Leg(torch, binding, w, dev, 0, 0, kfam)
+    stream = torch.cuda.current_stream()
+    for b in range(leg.batch):
+        leg.call(b)
+    cps = _calls_per_step(torch, stream, leg, steps, False)
+    sampler = ClockSampler(local)
+    l0 = binding.launch_count()
+    ms = _timed(torch, stream, lambda i: leg.call(i % leg.batch), steps * cps, sampler)
+    launches, calls = binding.launch_count() - l0, steps * cps
+    kernel_name = binding.last_kernel_name()
+    parity = leg.parity()
+    ms_ip = _timed(torch, stream, lambda i: leg.call_in_place(i % leg.batch), max(leg.batch, calls // 2))
+    roof = _roofline(leg.set_bytes, launches, calls, ms, kernel_name, name)
+    out = {"workload": name, "kernel": kernel_name, "calls": calls, "region_ms": ms, "avg_launch_us": roof["avg_launch_us"],
+           "value": calls * leg.set_bytes / (ms * 1e-3) / 1e9, "achieved": roof["achieved"], "frac": roof["frac"],
+           "frac_of_nominal_8000": roof["frac_of_nominal_8000"], "traffic": roof["traffic"],
+           "in_place_trv_allreduce_us": ms_ip * 1e3 / max(leg.batch, calls // 2), "parity_spot_check": parity,
+           "clocks": sampler.report("sampled during the timed region")}
+    leg.free()
+    return out
+
+
+def _e2e(torch, binding, leg, dev, steps, world):
+    """End to end through trv_allreduce_host: pinned host vectors in, pinned host vectors out (in place on the host),
+    every step; plus the rate of plain pinned copies of the same bytes in both directions at once, as the ceiling."""
+    import psutil
+    w, n = leg.w, leg.w.n
+    count = w.count
+    budget = int(psutil.virtual_memory().available * 0.5 / max(1, world))
+    if n * count * 4 > budget:          # a node too small to pin the whole set per GPU: a prefix of the columns
+        count = max(4096, budget // (4 * n) // 4096 * 4096)
+    sets = 1 if n * count * 4 >= 2**30 else min(leg.batch, 4)
+    host = [torch.empty((n, count), dtype=leg.tdt, pin_memory=True) for _ in range(sets)]
+    for b in range(sets):
+        host[b].copy_(leg.ins[b][:, :count])
+    ptrs = [binding.ptr_array([host[b][r].data_ptr() for r in range(n)]) for b in range(sets)]
+    wsb = leg.plan.host_workspace_bytes(count)
+    ws = torch.empty(wsb, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(_):
+        for b in range(sets):
+            leg.plan.allreduce_host(ptrs[b], None, count, leg.dcode, ws.data_ptr(), wsb, stream.cuda_stream)
+
+    step(0)                                     # first call: from the inputs; checked against the device path
+    torch.cuda.synchronize()
+    ok = None
+    if count == w.count:
+        ok = True
+        for r0 in range(0, n, 27):
+            up = host[0][r0:r0 + 27].to(dev, non_blocking=True)
+            ok = ok and bool(torch.equal(up.view(torch.int32), leg.outs[0][r0:r0 + 27].view(torch.int32)))
+    step(0)
+    steps = max(1, min(steps, 10 if sets > 1 else 5))
+    ms = _timed(torch, stream, step, steps)
+    nbytes = sets * n * count * 4
+    # ceiling: the same bytes up and down at once as plain copies between pinned memory and the device
+    chunk = min(n, max(1, (128 << 20) // (count * 4)))
+    dbuf = [torch.empty((chunk, count), dtype=leg.tdt, device=dev) for _ in range(2)]
+    s_up, s_dn = torch.cuda.Stream(), torch.cuda.Stream()
+
+    def copies(_):
+        s_up.wait_stream(stream)
+        s_dn.wait_stream(stream)
+        for b in range(sets):
+            for r0 in range(0, n, chunk):
+                r1 = min(n, r0 + chunk)
+                with torch.cuda.stream(s_up):
+                    dbuf[0][:r1 - r0].copy_(host[b][r0:r1], non_blocking=True)
+                with torch.cuda.stream(s_dn):
+                    host[b][r0:r1].copy_(dbuf[1][:r1 - r0], non_blocking=True)
+        stream.wait_stream(s_up)
+        stream.wait_stream(s_dn)
+
+    copies(0)
+    ms_copy = _timed(torch, stream, copies, 2) / 2
+    return {"value": world * steps * nbytes / (ms * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": nbytes,
+            "d2h_bytes_per_step": nbytes, "steps": steps, "ms_per_step": ms / steps,
+            "call": "trv_allreduce_host, in place on pinned host vectors (%d set%s of %d x %d elements), element-range "
+                    "windows pipelined inside the call" % (sets, "" if sets == 1 else "s", n, count),
+            "matches_device_path": ok,
+            "pinned_copy_ceiling": {"value": nbytes / (ms_copy * 1e-3) / 1e9, "unit": "GB/s",
+                                    "what": "the same bytes host->device and device->host at once, plain copies of 128 MiB"},
+            "frac_of_ceiling": (steps * nbytes / ms) / (nbytes / ms_copy)}
+
+
 def run_ours(args, w):
     import torch
     from paper_2602_17254_b200 import binding, build
@@ -214,54 +405,29 @@ def run_ours(args, w):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    n, count = w.n, w.count
-    set_bytes = n * count * 4
-    batch = args.batch or max(1, min(64, max(16, -(-4 * L2_BYTES // set_bytes)), (24 * 2**30) // set_bytes))   # >= 4x L2 per step
-    tdt = torch.int32 if w.dist == "int32" else torch.float32
-    dcode = binding.INT32 if w.dist == "int32" else binding.FLOAT32
-    plan = binding.Plan(w.dims, w.variant)
-
-    # synthetic inputs: set 0 is the workload's seeded vectors (and feeds the parity spot check);
-    # the other sets are the same recipe with other seeds (rank- and set-specific)
-    x0 = synth.workload_inputs(w) if set_bytes <= 2**31 else None
-    ins = torch.empty((batch, n, count), dtype=tdt, device=dev)
-    outs = torch.empty((batch, n, count), dtype=tdt, device=dev)
-    if x0 is not None:
-        ins[0].copy_(torch.from_numpy(x0))
-        g = torch.Generator(device=dev)
-        g.manual_seed(1000 * w.seed + rank)
-        for b in range(1, batch):
-            if w.dist == "int32":
-                ins[b].copy_(torch.randint(-1000, 1001, (n, count), generator=g, device=dev, dtype=tdt))
-            elif w.dist == "normal":
-                ins[b].normal_(generator=g)
-            else:
-                ins[b].uniform_(-1.0, 1.0, generator=g)
-    else:   # multi-GiB sets: drawn on the device (values do not influence the run time)
-        g = torch.Generator(device=dev)
-        g.manual_seed(1000 * w.seed + rank)
-        for b in range(batch):
-            ins[b].normal_(generator=g) if w.dist == "normal" else ins[b].uniform_(-1.0, 1.0, generator=g)
-    in_ptrs = [binding.ptr_array([ins[b, r].data_ptr() for r in range(n)]) for b in range(batch)]
-    out_ptrs = [binding.ptr_array([outs[b, r].data_ptr() for r in range(n)]) for b in range(batch)]
     kfam = {"auto": binding.KERNEL_AUTO, "step": binding.KERNEL_STEP, "fused": binding.KERNEL_FUSED,
             "pipelined": binding.KERNEL_PIPELINED}[args.kernel]
-    need = plan.scratch_bytes(count, kfam, in_place=False)
-    scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    leg = Leg(torch, binding, w, dev, rank, args.batch, kfam)
+    n, count, batch, set_bytes = w.n, w.count, leg.batch, leg.set_bytes
     stream = torch.cuda.current_stream()
-    sh = stream.cuda_stream
-
-    def step():
-        for b in range(batch):
-            plan.allreduce_ex(in_ptrs[b], out_ptrs[b], count, dcode, kernel=kfam,
-                              scratch_ptr=scratch.data_ptr() if need else 0, scratch_bytes=need,
-                              stream=torch.cuda.current_stream().cuda_stream)
 
     def barrier():
         torch.cuda.synchronize()
         if dist is not None:
             dist.barrier()
             torch.cuda.synchronize()
+
+    for b in range(batch):
+        leg.call(b)
+    cps = _calls_per_step(torch, stream, leg, args.steps, args.profile or args.graph or args.batch)
+    if dist is not None:        # every rank runs the same number of calls
+        t = torch.tensor([cps], dtype=torch.int64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        cps = int(t[0])
+
+    def step():
+        for i in range(cps):
+            leg.call(i % batch)
 
     for _ in range(args.warmup):
         step()
@@ -287,106 +453,61 @@ def run_ours(args, w):
         step()
     ev1.record(stream)
     barrier()
+    sampler.stop()
     launches = binding.launch_count() - l0
     if launches_per_step is not None:
         launches = launches_per_step * args.steps       # replayed launches are not seen by the library's counter
     ms = ev0.elapsed_time(ev1)
-    note = "sampled during the timed region"
-    if len(sampler.samples) < 8 and not args.profile:        # region too short for NVML: keep the same load running ~0.4 s more
-        t_end = time.perf_counter() + 0.4
-        while time.perf_counter() < t_end:
-            step()
-            torch.cuda.synchronize()
-        note = "timed region (%.1f ms) plus 0.4 s of the same load right after it" % ms
-    sampler.stop()
 
-    # parity spot check of what was just timed: set 0's output against the oracle on a window
-    parity = None
-    if rank == 0 and x0 is not None and not args.no_check:
-        import oracle
-        w1 = min(count, 4096)
-        want = oracle.allreduce(w.dims, w.variant, np.ascontiguousarray(x0[:, :w1]), E=count, e0=0)
-        got = outs[0, :, :w1].cpu().numpy()
-        parity = bool(np.array_equal(got.view(np.uint32), want.view(np.uint32)))
-
-    # end to end through the host-buffer entry point: pinned host inputs -> device -> host outputs,
-    # two streams so that one set's upload overlaps the previous set's download
-    do_e2e = not args.no_e2e and set_bytes <= 4 * 2**30
-    e2e_sets = min(batch, 4) if do_e2e else 0
-    hin = [torch.empty((n, count), dtype=tdt).pin_memory() for _ in range(e2e_sets)]
-    hout = [torch.empty((n, count), dtype=tdt).pin_memory() for _ in range(e2e_sets)]
-    for b in range(e2e_sets):
-        hin[b].copy_(ins[b])
-    wsb = plan.host_workspace_bytes(count)
-    ws = [torch.empty(wsb, dtype=torch.uint8, device=dev) for _ in range(2)]
-    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
-    hin_p = [binding.ptr_array([hin[b][r].data_ptr() for r in range(n)]) for b in range(e2e_sets)]
-    hout_p = [binding.ptr_array([hout[b][r].data_ptr() for r in range(n)]) for b in range(e2e_sets)]
-
-    def e2e_step():
-        for b in range(e2e_sets):
-            plan.allreduce_host(hin_p[b], hout_p[b], count, dcode, ws[b % 2].data_ptr(), wsb, streams[b % 2].cuda_stream)
-
-    e2e_steps = max(1, min(args.steps, 10))
-    e2e_ms, e2e_ok = 0.0, None
-    if do_e2e:
-        for _ in range(2):
-            e2e_step()
-        barrier()
-        e0, e1, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True), torch.cuda.Event()
-        streams[1].wait_stream(streams[0])
-        e0.record(streams[0])
-        streams[1].wait_event(e0)
-        for _ in range(e2e_steps):
-            e2e_step()
-        eb.record(streams[1])
-        streams[0].wait_event(eb)
-        e1.record(streams[0])
-        barrier()
-        e2e_ms = e0.elapsed_time(e1)
-        if parity is not None:
-            e2e_ok = bool(torch.equal(hout[0].view(torch.int32), outs[0].cpu().view(torch.int32)))
+    parity = leg.parity() if rank == 0 and not args.no_check else None
+    e2e = None
+    if not args.no_e2e:             # before the in-place leg: it compares with the outputs of the timed calls
+        e2e = _e2e(torch, binding, leg, dev, args.steps, world)
+    in_place_us = None
+    if not args.profile:
+        reps = max(batch, (args.steps * cps) // 2)
+        in_place_us = _timed(torch, stream, lambda i: leg.call_in_place(i % batch), reps) * 1e3 / reps
+    barrier()
 
     # max over ranks, sums over ranks
-    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
+    t = torch.tensor([ms, e2e["ms_per_step"] if e2e else 0.0], dtype=torch.float64, device=dev)
     cnt = torch.tensor([float(launches)], dtype=torch.float64, device=dev)
     if dist is not None:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dist.all_reduce(cnt, op=dist.ReduceOp.SUM)
-    ms, e2e_ms = float(t[0]), float(t[1])
+    ms = float(t[0])
+    if e2e:
+        e2e["value"] *= e2e["ms_per_step"] / float(t[1])
+        e2e["ms_per_step"] = float(t[1])
     launches_all = int(cnt[0])
+    leg.free()
 
     if rank == 0:
-        calls = args.steps * batch
-        value = world * calls * set_bytes / (ms * 1e-3) / 1e9
-        per_launch_ms = ms / launches                                          # this rank's launches
-        kernels_per_call = launches / calls
-        algo_bytes = 2 * set_bytes / kernels_per_call                         # per launch of the dominant kernel
-        peak, peak_src = _peak()
-        achieved = algo_bytes / (per_launch_ms * 1e-3) / 1e9
-        e2e_value = world * e2e_steps * e2e_sets * set_bytes / (e2e_ms * 1e-3) / 1e9 if do_e2e else None
+        calls = args.steps * cps
         out = {
-            "metric": "allreduce_effective_GBps", "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "int32" if w.dist == "int32" else "f32", "data": "synthetic",
+            "metric": "allreduce_effective_GBps", "value": world * calls * set_bytes / (ms * 1e-3) / 1e9, "unit": "GB/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int32" if w.dist == "int32" else "f32", "data": "synthetic",
             "config": {"workload": w.name, "dims": list(w.dims), "variant": "latency" if w.variant == 0 else "bandwidth",
-                       "ranks": n, "bytes_per_rank": w.bytes_per_rank, "calls_per_step": batch,
-                       "l2": "each step touches %d distinct buffer sets = %.0f MiB read + %.0f MiB written (L2 is 126 MiB): "
-                             "inputs larger than L2, no flush" % (batch, batch * set_bytes / 2**20, batch * set_bytes / 2**20),
-                       "kernel": kernel_name, "call": "trv_allreduce_ex, separate output buffers, TRV_KERNEL_%s" % args.kernel.upper()
+                       "ranks": n, "bytes_per_rank": w.bytes_per_rank, "calls_per_step": cps, "buffer_sets": batch,
+                       "l2": "consecutive calls run on %d distinct buffer set%s; one pass over them reads %.0f MiB and writes "
+                             "%.0f MiB (L2 is 126 MiB): inputs larger than L2, no flush"
+                             % (batch, "" if batch == 1 else "s", batch * set_bytes / 2**20, batch * set_bytes / 2**20),
+                       "timed_region_ms": ms, "kernel": kernel_name,
+                       "call": "trv_allreduce_ex, separate output buffers, TRV_KERNEL_%s" % args.kernel.upper()
                        + (", one step captured in a CUDA graph and replayed" if args.graph else ""),
                        "parallelism": "replicas" if world > 1 else "single GPU"},
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": _traffic(kernel_name, w.name), "peak_source": peak_src,
-                         "algorithmic_bytes_per_launch": algo_bytes, "avg_launch_us": per_launch_ms * 1e3,
-                         "frac_of_nominal_8000": achieved / 8000.0},
-            "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": e2e_sets * set_bytes,
-                    "d2h_bytes_per_step": e2e_sets * set_bytes, "steps": e2e_steps,
-                    "call": "trv_allreduce_host on pinned host buffers, two streams", "matches_device_path": e2e_ok},
+            "roofline": _roofline(set_bytes, launches, calls, ms, kernel_name, w.name),
+            "e2e": e2e if e2e else {"value": None, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": launches_all,
-            "clocks": sampler.report(note),
+            "clocks": sampler.report("sampled during the timed region"),
             "parity_spot_check": parity,
+            "in_place_trv_allreduce_us": in_place_us,
         }
+        if world == 1 and not args.no_side and not args.profile:
+            out["per_workload"] = [_side_leg(torch, binding, name, dev, local, args.steps, kfam)
+                                   for name in PER_WORKLOAD if name != w.name]
         if not args.no_cpu and world == 1:
             out["cpu_baseline"] = cpu_baseline(w)
         elif not args.no_cpu:
@@ -408,6 +529,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-check", action="store_true", help="skip the parity spot check")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--no-side", action="store_true", help="skip the per_workload legs of the other configurations")
     ap.add_argument("--dims", default="", help="ad-hoc torus sides, e.g. 27,27 (overrides the workload's topology)")
     ap.add_argument("--variant", default="latency", choices=["latency", "bandwidth"], help="form for --dims")
     ap.add_argument("--kernel", default="auto", choices=["auto", "step", "fused", "pipelined"],
@@ -419,10 +541,12 @@ def main():
                     help="for runs under ncu: only warm-up and timed launches (implies --no-cpu --no-check --no-e2e)")
     args = ap.parse_args()
     if args.profile:
-        args.no_cpu = args.no_check = args.no_e2e = True
+        args.no_cpu = args.no_check = args.no_e2e = args.no_side = True
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     w = synth.CONFIGS[args.workload]
+    if args.dims or args.count or args.workload != DEFAULT_WORKLOAD or args.kernel != "auto" or args.graph:
+        args.no_side = True         # per_workload belongs to the default run only
     if args.dims:       # ad-hoc topology: same recipe (float32 N(0,1)), for shapes outside the named configurations
         dims = tuple(int(v) for v in args.dims.split(","))
         variant = synth.LATENCY if args.variant == "latency" else synth.BANDWIDTH
