@@ -154,6 +154,7 @@ class ClockSampler:
 
     def __init__(self, index):
         self.samples, self.reason_bits, self.max_mhz, self._stop, self._thr, self._h = [], 0, None, threading.Event(), None, None
+        self.power = []
         try:
             import pynvml
             pynvml.nvmlInit()
@@ -173,6 +174,10 @@ class ClockSampler:
         while not self._stop.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    self.power.append(nv.nvmlDeviceGetPowerUsage(self._h) / 1e3)
+                except Exception:
+                    pass
                 try:
                     self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
                 except Exception:
@@ -198,7 +203,7 @@ class ClockSampler:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "note": "NVML unavailable"}
         reasons = [name for bit, name in self.REASONS.items() if self.reason_bits & bit]
         return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz, "reasons": reasons,
-                "samples": len(self.samples), "note": note}
+                "samples": len(self.samples), "power_w": float(np.median(self.power)) if self.power else None, "note": note}
 
 
 # ------------------------------------------------------------------ GPU legs
@@ -280,6 +285,23 @@ def _timed(torch, stream, fn, reps, sampler=None):
     return ev0.elapsed_time(ev1)
 
 
+def _timed_in_place(torch, stream, leg, reps):
+    """Microseconds per in-place trv_allreduce call.  Every call runs on fresh inputs (set b's outputs are refilled from
+    its inputs first, untimed): repeated in place on its own results the data would overflow to inf/NaN within a dozen
+    calls, and such data draws less power than the workload's."""
+    pairs = []
+    for i in range(reps):
+        b = i % leg.batch
+        leg.outs[b].copy_(leg.ins[b])
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        leg.call_in_place(b)
+        e1.record(stream)
+        pairs.append((e0, e1))
+    torch.cuda.synchronize()
+    return sum(a.elapsed_time(b) for a, b in pairs) * 1e3 / reps
+
+
 def _calls_per_step(torch, stream, leg, steps, fixed):
     """Calls per step: a whole number of passes over the batch, enough for a timed region of MIN_REGION_S."""
     if fixed:
@@ -313,12 +335,12 @@ def _side_leg(torch, binding, name, dev, local, steps, kfam):
     launches, calls = binding.launch_count() - l0, steps * cps
     kernel_name = binding.last_kernel_name()
     parity = leg.parity()
-    ms_ip = _timed(torch, stream, lambda i: leg.call_in_place(i % leg.batch), max(leg.batch, calls // 2))
+    us_ip = _timed_in_place(torch, stream, leg, max(leg.batch, min(200, calls // 2)))
     roof = _roofline(leg.set_bytes, launches, calls, ms, kernel_name, name)
     out = {"workload": name, "kernel": kernel_name, "calls": calls, "region_ms": ms, "avg_launch_us": roof["avg_launch_us"],
            "value": calls * leg.set_bytes / (ms * 1e-3) / 1e9, "achieved": roof["achieved"], "frac": roof["frac"],
            "frac_of_nominal_8000": roof["frac_of_nominal_8000"], "traffic": roof["traffic"],
-           "in_place_trv_allreduce_us": ms_ip * 1e3 / max(leg.batch, calls // 2), "parity_spot_check": parity,
+           "in_place_trv_allreduce_us": us_ip, "parity_spot_check": parity,
            "clocks": sampler.report("sampled during the timed region")}
     leg.free()
     return out
@@ -465,8 +487,7 @@ def run_ours(args, w):
         e2e = _e2e(torch, binding, leg, dev, args.steps, world)
     in_place_us = None
     if not args.profile:
-        reps = max(batch, (args.steps * cps) // 2)
-        in_place_us = _timed(torch, stream, lambda i: leg.call_in_place(i % batch), reps) * 1e3 / reps
+        in_place_us = _timed_in_place(torch, stream, leg, max(batch, min(200, (args.steps * cps) // 2)))
     barrier()
 
     # max over ranks, sums over ranks
