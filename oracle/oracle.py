@@ -73,6 +73,21 @@ def _general_ring(dims, algo=ALGO_TRIVANCE):
     return int(a[0]) if n != 1 else 0
 
 
+def _general_torus(dims, algo=ALGO_TRIVANCE):
+    """True if dims is a torus of two or more dimensions with a side that is no power of three (Sec. 4.4 + Sec. 5)."""
+    a = np.atleast_1d(np.asarray(dims)).reshape(-1)
+    if algo != ALGO_TRIVANCE or a.size < 2:
+        return False
+
+    def pow3(v):
+        v = int(v)
+        while v > 1 and v % 3 == 0:
+            v //= 3
+        return v == 1 and int(v) >= 1
+
+    return any(int(v) < 3 or not pow3(v) for v in a)
+
+
 def num_steps(dims, algo=ALGO_TRIVANCE):
     """(n, steps per phase) of the schedule on a torus with these dimensions."""
     _, p, nd = _dims(dims)
@@ -150,6 +165,10 @@ def allreduce(dims, variant, x, E=None, e0=0, max_steps=-1, counters=False):
         if variant != VARIANT_BANDWIDTH or max_steps >= 0:
             raise OracleError(2)
         return gen_allreduce(x, E=E, e0=e0, counters=counters)
+    if _general_torus(dims):
+        if variant != VARIANT_BANDWIDTH or max_steps >= 0:
+            raise OracleError(2)
+        return gent_allreduce(dims, x, E=E, e0=e0, counters=counters)
     x = np.ascontiguousarray(x)
     if x.dtype not in _DTYPES or x.ndim != 2:
         raise TypeError("x must be a 2-D int32, float32 or float64 array")
@@ -177,6 +196,10 @@ def link_loads(dims, variant, E, elem_size=4, algo=ALGO_TRIVANCE):
         if variant != VARIANT_BANDWIDTH:
             raise OracleError(2)
         return gen_link_loads(_general_ring(dims, algo), E, elem_size)
+    if _general_torus(dims, algo):
+        if variant != VARIANT_BANDWIDTH:
+            raise OracleError(2)
+        return gent_link_loads(dims, E, elem_size)
     a, p, nd = _dims(dims)
     n, s = num_steps(dims, algo)
     T = 2 * s if variant == VARIANT_BANDWIDTH else s
@@ -198,6 +221,10 @@ def bytes_sent(dims, variant, E, elem_size=4, algo=ALGO_TRIVANCE):
         if variant != VARIANT_BANDWIDTH:
             raise OracleError(2)
         return gen_link_loads(_general_ring(dims, algo), E, elem_size)["sent"]
+    if _general_torus(dims, algo):
+        if variant != VARIANT_BANDWIDTH:
+            raise OracleError(2)
+        return gent_link_loads(dims, E, elem_size)["sent"]
     _, p, nd = _dims(dims)
     n, _ = num_steps(dims, algo)
     out = np.zeros(n, np.int64)
@@ -210,7 +237,7 @@ def cost_model(dims, variant, E, elem_size, alpha, beta, algo=ALGO_TRIVANCE):
     """Sec. 2.1: C = steps * alpha + sum_k beta * m_k * c_k, with m_k * c_k = bytes on the most loaded
     link of step k; plus the optimality factors of Tables 1 and 2 (lambda, delta, theta)."""
     ll = link_loads(dims, variant, E, elem_size, algo)
-    n = _general_ring(dims, algo) or num_steps(dims, algo)[0]
+    n = _general_ring(dims, algo) or (gent_num_steps(dims)[0] if _general_torus(dims, algo) else num_steps(dims, algo)[0])
     T = ll["max_bytes"].size
     tx = int(ll["max_bytes"].sum())
     sent = int(bytes_sent(dims, variant, E, elem_size, algo).max())
@@ -271,4 +298,74 @@ def gen_link_loads(n, E, elem_size=4):
                                       msgs.ctypes.data_as(ctypes.c_void_p), byts.ctypes.data_as(ctypes.c_void_p),
                                       mm.ctypes.data_as(ctypes.c_void_p), mb.ctypes.data_as(ctypes.c_void_p),
                                       sent.ctypes.data_as(ctypes.c_void_p)))
+    return {"msgs": msgs, "bytes": byts, "max_msgs": mm, "max_bytes": mb, "sent": sent}
+
+
+# ------------------------------------------------------------------ tori with sides of any size (Sec. 4.4 + Sec. 5)
+
+def gent_num_steps(dims):
+    """(n, S): ranks and steps per phase (sum over dimensions of ceil(log3 side))."""
+    _, p, nd = _dims(dims)
+    n, s = ctypes.c_int(), ctypes.c_int()
+    _check(_load().orc_gent_num_steps(p, nd, ctypes.byref(n), ctypes.byref(s)))
+    return n.value, s.value
+
+
+def gent_step_list(dims, c=0):
+    """[(dim, dist), ...] of collective c: round-robin over the dimensions from c, each dimension's ring distances in order."""
+    _, p, nd = _dims(dims)
+    _, S = gent_num_steps(dims)
+    d = np.zeros(S, np.int32)
+    x = np.zeros(S, np.int32)
+    _check(_load().orc_gent_step_list(p, nd, ctypes.c_int(c), d.ctypes.data_as(ctypes.c_void_p), x.ctypes.data_as(ctypes.c_void_p)))
+    return [(int(a), int(b)) for a, b in zip(d, x)]
+
+
+def gent_tree(dims, c=0):
+    """(par, stp), both [n][n], of collective c: par[b][v] = node v gets block b from, stp[b][v] = in which of its steps."""
+    _, p, nd = _dims(dims)
+    n, _ = gent_num_steps(dims)
+    par = np.zeros((n, n), np.int32)
+    stp = np.zeros((n, n), np.int32)
+    _check(_load().orc_gent_tree(p, nd, ctypes.c_int(c), par.ctypes.data_as(ctypes.c_void_p), stp.ctypes.data_as(ctypes.c_void_p)))
+    return par, stp
+
+
+def gent_allreduce(dims, x, E=None, e0=0, counters=False):
+    """Bandwidth-optimal Trivance AllReduce on a torus with sides of any size >= 2; as ``allreduce``."""
+    x = np.ascontiguousarray(x)
+    if x.dtype not in _DTYPES or x.ndim != 2:
+        raise TypeError("x must be a 2-D int32, float32 or float64 array")
+    n, w = x.shape
+    nn, _ = gent_num_steps(dims)
+    if n != nn:
+        raise ValueError("x has %d rows, the topology has %d ranks" % (n, nn))
+    if E is None:
+        E = w
+    out = np.empty_like(x)
+    _, p, nd = _dims(dims)
+    ctr = [np.zeros(n, np.int64) for _ in range(3)] if counters else [None] * 3
+    ptr = [c.ctypes.data_as(ctypes.c_void_p) if c is not None else None for c in ctr]
+    _check(_load().orc_gent_allreduce(p, nd, ctypes.c_int(_DTYPES[x.dtype]), ctypes.c_int64(E), ctypes.c_int64(e0),
+                                      ctypes.c_int64(e0 + w), x.ctypes.data_as(ctypes.c_void_p),
+                                      out.ctypes.data_as(ctypes.c_void_p), *ptr))
+    if counters:
+        return out, {"sent_rs": ctr[0], "sent_ag": ctr[1], "reduced": ctr[2]}
+    return out
+
+
+def gent_link_loads(dims, E, elem_size=4):
+    """Link loads of that schedule: msgs/bytes [2S][n][D][2], max_msgs/max_bytes [2S], sent [n]."""
+    a, p, nd = _dims(dims)
+    n, S = gent_num_steps(dims)
+    T, D = 2 * S, a.size
+    msgs = np.zeros((T, n, D, 2), np.int32)
+    byts = np.zeros((T, n, D, 2), np.int64)
+    mm = np.zeros(T, np.int32)
+    mb = np.zeros(T, np.int64)
+    sent = np.zeros(n, np.int64)
+    _check(_load().orc_gent_link_loads(p, nd, ctypes.c_int64(E), ctypes.c_int64(elem_size),
+                                       msgs.ctypes.data_as(ctypes.c_void_p), byts.ctypes.data_as(ctypes.c_void_p),
+                                       mm.ctypes.data_as(ctypes.c_void_p), mb.ctypes.data_as(ctypes.c_void_p),
+                                       sent.ctypes.data_as(ctypes.c_void_p)))
     return {"msgs": msgs, "bytes": byts, "max_msgs": mm, "max_bytes": mb, "sent": sent}

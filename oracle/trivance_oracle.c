@@ -856,3 +856,274 @@ done:
     free(par); free(stp); free(lm); free(lb); free(mb); free(mc);
     return rc;
 }
+
+/* ------------------------------------------------------------------ tori with sides of any size (Sec. 4.4 + Sec. 5) */
+
+/*
+ * Bandwidth-optimal Trivance on a D-dimensional torus whose sides a_d >= 2 need not be powers of three.
+ *
+ * What the paper fixes: Sec. 5 runs one collective per dimension on 1/D of the vector, each collective on a
+ * different dimension in every step; Sec. 4.4 gives a ring of any size its step list (the regular distances,
+ * then one step at distance ceil((a - 3^floor(log3 a)) / 2)) and says that every block is forwarded at most
+ * once per phase.  The paper evaluates such tori (32 x 32, 8 x 64, 16 x 16 x 16) without spelling the
+ * combination out.
+ *
+ * Reading (PARITY UNPINNED by the paper): the two rules are composed literally.
+ *   - Step list of collective c: the dimensions in round-robin order starting at c, a dimension that has used
+ *     up its ceil(log3 a_d) steps being skipped; the k-th visit of dimension d uses the k-th distance of the
+ *     ring of a_d nodes.  S = sum_d ceil(log3 a_d) steps per phase.
+ *   - Block b is owned by linear rank b.  Its AllGather runs the steps in reverse; the nodes holding it are
+ *     kept in the order they got it; in a step along dimension d every holder, in that order, offers it to
+ *     the node `dist` before it along d, then to the node `dist` after it; a node that holds it already is
+ *     skipped.  The Reduce-Scatter runs the same tree backwards with (from_left + own) + from_right.
+ * For sides that are powers of three nothing is ever skipped and this is the regular schedule of Sec. 5.
+ */
+typedef struct {
+    int ndims, n, S;
+    int dims[ORC_MAX_DIMS], stride[ORC_MAX_DIMS];
+    int nd[ORC_MAX_DIMS];               /* steps of dimension d */
+    int ddist[ORC_MAX_DIMS][32];        /* its distances */
+} gent_topo;
+
+static int gent_init(gent_topo *g, const int32_t *dims, int ndims) {
+    if (!dims || ndims < 1 || ndims > ORC_MAX_DIMS) return ORC_BAD_ARG;
+    long long n = 1;
+    g->ndims = ndims; g->S = 0;
+    for (int d = 0; d < ndims; ++d) {
+        if (dims[d] < 2 || dims[d] > 4096) return ORC_BAD_ARG;
+        g->dims[d] = dims[d]; g->stride[d] = (int)n;
+        g->nd[d] = gen_steps(dims[d], g->ddist[d]);
+        g->S += g->nd[d];
+        n *= dims[d];
+        if (n > 4096) return ORC_BAD_ARG;
+    }
+    g->n = (int)n;
+    return ORC_OK;
+}
+
+static void gent_step_list(const gent_topo *g, int c, int *sdim, int *sdist) {
+    int visits[ORC_MAX_DIMS] = {0};
+    int cur = c % g->ndims;
+    for (int t = 0; t < g->S; ++t) {
+        int d = cur;
+        while (visits[d] >= g->nd[d]) d = (d + 1) % g->ndims;
+        sdim[t] = d; sdist[t] = g->ddist[d][visits[d]];
+        visits[d]++;
+        cur = (d + 1) % g->ndims;
+    }
+}
+
+static int gent_shift(const gent_topo *g, int r, int d, int delta) {
+    int a = g->dims[d], st = g->stride[d];
+    int x = (r / st) % a, y = ((x + delta) % a + a) % a;
+    return r + (y - x) * st;
+}
+
+/* par[b*n+v] = the node v gets block b from (-1 for v = b); stp[b*n+v] = the step (of collective c) in which */
+static int gent_build(const gent_topo *g, const int *sdim, const int *sdist, int32_t *par, int32_t *stp) {
+    int n = g->n, rc = ORC_OK;
+    int *list = (int *)malloc(sizeof(int) * (size_t)n);
+    uint8_t *have = (uint8_t *)malloc((size_t)n);
+    if (!list || !have) { free(list); free(have); return ORC_NOMEM; }
+    for (int b = 0; b < n && rc == ORC_OK; ++b) {
+        int len = 1;
+        memset(have, 0, (size_t)n);
+        list[0] = b; have[b] = 1; par[(size_t)b * n + b] = -1; stp[(size_t)b * n + b] = -1;
+        for (int t = g->S - 1; t >= 0; --t) {
+            int len0 = len;
+            for (int i = 0; i < len0; ++i) {
+                int h = list[i];
+                for (int side = 0; side < 2; ++side) {
+                    int v = gent_shift(g, h, sdim[t], side ? sdist[t] : -sdist[t]);
+                    if (have[v]) continue;
+                    have[v] = 1; par[(size_t)b * n + v] = h; stp[(size_t)b * n + v] = t; list[len++] = v;
+                }
+            }
+        }
+        if (len != n) rc = ORC_INTERNAL;
+    }
+    free(list); free(have);
+    return rc;
+}
+
+int orc_gent_num_steps(const int32_t *dims, int ndims, int *n_out, int *S_out) {
+    gent_topo g; int rc = gent_init(&g, dims, ndims);
+    if (rc) return rc;
+    if (n_out) *n_out = g.n;
+    if (S_out) *S_out = g.S;
+    return ORC_OK;
+}
+
+int orc_gent_step_list(const int32_t *dims, int ndims, int c, int32_t *dim_out, int32_t *dist_out) {
+    gent_topo g; int rc = gent_init(&g, dims, ndims);
+    if (rc) return rc;
+    if (c < 0 || c >= ndims || !dim_out || !dist_out) return ORC_BAD_ARG;
+    int sd[256], sx[256];
+    gent_step_list(&g, c, sd, sx);
+    for (int t = 0; t < g.S; ++t) { dim_out[t] = sd[t]; dist_out[t] = sx[t]; }
+    return ORC_OK;
+}
+
+int orc_gent_tree(const int32_t *dims, int ndims, int c, int32_t *par, int32_t *stp) {
+    gent_topo g; int rc = gent_init(&g, dims, ndims);
+    if (rc) return rc;
+    if (c < 0 || c >= ndims || !par || !stp) return ORC_BAD_ARG;
+    int sd[256], sx[256];
+    gent_step_list(&g, c, sd, sx);
+    return gent_build(&g, sd, sx, par, stp);
+}
+
+/* One collective (slice [slo, shi) of the global vector) on the window [e0, e1); arrays are [n][w], w = e1 - e0. */
+#define DEFINE_GENT(T, SUFFIX, ADD)                                                                         \
+static int gent_slice_##SUFFIX(const gent_topo *g, const int *sdim, const int *sdist, const int32_t *par,   \
+                               const int32_t *stp, int64_t slo, int64_t shi, int64_t e0, int64_t e1,        \
+                               T *partial, T *msg, orc_counters *ctr) {                                     \
+    int n = g->n, S = g->S;                                                                                 \
+    int64_t w = e1 - e0;                                                                                    \
+    int64_t *bs = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n + 1));                                     \
+    if (!bs) return ORC_NOMEM;                                                                              \
+    for (int j = 0; j <= n; ++j) bs[j] = clampi(block_bound(slo, shi, n, j), e0, e1) - e0;                  \
+    if (bs[n] <= bs[0]) { free(bs); return ORC_OK; }                                                        \
+    /* ---- Reduce-Scatter: every node first puts its current partials on the wire, then all receive */   \
+    for (int t = 0; t < S; ++t) {                                                                           \
+        for (int p = 0; p < n; ++p)                                                                         \
+            memcpy(msg + (size_t)p * w + bs[0], partial + (size_t)p * w + bs[0], sizeof(T) * (size_t)(bs[n] - bs[0])); \
+        for (int b = 0; b < n; ++b) {                                                                       \
+            int64_t bl = bs[b + 1] - bs[b];                                                                 \
+            for (int p = 0; p < n; ++p) {                                                                   \
+                int ql = gent_shift(g, p, sdim[t], -sdist[t]), qr = gent_shift(g, p, sdim[t], sdist[t]);    \
+                int hl = (stp[(size_t)b * n + ql] == t && par[(size_t)b * n + ql] == p);                    \
+                int hr = (qr != ql && stp[(size_t)b * n + qr] == t && par[(size_t)b * n + qr] == p);        \
+                if (!hl && !hr) continue;                                                                   \
+                T *own = partial + (size_t)p * w + bs[b];                                                   \
+                const T *ml = msg + (size_t)ql * w + bs[b], *mr = msg + (size_t)qr * w + bs[b];             \
+                for (int64_t e = 0; e < bl; ++e) {                                                          \
+                    T acc = own[e];                                                                         \
+                    if (hl) acc = ADD(ml[e], acc);                                                          \
+                    if (hr) acc = ADD(acc, mr[e]);                                                          \
+                    own[e] = acc;                                                                           \
+                }                                                                                           \
+                if (ctr && ctr->sent_rs) {                                                                  \
+                    if (hl) ctr->sent_rs[ql] += (int64_t)sizeof(T) * bl;                                    \
+                    if (hr) ctr->sent_rs[qr] += (int64_t)sizeof(T) * bl;                                    \
+                }                                                                                           \
+                if (ctr && ctr->reduced) ctr->reduced[p] += (int64_t)sizeof(T) * bl * (1 + hl + hr);        \
+            }                                                                                               \
+        }                                                                                                   \
+    }                                                                                                       \
+    /* ---- AllGather: the same trees, root first */                                                       \
+    for (int t = S - 1; t >= 0; --t) {                                                                      \
+        for (int p = 0; p < n; ++p)                                                                         \
+            memcpy(msg + (size_t)p * w + bs[0], partial + (size_t)p * w + bs[0], sizeof(T) * (size_t)(bs[n] - bs[0])); \
+        for (int b = 0; b < n; ++b)                                                                         \
+            for (int v = 0; v < n; ++v) if (stp[(size_t)b * n + v] == t) {                                  \
+                int q = par[(size_t)b * n + v]; int64_t bl = bs[b + 1] - bs[b];                             \
+                memcpy(partial + (size_t)v * w + bs[b], msg + (size_t)q * w + bs[b], sizeof(T) * (size_t)bl);\
+                if (ctr && ctr->sent_ag) ctr->sent_ag[q] += (int64_t)sizeof(T) * bl;                        \
+            }                                                                                               \
+    }                                                                                                       \
+    free(bs);                                                                                               \
+    return ORC_OK;                                                                                          \
+}
+DEFINE_GENT(uint32_t, i32, ADD_WRAP)
+DEFINE_GENT(float, f32, ADD_FP)
+DEFINE_GENT(double, f64, ADD_FP)
+
+/* AllReduce (bandwidth-optimal form) on a torus with sides of any size >= 2; arguments as orc_allreduce. */
+int orc_gent_allreduce(const int32_t *dims, int ndims, int dtype, int64_t E, int64_t e0, int64_t e1, const void *in,
+                       void *out, int64_t *sent_rs, int64_t *sent_ag, int64_t *reduced) {
+    gent_topo g; int rc = gent_init(&g, dims, ndims);
+    if (rc) return rc;
+    if (E < 0 || e0 < 0 || e1 < e0 || e1 > E || !in || !out) return ORC_BAD_ARG;
+    if (dtype != ORC_I32 && dtype != ORC_F32 && dtype != ORC_F64) return ORC_BAD_ARG;
+    int n = g.n;
+    int64_t w = e1 - e0;
+    size_t es = dtype == ORC_F64 ? 8 : 4;
+    if (w == 0) return ORC_OK;
+    int32_t *par = (int32_t *)malloc(sizeof(int32_t) * (size_t)n * n), *stp = (int32_t *)malloc(sizeof(int32_t) * (size_t)n * n);
+    void *msg = malloc(es * (size_t)n * (size_t)w);
+    orc_counters ctr = { sent_rs, sent_ag, reduced };
+    if (!par || !stp || !msg) { free(par); free(stp); free(msg); return ORC_NOMEM; }
+    memcpy(out, in, es * (size_t)n * (size_t)w);        /* the partials live in `out` */
+    for (int c = 0; c < ndims && rc == ORC_OK; ++c) {
+        int sd[256], sx[256];
+        int64_t slo, shi;
+        slice_bounds(E, ndims, c, &slo, &shi);
+        if (clampi(shi, e0, e1) <= clampi(slo, e0, e1)) continue;
+        gent_step_list(&g, c, sd, sx);
+        rc = gent_build(&g, sd, sx, par, stp);
+        if (rc) break;
+        if (dtype == ORC_I32) rc = gent_slice_i32(&g, sd, sx, par, stp, slo, shi, e0, e1, (uint32_t *)out, (uint32_t *)msg, &ctr);
+        else if (dtype == ORC_F32) rc = gent_slice_f32(&g, sd, sx, par, stp, slo, shi, e0, e1, (float *)out, (float *)msg, &ctr);
+        else rc = gent_slice_f64(&g, sd, sx, par, stp, slo, shi, e0, e1, (double *)out, (double *)msg, &ctr);
+    }
+    free(par); free(stp); free(msg);
+    return rc;
+}
+
+/*
+ * Link loads of that schedule: rows = S Reduce-Scatter steps, then the AllGather steps in reverse order;
+ * arrays [2S][n][D][2] as in orc_link_loads (index 0: the link leaving the node towards +, 1: towards -).
+ * All blocks a node sends to one peer in one step of one collective form ONE message; it walks `dist` links
+ * along the step's dimension in its direction of travel.  sent (optional, [n]): bytes a node sends in total.
+ */
+int orc_gent_link_loads(const int32_t *dims, int ndims, int64_t E, int64_t elem_size, int32_t *msgs, int64_t *bytes,
+                        int32_t *max_msgs, int64_t *max_bytes, int64_t *sent) {
+    gent_topo g; int rc = gent_init(&g, dims, ndims);
+    if (rc) return rc;
+    if (E < 0 || elem_size < 1) return ORC_BAD_ARG;
+    int n = g.n, S = g.S, T = 2 * S, D = ndims;
+    size_t links = (size_t)n * D * 2;
+    int32_t *par = (int32_t *)malloc(sizeof(int32_t) * (size_t)n * n), *stp = (int32_t *)malloc(sizeof(int32_t) * (size_t)n * n);
+    int32_t *lm = (int32_t *)calloc((size_t)T * links, sizeof(int32_t));
+    int64_t *lb = (int64_t *)calloc((size_t)T * links, sizeof(int64_t));
+    int64_t *mb = (int64_t *)malloc(sizeof(int64_t) * (size_t)n * 2);
+    int32_t *mc = (int32_t *)malloc(sizeof(int32_t) * (size_t)n * 2);
+    if (!par || !stp || !lm || !lb || !mb || !mc) { rc = ORC_NOMEM; goto done; }
+    if (sent) memset(sent, 0, sizeof(int64_t) * (size_t)n);
+    for (int c = 0; c < D; ++c) {
+        int sd[256], sx[256];
+        int64_t slo, shi;
+        slice_bounds(E, D, c, &slo, &shi);
+        gent_step_list(&g, c, sd, sx);
+        rc = gent_build(&g, sd, sx, par, stp);
+        if (rc) goto done;
+        for (int row = 0; row < T; ++row) {
+            int t = row < S ? row : T - 1 - row, d = sd[t];
+            memset(mb, 0, sizeof(int64_t) * (size_t)n * 2); memset(mc, 0, sizeof(int32_t) * (size_t)n * 2);
+            for (int b = 0; b < n; ++b)
+                for (int v = 0; v < n; ++v) if (stp[(size_t)b * n + v] == t) {
+                    int q = par[(size_t)b * n + v];
+                    int left_child = (v == gent_shift(&g, q, d, -sx[t]));   /* tried first: also when both peers coincide */
+                    int src = row < S ? v : q;
+                    int side = row < S ? left_child : !left_child;           /* 0: travels towards -, 1: towards + */
+                    mb[(size_t)src * 2 + side] += (block_bound(slo, shi, n, b + 1) - block_bound(slo, shi, n, b)) * elem_size;
+                    mc[(size_t)src * 2 + side] += 1;
+                }
+            for (int src = 0; src < n; ++src)
+                for (int side = 0; side < 2; ++side) if (mc[(size_t)src * 2 + side]) {
+                    int cur = src;
+                    if (sent) sent[src] += mb[(size_t)src * 2 + side];
+                    for (int h = 0; h < sx[t]; ++h) {
+                        size_t li = (((size_t)row * n + cur) * D + d) * 2 + (side ? 0 : 1);
+                        lm[li] += 1; lb[li] += mb[(size_t)src * 2 + side];
+                        cur = gent_shift(&g, cur, d, side ? 1 : -1);
+                    }
+                }
+        }
+    }
+    for (int row = 0; row < T; ++row) {
+        int32_t mm = 0; int64_t mx = 0;
+        for (size_t l = 0; l < links; ++l) {
+            if (lm[(size_t)row * links + l] > mm) mm = lm[(size_t)row * links + l];
+            if (lb[(size_t)row * links + l] > mx) mx = lb[(size_t)row * links + l];
+        }
+        if (max_msgs) max_msgs[row] = mm;
+        if (max_bytes) max_bytes[row] = mx;
+    }
+    if (msgs) memcpy(msgs, lm, sizeof(int32_t) * (size_t)T * links);
+    if (bytes) memcpy(bytes, lb, sizeof(int64_t) * (size_t)T * links);
+done:
+    free(par); free(stp); free(lm); free(lb); free(mb); free(mc);
+    return rc;
+}
