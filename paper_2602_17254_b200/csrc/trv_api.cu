@@ -132,7 +132,7 @@ trv_status_t trv_plan_send_set(trv_plan_t plan, int32_t c, int32_t step, int32_t
     const Plan& p = plan->plan;
     if (c < 0 || c >= p.nslices || step < 0 || step >= p.S || dst < 0 || dst >= p.n) return TRV_ERR_INVALID_ARG;
     for (int j = 0; j < p.n; ++j)
-        set[j] = p.general ? (uint8_t)general_recv_mask(p, step, dst, j) : (in_send_set(p, c, step, dst, j) ? 1 : 0);
+        set[j] = p.general ? (uint8_t)general_recv_mask(p, c, step, dst, j) : (in_send_set(p, c, step, dst, j) ? 1 : 0);
     return TRV_OK;
 }
 

@@ -145,6 +145,50 @@ __device__ __forceinline__ V add3v(const V& a, const V& b, const V& c) {
     return r;
 }
 
+// Torus geometry for kernels that do rank arithmetic on the device (sides of any size, at most four dimensions).
+struct TorusGeo {
+    int nd;
+    int dims[4], stride[4];
+};
+inline TorusGeo make_geo(const Plan& p) {
+    TorusGeo g;
+    g.nd = p.ndims;
+    for (int d = 0; d < 4; ++d) { g.dims[d] = d < p.ndims ? p.dims[d] : 1; g.stride[d] = d < p.ndims ? p.stride[d] : p.n; }
+    return g;
+}
+// node + offset and node - offset, coordinate by coordinate modulo the sides
+__device__ __forceinline__ int geo_add(const TorusGeo& g, int r, int o) {
+    int out = 0;
+#pragma unroll
+    for (int d = 0; d < 4; ++d)
+        if (d < g.nd) {
+            int x = (r / g.stride[d]) % g.dims[d] + (o / g.stride[d]) % g.dims[d];
+            if (x >= g.dims[d]) x -= g.dims[d];
+            out += x * g.stride[d];
+        }
+    return out;
+}
+__device__ __forceinline__ int geo_sub(const TorusGeo& g, int r, int o) {
+    int out = 0;
+#pragma unroll
+    for (int d = 0; d < 4; ++d)
+        if (d < g.nd) {
+            int x = (r / g.stride[d]) % g.dims[d] - (o / g.stride[d]) % g.dims[d];
+            if (x < 0) x += g.dims[d];
+            out += x * g.stride[d];
+        }
+    return out;
+}
+// the node `delta` positions further along dimension d (|delta| < side)
+__device__ __forceinline__ int geo_shift(const TorusGeo& g, int r, int d, int delta) {
+    const int a = g.dims[d], st = g.stride[d];
+    const int x = (r / st) % a;
+    int y = x + delta;
+    if (y < 0) y += a;
+    if (y >= a) y -= a;
+    return r + (y - x) * st;
+}
+
 // step-family launchers (trv_step.cu)
 trv_status_t run_step_latency(const Call& c);
 trv_status_t run_step_bandwidth(const Call& c);

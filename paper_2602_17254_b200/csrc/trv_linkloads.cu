@@ -151,7 +151,7 @@ trv_status_t run_link_loads(const Plan& p, size_t count, size_t elem_size, int32
                 const int t = p.step_of_row(row);
                 bool any[2] = {false, false};
                 for (int o = 1; o < n; ++o)
-                    if (p.gstep[o] == t) any[(row < p.S) == (p.gsgn[o] > 0) ? 1 : 0] = true;
+                    if (p.gstep[c][o] == t) any[(row < p.S) == (p.gsgn[c][o] > 0) ? 1 : 0] = true;
                 rs.nclass = 0;
                 if (any[0]) rs.cls[rs.nclass++] = MsgClass{-1, d, -d, 0, 0, 0, 0};
                 if (any[1]) rs.cls[rs.nclass++] = MsgClass{+1, d, +d, 0, 0, 0, 1};

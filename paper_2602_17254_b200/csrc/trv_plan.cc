@@ -20,34 +20,84 @@ static int exact_log(int a, int base) {
 // Sec. 4.4 with the reading stated in the header of the C interface: the AllGather of a block runs
 // the steps in reverse order (the extra distance first); holders are kept in the order they got
 // the block; in a step each holder, in that order, offers it to its left peer, then to its right
-// peer, and a node that holds it already is skipped.  Written in offsets from the block's owner.
-static void build_general_ring(Plan& p, int n) {
+// peer, and a node that holds it already is skipped.  Written in offsets from the block's owner:
+// kstep[o] = the ring's step in which the node at offset o sends its partial on, ksgn[o] = +1 / -1 towards
+// the node after / before it.  Returns the ring's distances.
+static std::vector<int> ring_tree(int n, std::vector<int8_t>& kstep, std::vector<int8_t>& ksgn) {
     int pw = 1;
-    std::vector<Step> steps;
-    while ((long long)pw * 3 <= n) { steps.push_back(Step{0, pw}); pw *= 3; }
-    steps.push_back(Step{0, (n - pw + 1) / 2});
-    p.general = true;
-    p.nslices = 1;
-    p.S = (int)steps.size();
-    p.gstep.assign(n, -1);
-    p.gsgn.assign(n, 0);
+    std::vector<int> dist;
+    while ((long long)pw * 3 <= n) { dist.push_back(pw); pw *= 3; }
+    if (pw != n) dist.push_back((n - pw + 1) / 2);
+    const int S = (int)dist.size();
+    kstep.assign(n, -1);
+    ksgn.assign(n, 0);
     std::vector<int> order(1, 0);
     std::vector<char> held(n, 0);
     held[0] = 1;
-    for (int t = p.S - 1; t >= 0; --t) {
+    for (int t = S - 1; t >= 0; --t) {
         const size_t cnt = order.size();
         for (size_t i = 0; i < cnt; ++i)
             for (int side = 0; side < 2; ++side) {
-                const int delta = side ? steps[t].dist : -steps[t].dist;
+                const int delta = side ? dist[t] : -dist[t];
                 const int v = ((order[i] + delta) % n + n) % n;
                 if (held[v]) continue;
                 held[v] = 1;
-                p.gstep[v] = (int8_t)t;
-                p.gsgn[v] = (int8_t)(side ? -1 : +1);      // the child sends back the way the block came
+                kstep[v] = (int8_t)t;
+                ksgn[v] = (int8_t)(side ? -1 : +1);      // the child sends back the way the block came
                 order.push_back(v);
             }
     }
-    p.steps.assign(1, steps);
+    return dist;
+}
+
+// Sides of any size, one collective per dimension (Sec. 5): collective c visits the dimensions in round-robin
+// order from c, a dimension that has used up its ring's steps being skipped; the k-th visit of a dimension uses
+// its ring's k-th distance.  Along every dimension a block travels by that ring's tree, so the tree on the torus
+// is the product of the ring trees: the node at offset o gets the block once ALL its coordinates have been
+// reached, i.e. in the AllGather step that reaches the last of them; as the AllGather runs the step list
+// backwards that is the SMALLEST of the steps t_d in which its non-zero coordinates o_d are reached, and it
+// gets the block along that dimension.  In the Reduce-Scatter it sends its partial on in that same step.
+static bool build_general(Plan& p) {
+    const int D = p.ndims, n = p.n;
+    std::vector<std::vector<int8_t>> kstep(D), ksgn(D);
+    std::vector<std::vector<int>> dist(D);
+    p.S = 0;
+    for (int d = 0; d < D; ++d) {
+        dist[d] = ring_tree(p.dims[d], kstep[d], ksgn[d]);
+        p.sdim[d] = (int)dist[d].size();
+        p.S += p.sdim[d];
+    }
+    if (p.S > 120) return false;
+    p.general = true;
+    p.nslices = D;
+    p.steps.assign(D, {});
+    p.gstep.assign(D, std::vector<int8_t>(n, -1));
+    p.gsgn.assign(D, std::vector<int8_t>(n, 0));
+    for (int c = 0; c < D; ++c) {
+        std::vector<std::vector<int>> where(D);         // where[d][k] = position of the k-th visit of dimension d
+        int visits[TRV_MAX_DIMS] = {0};
+        int cur = c;
+        for (int t = 0; t < p.S; ++t) {
+            int d = cur;
+            while (visits[d] >= p.sdim[d]) d = (d + 1) % D;
+            p.steps[c].push_back(Step{d, dist[d][visits[d]]});
+            where[d].push_back(t);
+            visits[d]++;
+            cur = (d + 1) % D;
+        }
+        for (int o = 1; o < n; ++o) {
+            int best = -1, best_d = -1;
+            for (int d = 0; d < D; ++d) {
+                const int od = p.coord(o, d);
+                if (od == 0) continue;
+                const int t = where[d][kstep[d][od]];
+                if (best < 0 || t < best) { best = t; best_d = d; }
+            }
+            p.gstep[c][o] = (int8_t)best;
+            p.gsgn[c][o] = ksgn[best_d][p.coord(o, best_d)];
+        }
+    }
+    return true;
 }
 
 static int swing_rho(int k) {      // sum_{i<=k} (-2)^i = 1, -1, 3, -5, 11, ...  (Sec. 2.4)
@@ -107,11 +157,21 @@ trv_status_t build_plan(const int32_t* dims, int32_t ndims, int variant, int alg
         *out = holder;
         return TRV_OK;
     }
-    if (algo == TRV_ALGO_TRIVANCE && ndims == 1 && exact_log(dims[0], 3) < 0) {
-        // a ring of any other size: only the bandwidth-optimal form is defined (Sec. 4.4)
-        if (variant != TRV_BANDWIDTH_OPTIMAL || dims[0] > TRV_MAX_RANKS) { delete holder; return TRV_ERR_UNSUPPORTED; }
-        p.dims[0] = dims[0]; p.stride[0] = 1; p.n = dims[0];
-        build_general_ring(p, dims[0]);
+    bool other_side = false;
+    for (int d = 0; d < ndims; ++d)
+        if (exact_log(dims[d], 3) < 1) other_side = true;
+    if (algo == TRV_ALGO_TRIVANCE && other_side) {
+        // a side that is no power of three: only the bandwidth-optimal form is defined (Sec. 4.4)
+        long long nn = 1;
+        for (int d = 0; d < ndims; ++d) nn *= dims[d];
+        if (variant != TRV_BANDWIDTH_OPTIMAL || nn > TRV_MAX_RANKS || ndims > 4) { delete holder; return TRV_ERR_UNSUPPORTED; }
+        nn = 1;
+        for (int d = 0; d < ndims; ++d) {
+            p.dims[d] = dims[d]; p.stride[d] = (int)nn; nn *= dims[d];
+            if (dims[d] != dims[0]) p.equal_dims = false;
+        }
+        p.n = (int)nn;
+        if (!build_general(p)) { delete holder; return TRV_ERR_UNSUPPORTED; }
         *out = holder;
         return TRV_OK;
     }
@@ -203,13 +263,13 @@ int send_peers(const Plan& p, int r, int dim, int dist, int peer[2], int dir[2],
     }
 }
 
-int general_recv_mask(const Plan& p, int t, int dst, int j) {
-    const int n = p.n, dist = p.steps[0][t].dist;
-    const int o = ((dst - j) % n + n) % n;
-    const int ol = ((o - dist) % n + n) % n, orr = (o + dist) % n;
+int general_recv_mask(const Plan& p, int c, int t, int dst, int j) {
+    const int d = p.steps[c][t].dim, dist = p.steps[c][t].dist;
+    const int o = p.sub(dst, j);
+    const int ol = p.shift(o, d, -dist), orr = p.shift(o, d, dist);
     int mask = 0;
-    if (p.gstep[ol] == t && p.gsgn[ol] > 0) mask |= 1;
-    if (orr != ol && p.gstep[orr] == t && p.gsgn[orr] < 0) mask |= 2;
+    if (p.gstep[c][ol] == t && p.gsgn[c][ol] > 0) mask |= 1;
+    if (orr != ol && p.gstep[c][orr] == t && p.gsgn[c][orr] < 0) mask |= 2;
     return mask;
 }
 
@@ -217,18 +277,19 @@ void message_bytes_side(const Plan& p, int64_t E, int64_t elem_size, int c, int 
     const int n = p.n;
     if (p.general) {
         // Reduce-Scatter row: the node at offset o sends block (node - o); AllGather row: the parent
-        // of the node at offset o, which sits at offset o + sgn * dist, sends it to that node.
-        const int t = p.step_of_row(row), dist = p.steps[0][t].dist;
+        // of the node at offset o, which sits at offset o + sgn * dist along the step's dimension, sends it to that node.
+        const int t = p.step_of_row(row), d = p.steps[c][t].dim, dist = p.steps[c][t].dist;
         const bool rs = row < p.S;
+        const int64_t lo = slice_lo(E, p.nslices, c), hi = slice_lo(E, p.nslices, c + 1);
         for (int r = 0; r < n; ++r) out[r] = 0;
         for (int o = 1; o < n; ++o) {
-            if (p.gstep[o] != t) continue;
-            const int sends_right = rs ? (p.gsgn[o] > 0) : (p.gsgn[o] < 0);
+            if (p.gstep[c][o] != t) continue;
+            const int sends_right = rs ? (p.gsgn[c][o] > 0) : (p.gsgn[c][o] < 0);
             if (sends_right != side) continue;
-            const int src_off = rs ? o : ((o + p.gsgn[o] * dist) % n + n) % n;
+            const int src_off = rs ? o : p.shift(o, d, p.gsgn[c][o] * dist);
             for (int r = 0; r < n; ++r) {
-                const int j = ((r - src_off) % n + n) % n;
-                out[r] += (block_lo(0, E, n, j + 1) - block_lo(0, E, n, j)) * elem_size;
+                const int j = p.sub(r, src_off);
+                out[r] += (block_lo(lo, hi, n, j + 1) - block_lo(lo, hi, n, j)) * elem_size;
             }
         }
         return;

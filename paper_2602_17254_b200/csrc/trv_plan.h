@@ -35,13 +35,14 @@ struct Plan {
     std::vector<std::vector<std::vector<uint64_t>>> reach;
     int words = 0;      // 64-bit words per bitset
 
-    // Rings whose size is no power of three (Sec. 4.4), bandwidth-optimal form only.  The tree a
-    // block follows is the same for every block up to rotation, so it is stored once, by the
-    // OFFSET o = (node - block) mod n:  gstep[o] = Reduce-Scatter step in which the node at
-    // offset o sends its partial on (-1 for the owner, o = 0); gsgn[o] = +1 if it sends it to
-    // node + dist, -1 if to node - dist.
+    // Rings and tori with a side that is no power of three (Sec. 4.4, per dimension as in Sec. 5), bandwidth-optimal
+    // form only.  The tree a block follows is the same for every block up to translation, so it is stored once per
+    // collective, by the OFFSET o = node - block (coordinate by coordinate, modulo the sides; o is the linear index
+    // of that offset vector):  gstep[c][o] = Reduce-Scatter step in which the node at offset o sends its partial on
+    // (-1 for the owner, o = 0), along the dimension of that step; gsgn[c][o] = +1 if it sends it to the node `dist`
+    // after it, -1 if to the node `dist` before it.
     bool general = false;
-    std::vector<int8_t> gstep, gsgn;
+    std::vector<std::vector<int8_t>> gstep, gsgn;
 
     // plan-owned scratch for trv_allreduce (STEP family of the latency form), grown on demand under
     // trv_plan_s::scratch_mu; scratch_device = ordinal of the GPU it was allocated on (-1: none yet)
@@ -57,6 +58,17 @@ struct Plan {
         int a = dims[d], x = coord(r, d);
         int y = ((x + delta) % a + a) % a;
         return r + (y - x) * stride[d];
+    }
+    // coordinate-wise r - j modulo the sides: the offset of node r from block j (and back: j + o)
+    int sub(int r, int j) const {
+        int o = 0;
+        for (int d = 0; d < ndims; ++d) o += ((coord(r, d) - coord(j, d) + dims[d]) % dims[d]) * stride[d];
+        return o;
+    }
+    int add(int j, int o) const {
+        int r = 0;
+        for (int d = 0; d < ndims; ++d) r += ((coord(j, d) + coord(o, d)) % dims[d]) * stride[d];
+        return r;
     }
 };
 
@@ -77,9 +89,9 @@ void message_bytes(const Plan& p, int64_t E, int64_t elem_size, int c, int row, 
 // bytes of the message every rank SENDS to its peer number `side` (0: first peer -- Trivance: the
 // left one; 1: second peer) in one row; 0 where it sends none.  Every kind of plan.
 void message_bytes_side(const Plan& p, int64_t E, int64_t elem_size, int c, int row, int side, int64_t* out);
-// general rings: what `dst` receives for block j in Reduce-Scatter step t: bit 0 = a partial from
-// its left peer, bit 1 = one from its right peer
-int general_recv_mask(const Plan& p, int t, int dst, int j);
+// sides of any size: what `dst` receives for block j in Reduce-Scatter step t of collective c: bit 0 = a partial
+// from the node before it along the step's dimension, bit 1 = one from the node after it
+int general_recv_mask(const Plan& p, int c, int t, int dst, int j);
 
 }  // namespace trv
 

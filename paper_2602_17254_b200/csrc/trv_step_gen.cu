@@ -1,6 +1,6 @@
-// STEP kernels for rings whose size is no power of three (Sec. 4.4), bandwidth-optimal form.
+// STEP kernels for rings and tori with a side that is no power of three (Sec. 4.4, Sec. 5), bandwidth-optimal form.
 //
-// One launch per schedule step, in place in the output buffers.  The tree a block follows is
+// One launch per schedule step and collective, in place in the output buffers.  The tree a block follows is
 // stored by offset from the block's owner (Plan::gstep / gsgn); per step the host lists
 //   Reduce-Scatter: the offsets o at which a node receives, with which sides send to it;
 //                   the node p at offset o from block b = p - o adds (left + own) + right,
@@ -8,6 +8,9 @@
 //   AllGather:      the offsets o at which a node receives the finished block, and from which side.
 // A node writes its partial of a block only in steps before the one in which it sends it on, and
 // the node it sends to reads it in exactly that step, so no step reads what the same step writes.
+#include <algorithm>
+#include <vector>
+
 #include "trv_dev.cuh"
 
 namespace trv {
@@ -21,13 +24,15 @@ struct GenTab {
     unsigned short e[CAP];
 };
 struct GenArgs {
-    long long gcount, w0, w1;   // global vector length; the buffers hold elements [w0, w1)
-    int n, dist;
+    long long slo, shi, w0, w1;     // the collective's slice of the global vector; the buffers hold elements [w0, w1)
+    int n, dim, dist;               // the step's dimension and distance
+    TorusGeo geo;
 };
 
 __device__ __forceinline__ void gen_block_range(const GenArgs& a, int j, long long* lo, long long* hi) {
-    long long b0 = (long long)(((unsigned long long)j * (unsigned long long)a.gcount) / (unsigned)a.n);
-    long long b1 = (long long)(((unsigned long long)(j + 1) * (unsigned long long)a.gcount) / (unsigned)a.n);
+    const unsigned long long len = (unsigned long long)(a.shi - a.slo);
+    long long b0 = a.slo + (long long)(((unsigned long long)j * len) / (unsigned)a.n);
+    long long b1 = a.slo + (long long)(((unsigned long long)(j + 1) * len) / (unsigned)a.n);
     b0 = b0 < a.w0 ? a.w0 : (b0 > a.w1 ? a.w1 : b0);
     b1 = b1 < a.w0 ? a.w0 : (b1 > a.w1 ? a.w1 : b1);
     *lo = b0 - a.w0;
@@ -68,9 +73,8 @@ __global__ void __launch_bounds__(kGenThreads) k_rs_gen(PtrTab<CAP> buf, GenTab<
     const unsigned ent = tab.e[blockIdx.y];
     const int o = ent & 1023;
     const bool from_left = ent & 1024, from_right = ent & 2048;
-    int b = p - o; if (b < 0) b += a.n;
-    int ql = p - a.dist; if (ql < 0) ql += a.n;
-    int qr = p + a.dist; if (qr >= a.n) qr -= a.n;
+    const int b = geo_sub(a.geo, p, o);
+    const int ql = geo_shift(a.geo, p, a.dim, -a.dist), qr = geo_shift(a.geo, p, a.dim, a.dist);
     const T* __restrict__ L = (const T*)buf.p[ql];
     const T* __restrict__ R = (const T*)buf.p[qr];
     T* __restrict__ O = (T*)buf.p[p];
@@ -99,10 +103,8 @@ __global__ void __launch_bounds__(kGenThreads) k_ag_gen(PtrTab<CAP> buf, GenTab<
     const int p = blockIdx.z;
     const unsigned ent = tab.e[blockIdx.y];
     const int o = ent & 1023;
-    int b = p - o; if (b < 0) b += a.n;
-    int q = (ent & 1024) ? p + a.dist : p - a.dist;
-    if (q < 0) q += a.n;
-    if (q >= a.n) q -= a.n;
+    const int b = geo_sub(a.geo, p, o);
+    const int q = geo_shift(a.geo, p, a.dim, (ent & 1024) ? a.dist : -a.dist);
     const uint32_t* __restrict__ S = (const uint32_t*)buf.p[q];
     uint32_t* __restrict__ O = (uint32_t*)buf.p[p];
     long long lo, hi;
@@ -139,29 +141,35 @@ static trv_status_t gen_impl(const Call& c) {
         launch_pdl(k_copy_gen<CAP>, grid, dim3(kGenThreads), 0, c.st, IN, OUT, (long long)c.count);
     }
     GenArgs a;
-    a.gcount = (long long)c.gcount; a.w0 = (long long)c.goff; a.w1 = (long long)(c.goff + c.count); a.n = n;
-    const long long max_len = (long long)(c.gcount / n) + 1;
+    a.w0 = (long long)c.goff; a.w1 = (long long)(c.goff + c.count); a.n = n;
+    a.geo = make_geo(p);
     for (int row = 0; row < 2 * S; ++row) {
         const int t = p.step_of_row(row);
-        a.dist = p.steps[0][t].dist;
-        GenTab<CAP> tab;
-        tab.cnt = 0;
-        if (row < S) {
-            for (int o = 0; o < n; ++o) {
-                const int ol = ((o - a.dist) % n + n) % n, orr = (o + a.dist) % n;
-                const bool fl = p.gstep[ol] == t && p.gsgn[ol] > 0;
-                const bool fr = orr != ol && p.gstep[orr] == t && p.gsgn[orr] < 0;
-                if (fl || fr) tab.e[tab.cnt++] = (unsigned short)(o | (fl ? 1024 : 0) | (fr ? 2048 : 0));
+        for (int sl = 0; sl < p.nslices; ++sl) {
+            a.slo = slice_lo((int64_t)c.gcount, p.nslices, sl); a.shi = slice_lo((int64_t)c.gcount, p.nslices, sl + 1);
+            if (std::min(a.shi, a.w1) <= std::max(a.slo, a.w0)) continue;      // nothing of this collective in the window
+            const long long max_len = (a.shi - a.slo) / n + 1;
+            const std::vector<int8_t>&gs = p.gstep[sl], &gg = p.gsgn[sl];
+            a.dim = p.steps[sl][t].dim; a.dist = p.steps[sl][t].dist;
+            GenTab<CAP> tab;
+            tab.cnt = 0;
+            if (row < S) {
+                for (int o = 0; o < n; ++o) {
+                    const int ol = p.shift(o, a.dim, -a.dist), orr = p.shift(o, a.dim, a.dist);
+                    const bool fl = gs[ol] == t && gg[ol] > 0;
+                    const bool fr = orr != ol && gs[orr] == t && gg[orr] < 0;
+                    if (fl || fr) tab.e[tab.cnt++] = (unsigned short)(o | (fl ? 1024 : 0) | (fr ? 2048 : 0));
+                }
+            } else {
+                for (int o = 1; o < n; ++o)
+                    if (gs[o] == t) tab.e[tab.cnt++] = (unsigned short)(o | (gg[o] > 0 ? 1024 : 0));
             }
-        } else {
-            for (int o = 1; o < n; ++o)
-                if (p.gstep[o] == t) tab.e[tab.cnt++] = (unsigned short)(o | (p.gsgn[o] > 0 ? 1024 : 0));
+            if (tab.cnt == 0) continue;
+            dim3 grid(gen_grid_x(max_len), tab.cnt, n);
+            if (row >= S) launch_pdl(k_ag_gen<CAP>, grid, dim3(kGenThreads), 0, c.st, OUT, tab, a);
+            else if (c.dtype == TRV_FLOAT32) launch_pdl(k_rs_gen<float, CAP>, grid, dim3(kGenThreads), 0, c.st, OUT, tab, a);
+            else launch_pdl(k_rs_gen<uint32_t, CAP>, grid, dim3(kGenThreads), 0, c.st, OUT, tab, a);
         }
-        if (tab.cnt == 0) continue;
-        dim3 grid(gen_grid_x(max_len), tab.cnt, n);
-        if (row >= S) launch_pdl(k_ag_gen<CAP>, grid, dim3(kGenThreads), 0, c.st, OUT, tab, a);
-        else if (c.dtype == TRV_FLOAT32) launch_pdl(k_rs_gen<float, CAP>, grid, dim3(kGenThreads), 0, c.st, OUT, tab, a);
-        else launch_pdl(k_rs_gen<uint32_t, CAP>, grid, dim3(kGenThreads), 0, c.st, OUT, tab, a);
     }
     return cudaGetLastError() == cudaSuccess ? TRV_OK : TRV_ERR_CUDA;
 }

@@ -94,3 +94,8 @@ def workload_inputs(w: Workload, count=None):
 for _n in (32, 100):
     _name = "ring%d_bw_8MiB" % _n
     CONFIGS[_name] = Workload(_name, (_n,), BANDWIDTH, 8 * MiB // 4, "normal", 5)
+# Tori with sides that are no powers of three (Sec. 4.4 per dimension; 32 x 32, 8 x 64 and 16 x 16 x 16 are tori the
+# paper evaluates -- 16 x 16 x 4 stands in for the last, which has more ranks than the engine takes), bandwidth form.
+for _dims in ((32, 32), (8, 64), (16, 16, 4)):
+    _name = "torus%s_bw_8MiB" % "x".join(map(str, _dims))
+    CONFIGS[_name] = Workload(_name, _dims, BANDWIDTH, 8 * MiB // 4, "normal", 6)

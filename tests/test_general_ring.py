@@ -234,7 +234,8 @@ def test_message_bytes_side_regular_plans():
 
 
 def test_unsupported_forms():
-    for dims, variant in (([7], binding.LATENCY_OPTIMAL), ([7, 3], binding.BANDWIDTH_OPTIMAL), ([3, 10], binding.BANDWIDTH_OPTIMAL), ([1025], binding.BANDWIDTH_OPTIMAL)):
+    for dims, variant in (([7], binding.LATENCY_OPTIMAL), ([7, 3], binding.LATENCY_OPTIMAL), ([33, 32], binding.BANDWIDTH_OPTIMAL),
+                          ([2, 2, 2, 2, 2], binding.BANDWIDTH_OPTIMAL), ([1025], binding.BANDWIDTH_OPTIMAL)):
         with pytest.raises(binding.TrivanceError) as e:
             binding.Plan(dims, variant)
         assert e.value.status == binding.ERR_UNSUPPORTED

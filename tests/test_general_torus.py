@@ -5,6 +5,7 @@ import numpy as np
 import pytest
 
 import oracle
+from paper_2602_17254_b200 import binding
 
 TORI = [(4, 4), (8, 8), (7, 3), (3, 10), (2, 5), (5, 5), (2, 2), (4, 4, 4), (2, 3, 4), (6, 9), (16, 8)]
 BW = oracle.VARIANT_BANDWIDTH
@@ -229,3 +230,45 @@ def test_float32_order_against_tree_evaluator(dims):
     exact = x.astype(np.float64).sum(0)
     bound = 2e-6 * np.abs(x.astype(np.float64)).sum(0)
     assert (np.abs(y.astype(np.float64) - exact[None]) <= bound[None]).all()
+
+
+# ------------------------------------------------------------------ the library's host side
+
+@pytest.mark.parametrize("dims", TORI + [(32, 32), (8, 64), (16, 16, 4)])
+def test_plan_matches_oracle(dims):
+    """The library derives the tree as the product of per-dimension ring trees (no holder list); the oracle grows it
+    with the holder list.  Step lists, receive masks and bytes sent must agree."""
+    n, S = oracle.gent_num_steps(dims)
+    D = len(dims)
+    plan = binding.Plan(dims, binding.BANDWIDTH_OPTIMAL)
+    assert plan.n == n and plan.rows == 2 * S and plan.nslices == D
+    assert plan.kernel_supported(binding.KERNEL_FUSED) and plan.kernel_supported(binding.KERNEL_STEP)
+    E = 3 * n * D + 5
+    sent = np.zeros(n, np.int64)
+    for c in range(D):
+        steps = oracle.gent_step_list(dims, c)
+        for row in range(2 * S):
+            t = row if row < S else 2 * S - 1 - row
+            assert plan.step(c, row) == steps[t]
+            for side in (0, 1):
+                sent += plan.message_bytes_side(E, 4, c, row, side)
+        par, stp = oracle.gent_tree(dims, c)
+        for t, (d, dist) in enumerate(steps):
+            for dst in sorted({0, 1, n // 2, n - 1}):
+                cd = _coords(dst, dims)
+                ql = _rank([cd[k] - (dist if k == d else 0) for k in range(D)], dims)
+                qr = _rank([cd[k] + (dist if k == d else 0) for k in range(D)], dims)
+                want = np.zeros(n, np.uint8)
+                want[(par[:, ql] == dst) & (stp[:, ql] == t)] |= 1
+                if qr != ql:
+                    want[(par[:, qr] == dst) & (stp[:, qr] == t)] |= 2
+                assert np.array_equal(plan.send_mask(c, t, dst), want), (c, t, dst)
+    assert np.array_equal(sent, oracle.gent_link_loads(dims, E, 4)["sent"])
+    plan.destroy()
+
+
+def test_latency_form_is_refused_for_such_sides():
+    for dims in ((4, 4), (7, 3), (3, 10)):
+        with pytest.raises(binding.TrivanceError) as e:
+            binding.Plan(dims, binding.LATENCY_OPTIMAL)
+        assert e.value.status == binding.ERR_UNSUPPORTED
