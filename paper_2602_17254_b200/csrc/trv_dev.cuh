@@ -149,12 +149,42 @@ __device__ __forceinline__ V add3v(const V& a, const V& b, const V& c) {
 struct TorusGeo {
     int nd;
     int dims[4], stride[4];
+    int shift[4];       // bit position of coordinate d in a packed coordinate vector (fields of ceil(log2 side) bits)
 };
 inline TorusGeo make_geo(const Plan& p) {
     TorusGeo g;
     g.nd = p.ndims;
-    for (int d = 0; d < 4; ++d) { g.dims[d] = d < p.ndims ? p.dims[d] : 1; g.stride[d] = d < p.ndims ? p.stride[d] : p.n; }
+    int pos = 0;
+    for (int d = 0; d < 4; ++d) {
+        g.dims[d] = d < p.ndims ? p.dims[d] : 1;
+        g.stride[d] = d < p.ndims ? p.stride[d] : p.n;
+        g.shift[d] = pos;
+        int w = 0;
+        while ((1 << w) < g.dims[d]) ++w;
+        pos += w;
+    }
     return g;
+}
+// coordinates of a rank (or of an offset), packed; and base + offset from two packed vectors
+__device__ __forceinline__ unsigned geo_pack(const TorusGeo& g, int r) {
+    unsigned v = 0;
+#pragma unroll
+    for (int d = 0; d < 4; ++d)
+        if (d < g.nd) v |= (unsigned)((r / g.stride[d]) % g.dims[d]) << g.shift[d];
+    return v;
+}
+__device__ __forceinline__ int geo_add_packed(const TorusGeo& g, unsigned base, unsigned off) {
+    int out = 0;
+#pragma unroll
+    for (int d = 0; d < 4; ++d)
+        if (d < g.nd) {
+            const unsigned hi = d + 1 < g.nd ? (unsigned)g.shift[d + 1] : 32u;
+            const unsigned m = hi - g.shift[d] >= 32u ? ~0u : ((1u << (hi - g.shift[d])) - 1u);
+            int x = (int)((base >> g.shift[d]) & m) + (int)((off >> g.shift[d]) & m);
+            if (x >= g.dims[d]) x -= g.dims[d];
+            out += x * g.stride[d];
+        }
+    return out;
 }
 // node + offset and node - offset, coordinate by coordinate modulo the sides
 __device__ __forceinline__ int geo_add(const TorusGeo& g, int r, int o) {

@@ -26,7 +26,8 @@ namespace trv {
 
 constexpr int kTreeThreads = 128;
 constexpr int kTreeChunk = 8;       // program entries whose loads are in flight together
-constexpr int kTreeDepth = 10;      // stack slots: tree height <= steps + 1 <= 8 for n <= 1024
+constexpr int kTreeDepth = 12;      // stack slots: tree height <= steps + 1 <= 11 for n <= 1024 in up to four dimensions
+constexpr int kTreeAlign = 64;      // tiles start on multiples of 64 elements of the buffers: a warp's access is whole 128-byte lines
 
 // entry: offset from the block's owner (bits 0..9) | additions after this node (bits 10..13); one program per collective
 constexpr int kTreeMaxSlices = 4;
@@ -38,6 +39,7 @@ struct TreeArgs {
     int n;
     long long w0, count;                                // global index of local element 0; local elements
     long long slo[kTreeMaxSlices], shi[kTreeMaxSlices]; // the collectives' slices of the global vector
+    int two_blocks;                                     // every block is at least a CTA's span long
     TorusGeo geo;
 };
 
@@ -55,21 +57,31 @@ struct TreeStrideTabs {
     __device__ __forceinline__ T* out(int r) const { return reinterpret_cast<T*>(o.ptr(r)); }
 };
 
-// V columns starting at local element e, all inside block b: evaluate the tree, store to all ranks.
-// `stack` is this thread's slot of level 0; levels are kTreeThreads * SLOT elements apart, SLOT being
-// the slot width of the kernel (its own V) also when a thread walks single columns, so that the
-// slots of different threads never overlap.
-template <typename T, int V, int SLOT, typename Tabs, typename RankOf>
+// V columns starting at local element e: evaluate the tree, store to all ranks.  rank_of(o, k) = the rank at offset o
+// from the block that column k lies in.  SPLIT = false: both columns lie in one block and are loaded and stored as one
+// vector.  SPLIT = true (V = 2): the columns may lie in different blocks, or one of them outside the collective
+// (live[k] = false): one scalar access per column, same walk.  A warp takes ONE of the two forms as a whole, so a
+// block boundary inside a warp costs no second pass.
+// `stack` is this thread's slot of level 0; levels are kTreeThreads * V elements apart.
+template <typename T, int V, bool SPLIT, typename Tabs, typename RankOf>
 __device__ __forceinline__ void tree_column(const TreeArgs& a, const unsigned short* prog, const Tabs& tabs, long long e,
-                                            RankOf rank_of, T* stack) {
-    static_assert(V <= SLOT, "slot too narrow");
+                                            RankOf rank_of, T* stack, bool live0, bool live1) {
     using P = Elem<T, V>;
     const int n = a.n;
+    const long long e0 = live0 ? e : e + 1, e1 = live1 ? e + 1 : e;     // a column that is not live re-reads the live one
     auto load_chunk = [&](int i0, P (&v)[kTreeChunk]) {
 #pragma unroll
         for (int m = 0; m < kTreeChunk; ++m) {
             const int idx = i0 + m;
-            if (idx < n) v[m] = *reinterpret_cast<const P*>(tabs.in(rank_of(prog[idx] & 1023)) + e);
+            if (idx < n) {
+                const int o = prog[idx] & 1023;
+                if constexpr (!SPLIT) {
+                    v[m] = *reinterpret_cast<const P*>(tabs.in(rank_of(o, 0)) + e);
+                } else {
+                    v[m].x[0] = tabs.in(rank_of(o, 0))[e0];
+                    v[m].x[1] = tabs.in(rank_of(o, 1))[e1];
+                }
+            }
         }
     };
     P nxt[kTreeChunk];
@@ -87,66 +99,93 @@ __device__ __forceinline__ void tree_column(const TreeArgs& a, const unsigned sh
             if (idx < n) {
                 int k = prog[idx] >> 10;
                 if (k == 0) {           // an inner node: its subtrees follow
-                    if (idx > 0) *reinterpret_cast<P*>(stack + (sp++) * (kTreeThreads * SLOT)) = tos;
+                    if (idx > 0) *reinterpret_cast<P*>(stack + (sp++) * (kTreeThreads * V)) = tos;
                     tos = cur[m];
                 } else {                // a leaf closes at once: add it to the value on top, no stack traffic
                     tos = add2(tos, cur[m]);
-                    for (--k; k > 0; --k) tos = add2(*reinterpret_cast<const P*>(stack + (--sp) * (kTreeThreads * SLOT)), tos);
+                    for (--k; k > 0; --k) tos = add2(*reinterpret_cast<const P*>(stack + (--sp) * (kTreeThreads * V)), tos);
                 }
             }
         }
     }
+    if constexpr (!SPLIT) {
 #pragma unroll 8
-    for (int r = 0; r < n; ++r) *reinterpret_cast<P*>(tabs.out(r) + e) = tos;
+        for (int r = 0; r < n; ++r) *reinterpret_cast<P*>(tabs.out(r) + e) = tos;
+    } else {
+#pragma unroll 4
+        for (int r = 0; r < n; ++r) {
+            if (live0) tabs.out(r)[e] = tos.x[0];
+            if (live1) tabs.out(r)[e + 1] = tos.x[1];
+        }
+    }
 }
 
 template <typename T, int V, int CAP, typename Tabs>
 __device__ __forceinline__ void tree_tile(const TreeArgs& a, const TreeProg<CAP>& progs, const Tabs& tabs, void* stack_raw,
-                                          unsigned short* rk) {
+                                          unsigned short* rk, unsigned* oc) {
     const int c = blockIdx.y, n = a.n;                  // CTA-uniform: the collective
     const unsigned short* prog = progs.e[c];
     const long long slo = a.slo[c], shi = a.shi[c];
-    // local range of the collective inside the window, tiles aligned to V elements of the buffers
+    // local range of the collective inside the window; tiles aligned to whole lines of the buffers (a collective
+    // that starts inside a line leaves the columns before its start to the previous collective's last tile)
     long long llo = slo - a.w0, lhi = shi - a.w0;
     if (llo < 0) llo = 0;
     if (lhi > a.count) lhi = a.count;
-    const long long t0 = (llo / V) * V + (long long)blockIdx.x * kTreeThreads * V;
+    const long long t0 = (llo / kTreeAlign) * kTreeAlign + (long long)blockIdx.x * kTreeThreads * V;
     if (t0 >= lhi) return;
     auto owner = [&](long long el) -> int {
         const unsigned long long x = (unsigned long long)(a.w0 + el - slo);
         return (int)(((x + 1) * (unsigned)n - 1) / (unsigned long long)(shi - slo));
     };
-    // block + offset for the block the CTA's first column lies in
-    const int b0 = owner(t0 < llo ? llo : t0);
-    if (a.geo.nd > 1) {
-        for (int o = threadIdx.x; o < n; o += kTreeThreads) rk[o] = (unsigned short)geo_add(a.geo, b0, o);
+    // Torus: block + offset is tabulated for the block the CTA's first column lies in and for the next one; where
+    // blocks are at least a CTA's span long (a.two_blocks) no CTA reaches a third.  Otherwise (short vectors) it is
+    // computed from the packed coordinates oc of the offsets.
+    const bool torus = a.geo.nd > 1;
+    const int b0 = owner(t0 < llo ? llo : t0), b1 = b0 + 1 < n ? b0 + 1 : b0;
+    if (torus) {
+        for (int o = threadIdx.x; o < n; o += kTreeThreads) oc[o] = geo_pack(a.geo, o);
         __syncthreads();
+        if (a.two_blocks) {
+            const unsigned c0 = geo_pack(a.geo, b0), c1 = geo_pack(a.geo, b1);
+            for (int o = threadIdx.x; o < n; o += kTreeThreads) {
+                rk[o] = (unsigned short)geo_add_packed(a.geo, c0, oc[o]);
+                rk[CAP + o] = (unsigned short)geo_add_packed(a.geo, c1, oc[o]);
+            }
+            __syncthreads();
+        }
     }
     const long long e = t0 + (long long)threadIdx.x * V;
-    if (e >= lhi) return;
     T* const stack = reinterpret_cast<T*>(stack_raw) + threadIdx.x * V;
-    auto run = [&](auto width, long long el, int b) {
-        constexpr int W = decltype(width)::value;
-        if (a.geo.nd == 1) {
-            tree_column<T, W, V>(a, prog, tabs, el, [&](int o) { int r = b + o; return r >= n ? r - n : r; }, stack);
-        } else if (b == b0) {
-            tree_column<T, W, V>(a, prog, tabs, el, [&](int o) { return (int)rk[o]; }, stack);
-        } else {
-            tree_column<T, W, V>(a, prog, tabs, el, [&](int o) { return geo_add(a.geo, b, o); }, stack);
-        }
-    };
     if constexpr (V == 1) {
-        run(std::integral_constant<int, 1>{}, e, owner(e));
-    } else {
-        const bool inside = e >= llo && e + V <= lhi;
-        int bf = 0;
-        bool same = false;
-        if (inside) { bf = owner(e); same = owner(e + V - 1) == bf; }
-        if (same) {
-            run(std::integral_constant<int, V>{}, e, bf);
+        if (e >= lhi || e < llo) return;
+        const int b = owner(e);
+        if (!torus) {
+            tree_column<T, 1, false>(a, prog, tabs, e, [&](int o, int) { int r = b + o; return r >= n ? r - n : r; }, stack, true, true);
+        } else if (a.two_blocks) {
+            const unsigned short* tab = b == b0 ? rk : rk + CAP;
+            tree_column<T, 1, false>(a, prog, tabs, e, [&](int o, int) { return (int)tab[o]; }, stack, true, true);
         } else {
-            for (int k = 0; k < V; ++k)
-                if (e + k >= llo && e + k < lhi) run(std::integral_constant<int, 1>{}, e + k, owner(e + k));
+            const unsigned cb = geo_pack(a.geo, b);
+            tree_column<T, 1, false>(a, prog, tabs, e, [&](int o, int) { return geo_add_packed(a.geo, cb, oc[o]); }, stack, true, true);
+        }
+    } else {
+        static_assert(V == 2, "one or two columns per thread");
+        const bool live0 = e >= llo && e < lhi, live1 = e + 1 >= llo && e + 1 < lhi;
+        const bool dead = !(live0 || live1);
+        const int bA = dead ? 0 : owner(live0 ? e : e + 1), bB = dead ? 0 : owner(live1 ? e + 1 : e);
+        // all 32 lanes are here (every return above is CTA-uniform): the warp picks one form
+        const bool vec = __all_sync(0xffffffffu, dead || (live0 && live1 && bA == bB));
+        if (dead) return;
+        if (!torus) {
+            auto rank_of = [&](int o, int k) { int r = (k ? bB : bA) + o; return r >= n ? r - n : r; };
+            if (vec) tree_column<T, 2, false>(a, prog, tabs, e, rank_of, stack, true, true);
+            else tree_column<T, 2, true>(a, prog, tabs, e, rank_of, stack, live0, live1);
+        } else {        // the host takes this kernel only where a.two_blocks holds
+            const unsigned short* tA = bA == b0 ? rk : rk + CAP;
+            const unsigned short* tB = bB == b0 ? rk : rk + CAP;
+            auto rank_of = [&](int o, int k) { return (int)(k ? tB : tA)[o]; };
+            if (vec) tree_column<T, 2, false>(a, prog, tabs, e, rank_of, stack, true, true);
+            else tree_column<T, 2, true>(a, prog, tabs, e, rank_of, stack, live0, live1);
         }
     }
 }
@@ -157,20 +196,22 @@ __global__ void __launch_bounds__(kTreeThreads) k_bw_tree(PtrTab<CAP> in, PtrTab
     __shared__ const T* sin[CAP];
     __shared__ T* sout[CAP];
     __shared__ __align__(16) unsigned char stack[kTreeDepth * kTreeThreads * V * sizeof(T)];
-    __shared__ unsigned short rk[CAP];
+    __shared__ unsigned short rk[2 * CAP];
+    __shared__ unsigned oc[CAP];
     for (int r = threadIdx.x; r < a.n; r += kTreeThreads) { sin[r] = (const T*)in.p[r]; sout[r] = (T*)out.p[r]; }
     __syncthreads();
     pdl_wait();
-    tree_tile<T, V, CAP>(a, prog, TreeSmemTabs<T, CAP>{sin, sout}, stack, rk);
+    tree_tile<T, V, CAP>(a, prog, TreeSmemTabs<T, CAP>{sin, sout}, stack, rk, oc);
 }
 
 template <typename T, int V, int CAP>
 __global__ void __launch_bounds__(kTreeThreads) k_bw_tree_strided(StrideAddr in, StrideAddr out, TreeProg<CAP> prog, TreeArgs a) {
     pdl_trigger();
     __shared__ __align__(16) unsigned char stack[kTreeDepth * kTreeThreads * V * sizeof(T)];
-    __shared__ unsigned short rk[CAP];
+    __shared__ unsigned short rk[2 * CAP];
+    __shared__ unsigned oc[CAP];
     pdl_wait();
-    tree_tile<T, V, CAP>(a, prog, TreeStrideTabs<T>{in, out}, stack, rk);
+    tree_tile<T, V, CAP>(a, prog, TreeStrideTabs<T>{in, out}, stack, rk, oc);
 }
 
 // ------------------------------------------------------------------ host side
@@ -203,6 +244,7 @@ static trv_status_t launch_tree(const Call& c, const std::vector<std::vector<uns
     TreeArgs a;
     a.n = p.n; a.w0 = (long long)c.goff; a.count = (long long)c.count;
     a.geo = make_geo(p);
+    a.two_blocks = (long long)(c.gcount / p.nslices / p.n) >= (long long)V * kTreeThreads ? 1 : 0;
     long long tiles = 0;
     for (int sl = 0; sl < kTreeMaxSlices; ++sl) {
         a.slo[sl] = a.shi[sl] = 0;
@@ -212,7 +254,8 @@ static trv_status_t launch_tree(const Call& c, const std::vector<std::vector<uns
         a.shi[sl] = slice_lo((int64_t)c.gcount, p.nslices, sl + 1);
         long long lo, hi;
         local_slice(c, sl, &lo, &hi);
-        if (hi > lo) tiles = std::max(tiles, (hi - (lo / V) * V + (long long)V * kTreeThreads - 1) / ((long long)V * kTreeThreads));
+        if (hi > lo)
+            tiles = std::max(tiles, (hi - (lo / kTreeAlign) * kTreeAlign + (long long)V * kTreeThreads - 1) / ((long long)V * kTreeThreads));
     }
     if (tiles == 0) return TRV_OK;
     const dim3 grid((unsigned)tiles, p.nslices, 1);
