@@ -28,7 +28,7 @@ typedef struct trv_plan_s *trv_plan_t;          /* opaque; owned by the library 
 typedef enum {
     TRV_OK = 0,
     TRV_ERR_INVALID_ARG = 1,        /* NULL pointer, bad enum, misaligned or aliasing buffers ... */
-    TRV_ERR_UNSUPPORTED = 2,        /* a side that is no power of three (other than a ring in the bandwidth form), too many ranks, op != sum */
+    TRV_ERR_UNSUPPORTED = 2,        /* a side that is no power of three in the latency form, too many ranks or dimensions, op != sum */
     TRV_ERR_UNDEFINED_SCHEDULE = 3, /* the schedule does not exist for this n (Recursive Doubling, n != 2^q) */
     TRV_ERR_ALLOC = 4,
     TRV_ERR_CUDA = 5,               /* a CUDA runtime call failed; cudaGetLastError has the reason */
@@ -51,11 +51,14 @@ typedef enum { TRV_SUM = 0 } trv_op_t;
  *          Exists for the shapes trv_kernel_supported() reports.
  *   AUTO : FUSED where it exists, else STEP.
  *   PIPELINED: the chunk-level readiness engine the paper sketches for a collective-library
- *          backend (App. D): latency form only; one persistent kernel; a work item per (rank,
- *          step, chunk) runs as soon as the chunks of both peers and the local partial of the
- *          previous step are marked ready, with no barrier between steps.  Never chosen by AUTO.
- *          Needs scratch (trv_scratch_bytes); all its device-side waits are bounded, see
- *          trv_pipeline_status.
+ *          backend (App. D): one persistent kernel; a work item per (rank, step, chunk) runs as soon
+ *          as what it reads is marked ready, with no barrier between steps.  Latency form: the chunks
+ *          of both peers and the local partial of the previous step.  Bandwidth form (power-of-three
+ *          sides): a chunk is a piece of one block; a Reduce-Scatter item binds the two incoming
+ *          chunks to the local partial of the same block range, an AllGather item copies the finished
+ *          chunk from the peer that holds it.  Never chosen by AUTO.  Needs scratch
+ *          (trv_scratch_bytes; for a sharded call of the bandwidth form ask with the GLOBAL count);
+ *          all its device-side waits are bounded, see trv_pipeline_status.
  * All families give bit-identical results. */
 typedef enum { TRV_KERNEL_AUTO = 0, TRV_KERNEL_STEP = 1, TRV_KERNEL_FUSED = 2, TRV_KERNEL_PIPELINED = 3 } trv_kernel_t;
 
@@ -76,19 +79,23 @@ typedef enum { TRV_KERNEL_AUTO = 0, TRV_KERNEL_STEP = 1, TRV_KERNEL_FUSED = 2, T
  * Errors: INVALID_ARG (NULL, ndims out of range, side < 2), UNSUPPORTED (side not a power
  * of three, more than TRV_MAX_RANKS ranks).
  *
- * Rings of any other size (Sec. 4.4): with ndims = 1 and the bandwidth-optimal variant, a side
- * n >= 2 that is no power of three gives the schedule of ceil(log3 n) steps per phase: the
- * regular distances 3^0 .. 3^(s-1), s = floor(log3 n), then one step at distance
- * ceil((n - 3^s) / 2).  The paper fixes the steps, the distances, that no block is sent twice
- * by a node in a phase and that a node sends at most m bytes per phase; which tree a block
- * follows it leaves open.  This library's reading: the AllGather of a block runs the steps in
- * reverse order; the nodes holding the block are kept in the order they got it; in a step
- * every holder, in that order, offers it to its left peer (h - dist), then to its right peer
- * (h + dist); a node that already holds it is skipped.  The Reduce-Scatter runs the same tree
- * backwards, a receiver adding (from_left + own) + from_right and leaving out a side nothing
- * comes from.  Such plans have a STEP family (one launch per step) and, up to TRV_MAX_RANKS ranks, a
- * FUSED kernel that walks the block's tree as a stack machine.  The latency-optimal variant is
- * not defined for these sizes: UNSUPPORTED, as for tori with such a side. */
+ * Sides of any other size (Sec. 4.4), bandwidth-optimal variant only.  A ring of n >= 2 nodes, n no power of
+ * three, gets ceil(log3 n) steps per phase: the regular distances 3^0 .. 3^(s-1), s = floor(log3 n), then one
+ * step at distance ceil((n - 3^s) / 2).  The paper fixes the steps, the distances, that no block is sent twice
+ * by a node in a phase and that a node sends at most m bytes per phase; which tree a block follows it leaves
+ * open.  This library's reading: the AllGather of a block runs the steps in reverse order; the nodes holding
+ * the block are kept in the order they got it; in a step every holder, in that order, offers it to its left
+ * peer (h - dist), then to its right peer (h + dist); a node that already holds it is skipped.  The
+ * Reduce-Scatter runs the same tree backwards, a receiver adding (from_left + own) + from_right and leaving
+ * out a side nothing comes from.
+ * A torus with such sides (up to four dimensions; the paper evaluates 32 x 32, 8 x 64 and 16 x 16 x 16)
+ * composes this with Sec. 5: one collective per dimension on 1/D of the vector; collective c visits the
+ * dimensions in round-robin order from c, a dimension whose ring steps are used up being skipped, the k-th
+ * visit of a dimension using its ring's k-th distance; sum over d of ceil(log3 a_d) steps per phase.  Along
+ * every dimension a block travels by that ring's tree (the same holder rule applied to the torus gives exactly
+ * this product of ring trees).  Block j of every collective is owned by linear rank j.
+ * Such plans have a STEP family (one launch per step and collective) and a FUSED kernel that walks the block's
+ * tree as a stack machine.  The latency-optimal variant is not defined for these sizes: UNSUPPORTED. */
 trv_status_t trv_plan_create(const int32_t *dims, int32_t ndims, trv_variant_t variant, trv_plan_t *out);
 
 /* Same, for a comparator schedule (Sec. 2.4, Fig. 1).  TRV_ALGO_BRUCK: peers r + 3^k and
@@ -128,9 +135,9 @@ trv_status_t trv_plan_peers(trv_plan_t plan, int32_t c, int32_t row, int32_t *pe
 /* set: HOST array of n bytes; set[j] = 1 iff block j is part of the message sent to rank
  * `dst` in Reduce-Scatter step `step` of collective c (closed form Pi of Sec. 4.3: the
  * blocks that agree with dst modulo 3^(visits so far) in every dimension). */
-/* For a ring whose size is no power of three (Sec. 4.4) the two senders' sets differ:
- * set[j] then has bit 0 set if dst receives a partial of block j from its left peer in that
- * step and bit 1 if it receives one from its right peer. */
+/* With a side that is no power of three (Sec. 4.4) the two senders' sets differ:
+ * set[j] then has bit 0 set if dst receives a partial of block j from the node before it along the
+ * step's dimension and bit 1 if it receives one from the node after it. */
 trv_status_t trv_plan_send_set(trv_plan_t plan, int32_t c, int32_t step, int32_t dst, uint8_t *set);
 
 /* bounds: HOST array of n+1 global element indices: block j of collective c covers
@@ -286,7 +293,7 @@ trv_status_t trv_link_loads(trv_plan_t plan, size_t count, size_t elem_size, int
 /* bytes: HOST int64 [n].  Row < S (Reduce-Scatter or latency form): bytes of the message a
  * rank RECEIVES from each sender in that row, indexed by destination.  Row >= S (AllGather):
  * bytes of the message a rank SENDS to each of its peers, indexed by source.  Host-only. */
-/* UNSUPPORTED for a ring whose size is no power of three (its two messages differ): use the next call. */
+/* UNSUPPORTED for plans with a side that is no power of three (the two messages differ): use the next call. */
 trv_status_t trv_plan_message_bytes(trv_plan_t plan, size_t count, size_t elem_size, int32_t c, int32_t row,
                                     int64_t *bytes);
 

@@ -48,7 +48,8 @@ static trv_status_t check_buffers(const Plan& p, const void* const* in, void* co
 static trv_status_t dispatch(Call& c, trv_kernel_t kernel) {
     const Plan& p = *c.plan;
     bool fused = false;
-    if (kernel == TRV_KERNEL_PIPELINED) return run_pipeline_latency(c);
+    if (kernel == TRV_KERNEL_PIPELINED)
+        return p.variant == TRV_BANDWIDTH_OPTIMAL && !p.general ? run_pipeline_bandwidth(c) : run_pipeline_latency(c);
     if (kernel == TRV_KERNEL_FUSED) {
         if (!fused_supported(p)) return TRV_ERR_UNSUPPORTED;
         fused = true;
@@ -167,7 +168,7 @@ trv_status_t trv_plan_message_bytes_side(trv_plan_t plan, size_t count, size_t e
 int32_t trv_kernel_supported(trv_plan_t plan, trv_kernel_t kernel) {
     if (!plan || plan->plan.algo != TRV_ALGO_TRIVANCE) return 0;
     if (kernel == TRV_KERNEL_FUSED) return fused_supported(plan->plan) ? 1 : 0;
-    if (kernel == TRV_KERNEL_PIPELINED) return pipeline_supported(plan->plan, false) ? 1 : 0;
+    if (kernel == TRV_KERNEL_PIPELINED) return (pipeline_supported(plan->plan, false) || pipeline_bw_supported(plan->plan)) ? 1 : 0;
     return (kernel == TRV_KERNEL_AUTO || kernel == TRV_KERNEL_STEP) ? 1 : 0;
 }
 
@@ -177,6 +178,7 @@ trv_status_t trv_scratch_bytes(trv_plan_t plan, size_t count, trv_kernel_t kerne
     if (p.algo != TRV_ALGO_TRIVANCE) return TRV_ERR_UNSUPPORTED;
     bool fused = false;
     if (kernel == TRV_KERNEL_PIPELINED) {
+        if (pipeline_bw_supported(p)) { *bytes = pipeline_bw_scratch_bytes(p, count); return TRV_OK; }
         if (!pipeline_supported(p, in_place != 0)) return TRV_ERR_UNSUPPORTED;
         *bytes = pipeline_scratch_bytes(p, count);
         return TRV_OK;

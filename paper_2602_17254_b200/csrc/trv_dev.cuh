@@ -240,6 +240,10 @@ size_t pipeline_scratch_bytes(const Plan& p, size_t count);
 trv_status_t run_pipeline_latency(const Call& c);
 trv_status_t pipeline_status(const void* scratch, cudaStream_t st);
 trv_status_t pipeline_selftest_timeout(void* scratch, size_t scratch_bytes, cudaStream_t st);
+// the same engine for the bandwidth-optimal form (trv_pipe_bw.cu)
+bool pipeline_bw_supported(const Plan& p);
+size_t pipeline_bw_scratch_bytes(const Plan& p, size_t gcount);
+trv_status_t run_pipeline_bandwidth(const Call& c);
 
 // link-load tally (trv_linkloads.cu)
 trv_status_t run_link_loads(const Plan& p, size_t count, size_t elem_size, int32_t* msgs, int64_t* bytes,

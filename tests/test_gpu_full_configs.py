@@ -53,8 +53,8 @@ def test_config_every_element(name):
     xd.copy_(torch.from_numpy(xh))
     got2 = run_gpu(plan, xd, binding.KERNEL_STEP).cpu().numpy()
     assert np.array_equal(got.view(np.uint32), got2.view(np.uint32))
-    # and so must the chunk-level readiness engine (latency form only)
-    if w.variant == LAT and plan.kernel_supported(binding.KERNEL_PIPELINED):
+    # and so must the chunk-level readiness engine
+    if plan.kernel_supported(binding.KERNEL_PIPELINED):
         xd.copy_(torch.from_numpy(xh))
         got3 = run_gpu(plan, xd, binding.KERNEL_PIPELINED).cpu().numpy()
         assert np.array_equal(got.view(np.uint32), got3.view(np.uint32))

@@ -21,8 +21,8 @@ def _built():
     binding.lib()
 
 
-def _run(dims, count, dist, seed, in_place=True, shard=None, scattered=False):
-    plan = binding.Plan(dims, LAT)
+def _run(dims, count, dist, seed, in_place=True, shard=None, scattered=False, variant=LAT):
+    plan = binding.Plan(dims, variant)
     n = plan.n
     x = synth.rank_matrix(dist, seed, n, count)
     pad = (count + 3) // 4 * 4 + 4
@@ -36,7 +36,7 @@ def _run(dims, count, dist, seed, in_place=True, shard=None, scattered=False):
         opool = torch.full((n, pad), -77, dtype=pool.dtype, device=DEV)
         outp = [opool[r].data_ptr() for r in range(n)]
     gc, go = (count, 0) if shard is None else shard
-    need = plan.scratch_bytes(count, PIPE, in_place=in_place)
+    need = plan.scratch_bytes(gc if variant == BW else count, PIPE, in_place=in_place)
     assert need > 0
     scratch = torch.empty(need, dtype=torch.uint8, device=DEV)
     before = binding.launch_count()
@@ -44,7 +44,7 @@ def _run(dims, count, dist, seed, in_place=True, shard=None, scattered=False):
                       binding.INT32 if x.dtype == np.int32 else binding.FLOAT32, global_count=gc, global_offset=go,
                       kernel=PIPE, scratch_ptr=scratch.data_ptr(), scratch_bytes=need,
                       stream=torch.cuda.current_stream().cuda_stream)
-    assert binding.last_kernel_name() == "lat_pipe" and binding.launch_count() - before == 1
+    assert binding.last_kernel_name() == ("lat_pipe" if variant == LAT else "bw_pipe") and binding.launch_count() - before == 1
     assert binding.pipeline_status(scratch.data_ptr(), torch.cuda.current_stream().cuda_stream) == binding.OK
     if in_place:
         got = np.stack([rows[r][:count].cpu().numpy() for r in range(n)])
@@ -54,7 +54,7 @@ def _run(dims, count, dist, seed, in_place=True, shard=None, scattered=False):
         got = opool[:, :count].cpu().numpy()
         assert (opool[:, count:] == -77).all().item(), "wrote past the end of a rank buffer"
         assert np.array_equal(np.stack([rows[r][:count].cpu().numpy() for r in range(n)]), x), "input modified"
-    compare(dims, LAT, x, got, E=gc, e0=go)
+    compare(dims, variant, x, got, E=gc, e0=go)
     plan.destroy()
 
 
@@ -68,6 +68,31 @@ def test_matches_oracle(dims):
     _run(dims, count, "normal", 41)
     _run(dims, count, "int32", 42, in_place=False)
     _run(dims, count, "uniform", 43, scattered=True)
+
+
+@pytest.mark.parametrize("dims", SHAPES + [(3,)])
+def test_bandwidth_form_matches_oracle(dims):
+    """Reduce-Scatter and AllGather by the readiness engine: a chunk is a piece of one block (its active block range)."""
+    n = int(np.prod(dims))
+    count = 40009 if n <= 243 else 9001         # blocks of ragged length; the ring of 27 gets blocks of several chunks below
+    _run(dims, count, "normal", 51, variant=BW)
+    _run(dims, count, "int32", 52, in_place=False, variant=BW)
+    _run(dims, count, "uniform", 53, scattered=True, variant=BW)
+
+
+def test_bandwidth_form_blocks_of_several_chunks_and_many_groups():
+    _run((27,), 200003, "normal", 54, variant=BW)                   # 7408 elements per block: four chunks
+    _run((9,), 1500007, "int32", 55, in_place=False, variant=BW)    # 82 chunks per block
+    _run((9, 9), 700001, "normal", 56, variant=BW)
+    _run((3, 3, 3), 5, "int32", 57, variant=BW)                     # most blocks empty
+
+
+@pytest.mark.parametrize("dims", [(27,), (9, 9), (9, 9, 9)])
+def test_bandwidth_form_sharded_window(dims):
+    gcount = 30011
+    for lo, hi in ((0, 15004), (15004, gcount), (7000, 7000 + 4096)):
+        _run(dims, hi - lo, "int32", 58, shard=(gcount, lo), variant=BW)
+        _run(dims, hi - lo, "normal", 59, in_place=False, shard=(gcount, lo), variant=BW)
 
 
 @pytest.mark.parametrize("dims", [(3,), (9,), (27,)])
@@ -97,7 +122,8 @@ def test_unsupported_and_scratch_checks():
     x = torch.zeros((27, 64), dtype=torch.int32, device=DEV)
     ptrs = [x[r].data_ptr() for r in range(27)]
     scratch = torch.empty(1 << 20, dtype=torch.uint8, device=DEV)
-    for dims, variant in (((27,), BW), ((10,), BW)):
+    assert binding.Plan((27,), BW).kernel_supported(PIPE)
+    for dims, variant in (((10,), BW), ((4, 4), BW)):
         plan = binding.Plan(dims, variant)
         assert not plan.kernel_supported(PIPE)
         with pytest.raises(binding.TrivanceError) as e:
