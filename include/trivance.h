@@ -248,6 +248,21 @@ trv_status_t trv_allreduce_noalloc(trv_plan_t plan, void *const *rank_buffers, s
                                    trv_op_t op, void *cuda_stream);
 size_t trv_noalloc_max_scratch_bytes(void);
 
+/* ---------------------------------------------------------------- one joint reduction on caller-described segments
+ *
+ * out[s][e] = (left[s][e] + own[s][e]) + right[s][e] for e < counts[s], s < nsegments: the joint reduction of the two
+ * received partials with the local one (Sec. 3.1, 4.2), in the association order of trv_allreduce.  A NULL left[s] or
+ * right[s] (or a NULL array) leaves that side out: left + own, own + right, or a copy.  It serves schedules whose steps
+ * are driven from outside the library, above all the rank-sharded form in which every process holds the partials of its
+ * own ranks and the partials of the ranks at distance 3^k arrive in receive buffers (Discussion; App. D).
+ *   left, own, right, out: HOST arrays of nsegments DEVICE pointers, 4-byte aligned (16-byte accesses are used where a
+ *                 segment's pointers share their alignment); out[s] may equal own[s]; no out[] may overlap a left[] or
+ *                 right[] of the same call
+ *   counts      : HOST array of element counts
+ * Asynchronous on cuda_stream; allocates nothing.  Errors: INVALID_ARG, UNSUPPORTED (a count of 2^40 or more), CUDA. */
+trv_status_t trv_joint_reduce(const void *const *left, const void *const *own, const void *const *right, void *const *out,
+                              const size_t *counts, size_t nsegments, trv_dtype_t dtype, void *cuda_stream);
+
 /* ---------------------------------------------------------------- PIPELINED family: status
  *
  * The PIPELINED kernel (App. D; Discussion, "Joint Reduction Overheads") waits on readiness entries

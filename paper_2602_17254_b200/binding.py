@@ -30,7 +30,7 @@ SYMBOLS = [
     "trv_kernel_supported", "trv_allreduce_ex", "trv_allreduce_host", "trv_host_workspace_bytes",
     "trv_link_loads", "trv_plan_message_bytes", "trv_plan_message_bytes_side", "trv_strerror", "trv_launch_count", "trv_last_kernel_name",
     "trv_allreduce_noalloc", "trv_noalloc_max_scratch_bytes", "trv_cost_model", "trv_pipeline_status",
-    "trv_pipeline_selftest_timeout", "trv_tma_giveups", "trv_plan_reserve_scratch",
+    "trv_pipeline_selftest_timeout", "trv_tma_giveups", "trv_plan_reserve_scratch", "trv_joint_reduce",
 ]
 
 
@@ -73,6 +73,7 @@ def lib():
         L.trv_pipeline_selftest_timeout.argtypes = [vp, sz, vp]
         L.trv_allreduce.argtypes = [vp, vp, sz, ctypes.c_int, ctypes.c_int, vp]
         L.trv_plan_reserve_scratch.argtypes = [vp, sz]
+        L.trv_joint_reduce.argtypes = [vp, vp, vp, vp, vp, sz, ctypes.c_int, vp]
         L.trv_scratch_bytes.argtypes = [vp, sz, ctypes.c_int, i32, ctypes.POINTER(sz)]
         L.trv_kernel_supported.argtypes = [vp, ctypes.c_int]
         L.trv_kernel_supported.restype = i32
@@ -116,6 +117,15 @@ def tma_giveups():
     v = ctypes.c_uint32()
     _check(lib().trv_tma_giveups(ctypes.byref(v)), "trv_tma_giveups")
     return v.value
+
+
+def joint_reduce(left, own, right, out, counts, dtype, stream=0):
+    """trv_joint_reduce: out[s] = (left[s] + own[s]) + right[s] on segments given as lists of device addresses (0 = side left out)."""
+    k = len(own)
+    arr = lambda p: None if p is None else (ctypes.c_void_p * k)(*[int(v) if v else None for v in p])
+    cnt = (ctypes.c_size_t * k)(*[int(c) for c in counts])
+    _check(lib().trv_joint_reduce(arr(left), arr(own), arr(right), arr(out), cnt, k, int(dtype), ctypes.c_void_p(int(stream))),
+           "trv_joint_reduce")
 
 
 def launch_count():
