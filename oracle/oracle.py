@@ -190,6 +190,27 @@ def allreduce(dims, variant, x, E=None, e0=0, max_steps=-1, counters=False):
     return out
 
 
+def allreduce_algo(dims, variant, x, algo, E=None, e0=0, counters=False):
+    """AllReduce of x by a comparator schedule (Bruck, Recursive Doubling, Swing, Bucket; ``| ALGO_MIRROR`` adds the
+    mirrored sub-collective on the other half of the vector), executed message by message; as ``allreduce``."""
+    x = np.ascontiguousarray(x)
+    if x.dtype not in _DTYPES or x.ndim != 2:
+        raise TypeError("x must be a 2-D int32, float32 or float64 array")
+    n, w = x.shape
+    if E is None:
+        E = w
+    out = np.empty_like(x)
+    _, p, nd = _dims(dims)
+    ctr = [np.zeros(n, np.int64) for _ in range(3)] if counters else [None] * 3
+    ptr = [c.ctypes.data_as(ctypes.c_void_p) if c is not None else None for c in ctr]
+    _check(_load().orc_allreduce_algo(p, nd, ctypes.c_int(variant), ctypes.c_int(algo), ctypes.c_int(_DTYPES[x.dtype]),
+                                      ctypes.c_int64(E), ctypes.c_int64(e0), ctypes.c_int64(e0 + w),
+                                      x.ctypes.data_as(ctypes.c_void_p), out.ctypes.data_as(ctypes.c_void_p), *ptr))
+    if counters:
+        return out, {"sent_rs": ctr[0], "sent_ag": ctr[1], "reduced": ctr[2]}
+    return out
+
+
 def link_loads(dims, variant, E, elem_size=4, algo=ALGO_TRIVANCE):
     """Per-step link loads: dict with msgs/bytes [T][n][D][2] and max_msgs/max_bytes [T]."""
     if _general_ring(dims, algo):

@@ -1127,3 +1127,127 @@ done:
     free(par); free(stp); free(lm); free(lb); free(mb); free(mc);
     return rc;
 }
+
+/* ------------------------------------------------------------------ comparator schedules as data paths (Sec. 2.4, 3.1) */
+
+/*
+ * The comparison algorithms of the paper -- Bruck with joint reductions (Sec. 3.1; peers r + 3^k and r + 2 3^k),
+ * Recursive Doubling (peer r XOR 2^k), Swing (peer r +- rho(k)), the ring (Bucket) algorithm, each optionally with
+ * its mirrored sub-collective on the other half of the vector (Sec. 2.4) -- executed literally: in every step every
+ * rank puts a message for each of its peers on the wire, then every rank reduces what it received.
+ *   latency form   : a message is the sender's whole current partial of the collective's slice;
+ *   bandwidth form : Reduce-Scatter: the message to peer p carries the blocks p still answers for after the step
+ *                    (p's own and all it forwards later: the same sets the link-load tally uses); AllGather: the
+ *                    steps in reverse order, a rank sends every finished block it holds to the step's peers.
+ *                    Bucket: step t passes block r - t - 1 (Reduce-Scatter) resp. r - t (AllGather) to r + 1.
+ * Reading (PARITY UNPINNED by the paper, which never states an association order): a rank that receives m0 from the
+ * sender whose FIRST peer it is and m1 from the sender whose SECOND peer it is forms (m1 + own) + m0; with one
+ * message own + m0.  For Trivance's peers (first = left, second = right) this is (from_left + own) + from_right.
+ */
+#define DEFINE_ALGO(T, SUFFIX, ADD)                                                                            \
+static int algo_slice_##SUFFIX(const orc_topo *tp, int c, int variant, int64_t slo, int64_t shi, int64_t e0,    \
+                               int64_t e1, int64_t w, T *data, orc_counters *ctr) {                             \
+    int n = tp->n, S = tp->S, rc = ORC_OK;                                                                      \
+    int64_t c0 = clampi(slo, e0, e1) - e0, c1 = clampi(shi, e0, e1) - e0, wc = c1 - c0;                         \
+    if (wc <= 0) return ORC_OK;                                                                                 \
+    int sd[64], sx[64];                                                                                         \
+    int sg = c >= tp->ndims ? -1 : 1;                                                                           \
+    if (tp->algo != ORC_BUCKET) step_list(tp, c, sd, sx);                                                       \
+    int64_t *bs = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n + 1));                                         \
+    T *wire = (T *)malloc(sizeof(T) * (size_t)n * (size_t)wc);       /* what every rank puts on the wire */       \
+    int *from = (int *)malloc(sizeof(int) * (size_t)n * 2);          /* from[2p+k]: the sender whose k-th peer is p */\
+    uint8_t *set = (uint8_t *)malloc((size_t)n);                                                                \
+    uint8_t *have = (uint8_t *)calloc((size_t)n, (size_t)n), *snap = (uint8_t *)malloc((size_t)n * (size_t)n);  \
+    if (!bs || !wire || !from || !set || !have || !snap) { rc = ORC_NOMEM; goto done; }                         \
+    for (int j = 0; j <= n; ++j) bs[j] = clampi(block_bound(slo, shi, n, j), e0, e1) - e0;                      \
+    for (int t = 0; t < S; ++t) {                                   /* ---- latency form, or Reduce-Scatter */   \
+        for (int r = 0; r < n; ++r) memcpy(wire + (size_t)r * wc, data + (size_t)r * w + c0, sizeof(T) * (size_t)wc); \
+        for (int i = 0; i < 2 * n; ++i) from[i] = -1;                                                           \
+        for (int r = 0; r < n; ++r) {                                                                           \
+            int peer[2] = {-1, -1}, dir[2], hops[2];                                                            \
+            int np = tp->algo == ORC_BUCKET ? 1 : send_peers(tp, r, sd[t], sx[t], peer, dir, hops);             \
+            if (tp->algo == ORC_BUCKET) peer[0] = ((r + sg) % n + n) % n;                                       \
+            for (int k = 0; k < np; ++k) {                                                                      \
+                if (from[2 * peer[k] + k] >= 0) { rc = ORC_INTERNAL; goto done; }                               \
+                from[2 * peer[k] + k] = r;                                                                      \
+            }                                                                                                   \
+        }                                                                                                       \
+        for (int p = 0; p < n; ++p) {                                                                           \
+            int r0 = from[2 * p], r1 = from[2 * p + 1];                                                         \
+            if (variant == ORC_LATENCY) memset(set, 1, (size_t)n);                                              \
+            else if (tp->algo == ORC_BUCKET) { memset(set, 0, (size_t)n); set[(((p - sg * (t + 2)) % n) + n) % n] = 1; } \
+            else send_set(tp, sd, sx, p, t, set);                                                               \
+            for (int j = 0; j < n; ++j) if (set[j]) {                                                           \
+                T *own = data + (size_t)p * w + bs[j];                                                          \
+                int64_t bl = bs[j + 1] - bs[j];                                                                 \
+                const T *m0 = r0 >= 0 ? wire + (size_t)r0 * wc + (bs[j] - c0) : NULL;                           \
+                const T *m1 = r1 >= 0 ? wire + (size_t)r1 * wc + (bs[j] - c0) : NULL;                           \
+                for (int64_t e = 0; e < bl; ++e) {                                                              \
+                    T acc = own[e];                                                                             \
+                    if (m1) acc = ADD(m1[e], acc);                                                              \
+                    if (m0) acc = ADD(acc, m0[e]);                                                              \
+                    own[e] = acc;                                                                               \
+                }                                                                                               \
+                if (ctr && ctr->sent_rs) {                                                                      \
+                    if (r0 >= 0) ctr->sent_rs[r0] += (int64_t)sizeof(T) * bl;                                   \
+                    if (r1 >= 0) ctr->sent_rs[r1] += (int64_t)sizeof(T) * bl;                                   \
+                }                                                                                               \
+                if (ctr && ctr->reduced) ctr->reduced[p] += (int64_t)sizeof(T) * bl * (1 + (r0 >= 0) + (r1 >= 0)); \
+            }                                                                                                   \
+        }                                                                                                       \
+    }                                                                                                           \
+    if (variant == ORC_BANDWIDTH) {                                 /* ---- AllGather */                        \
+        for (int r = 0; r < n; ++r) have[(size_t)r * n + r] = 1;                                                \
+        for (int row = 0; row < S; ++row) {                                                                     \
+            int t = S - 1 - row;                                                                                \
+            memcpy(snap, have, (size_t)n * (size_t)n);                                                          \
+            for (int r = 0; r < n; ++r) memcpy(wire + (size_t)r * wc, data + (size_t)r * w + c0, sizeof(T) * (size_t)wc); \
+            for (int r = 0; r < n; ++r) {                                                                       \
+                int peer[2] = {-1, -1}, dir[2], hops[2];                                                        \
+                int np = tp->algo == ORC_BUCKET ? 1 : send_peers(tp, r, sd[t], sx[t], peer, dir, hops);         \
+                if (tp->algo == ORC_BUCKET) peer[0] = ((r + sg) % n + n) % n;                                   \
+                for (int k = 0; k < np; ++k)                                                                    \
+                    for (int j = 0; j < n; ++j) {                                                               \
+                        int sends = tp->algo == ORC_BUCKET ? (j == (((r - sg * row) % n) + n) % n) : snap[(size_t)r * n + j]; \
+                        if (!sends) continue;                                                                   \
+                        if (have[(size_t)peer[k] * n + j]) { rc = ORC_INTERNAL; goto done; }     /* never twice */ \
+                        memcpy(data + (size_t)peer[k] * w + bs[j], wire + (size_t)r * wc + (bs[j] - c0),        \
+                               sizeof(T) * (size_t)(bs[j + 1] - bs[j]));                                        \
+                        have[(size_t)peer[k] * n + j] = 1;                                                      \
+                        if (ctr && ctr->sent_ag) ctr->sent_ag[r] += (int64_t)sizeof(T) * (bs[j + 1] - bs[j]);   \
+                    }                                                                                           \
+            }                                                                                                   \
+        }                                                                                                       \
+        for (size_t i = 0; i < (size_t)n * (size_t)n; ++i) if (!have[i]) { rc = ORC_INTERNAL; goto done; }      \
+    }                                                                                                           \
+done:                                                                                                           \
+    free(bs); free(wire); free(from); free(set); free(have); free(snap);                                        \
+    return rc;                                                                                                  \
+}
+DEFINE_ALGO(uint32_t, i32, ADD_WRAP)
+DEFINE_ALGO(float, f32, ADD_FP)
+DEFINE_ALGO(double, f64, ADD_FP)
+
+/* AllReduce by a comparator schedule (algo may carry ORC_MIRROR); arguments as orc_allreduce. */
+int orc_allreduce_algo(const int32_t *dims, int ndims, int variant, int algo, int dtype, int64_t E, int64_t e0, int64_t e1,
+                       const void *in, void *out, int64_t *sent_rs, int64_t *sent_ag, int64_t *reduced) {
+    orc_topo tp; int rc = topo_init(&tp, dims, ndims, algo);
+    if (rc) return rc;
+    if (E < 0 || e0 < 0 || e1 < e0 || e1 > E || !in || !out) return ORC_BAD_ARG;
+    if (variant != ORC_LATENCY && variant != ORC_BANDWIDTH) return ORC_BAD_ARG;
+    if (dtype != ORC_I32 && dtype != ORC_F32 && dtype != ORC_F64) return ORC_BAD_ARG;
+    if (tp.algo == ORC_BUCKET && variant != ORC_BANDWIDTH) return ORC_UNDEFINED;
+    if (tp.S > 64 && tp.algo != ORC_BUCKET) return ORC_BAD_ARG;
+    orc_counters ctr = { sent_rs, sent_ag, reduced };
+    int64_t w = e1 - e0;
+    size_t es = dtype == ORC_F64 ? 8 : 4;
+    memcpy(out, in, es * (size_t)tp.n * (size_t)w);         /* the partials live in `out` */
+    for (int c = 0; c < tp.nsl && rc == ORC_OK; ++c) {
+        int64_t slo, shi;
+        slice_bounds(E, tp.nsl, c, &slo, &shi);
+        if (dtype == ORC_I32) rc = algo_slice_i32(&tp, c, variant, slo, shi, e0, e1, w, (uint32_t *)out, &ctr);
+        else if (dtype == ORC_F32) rc = algo_slice_f32(&tp, c, variant, slo, shi, e0, e1, w, (float *)out, &ctr);
+        else rc = algo_slice_f64(&tp, c, variant, slo, shi, e0, e1, w, (double *)out, &ctr);
+    }
+    return rc;
+}

@@ -164,3 +164,86 @@ def test_mirror_flag_is_for_ring_comparators_only():
     with pytest.raises(binding.TrivanceError) as e:
         binding.Plan((12,), BW, oracle.ALGO_SWING)
     assert e.value.status == binding.ERR_UNDEFINED_SCHEDULE
+
+
+# ------------------------------------------------------------------ the comparators as data paths (Sec. 2.4, 3.1)
+
+DATA_ALGOS = [(oracle.ALGO_BRUCK, [3, 9, 27]), (oracle.ALGO_RECDOUB, [2, 4, 8, 16]), (oracle.ALGO_SWING, [2, 4, 8, 16, 32]),
+              (oracle.ALGO_BUCKET, [2, 3, 5, 8, 12])]
+
+
+@pytest.mark.parametrize("algo,sizes", DATA_ALGOS)
+@pytest.mark.parametrize("mirror", [0, oracle.ALGO_MIRROR])
+def test_comparator_paths_give_the_column_sums_and_the_modelled_bytes(algo, sizes, mirror):
+    """Every rank ends with the sum of all inputs (int32, wrapping); the bytes each node put on the wire are the ones
+    the link-load model counts for the same schedule."""
+    for n in sizes:
+        for variant in (0, 1):
+            if algo == oracle.ALGO_BUCKET and variant == 0:
+                with pytest.raises(oracle.OracleError):
+                    oracle.allreduce_algo((n,), 0, np.zeros((n, 4), np.int32), algo)
+                continue
+            E = 3 * n + 5
+            x = np.random.default_rng(n).integers(-2 ** 31, 2 ** 31 - 1, size=(n, E), dtype=np.int64).astype(np.int32)
+            y, ctr = oracle.allreduce_algo((n,), variant, x, algo | mirror, counters=True)
+            assert (y == x.astype(np.int64).sum(0).astype(np.int32)[None]).all()
+            assert np.array_equal(ctr["sent_rs"] + ctr["sent_ag"], oracle.bytes_sent((n,), variant, E, 4, algo | mirror))
+            part = oracle.allreduce_algo((n,), variant, np.ascontiguousarray(x[:, 2:E - 3]), algo | mirror, E=E, e0=2)
+            assert np.array_equal(part, y[:, 2:E - 3])          # a window gives the full run's columns
+
+
+@pytest.mark.parametrize("dims", [(9,), (27,), (3, 3), (9, 9), (3, 9), (3, 3, 3)])
+@pytest.mark.parametrize("variant", [0, 1])
+def test_generic_path_with_trivance_peers_is_the_trivance_path(dims, variant):
+    """The message-by-message executor of the comparators, given Trivance's own peers, reproduces the dedicated
+    Trivance oracle bit for bit: its association rule (m1 + own) + m0 is (from_left + own) + from_right there."""
+    n = int(np.prod(dims))
+    x = np.random.default_rng(n).standard_normal((n, 5 * n + 3)).astype(np.float32)
+    a = oracle.allreduce_algo(dims, variant, x, oracle.ALGO_TRIVANCE)
+    b = oracle.allreduce(dims, variant, x)
+    assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
+def _swing_peer(p, k, n):
+    rho = sum((-2) ** i for i in range(k + 1))
+    return (p + rho) % n if p % 2 == 0 else (p - rho) % n
+
+
+@pytest.mark.parametrize("algo,n", [(oracle.ALGO_RECDOUB, 8), (oracle.ALGO_RECDOUB, 32), (oracle.ALGO_SWING, 8), (oracle.ALGO_SWING, 32),
+                                    (oracle.ALGO_BRUCK, 9), (oracle.ALGO_BRUCK, 27)])
+def test_latency_forms_against_their_step_formulas(algo, n):
+    """Sec. 2.4 / 3.1: Recursive Doubling v[p] += v[p XOR 2^k]; Swing v[p] += v[pi(p, k)]; Bruck with joint reductions
+    v[p] = (v[p - 2 3^k] + v[p]) + v[p - 3^k] (the reading of the association order), step by step in binary32."""
+    x = (np.random.default_rng(n).standard_normal((n, 64)) * 100).astype(np.float32)
+    v = x.copy()
+    if algo == oracle.ALGO_BRUCK:
+        d = 1
+        while d < n:
+            v = (np.roll(v, 2 * d, axis=0) + v) + np.roll(v, d, axis=0)
+            d *= 3
+    else:
+        k = 0
+        while (1 << k) < n:
+            perm = [p ^ (1 << k) for p in range(n)] if algo == oracle.ALGO_RECDOUB else [_swing_peer(p, k, n) for p in range(n)]
+            v = v + v[perm]
+            k += 1
+    got = oracle.allreduce_algo((n,), 0, x, algo)
+    assert np.array_equal(got.view(np.uint32), v.view(np.uint32))
+    exact = x.astype(np.float64).sum(0)
+    assert (np.abs(got.astype(np.float64) - exact[None]) <= 2e-6 * np.abs(x.astype(np.float64)).sum(0)[None]).all()
+
+
+@pytest.mark.parametrize("algo,n", [(oracle.ALGO_RECDOUB, 16), (oracle.ALGO_SWING, 16), (oracle.ALGO_BRUCK, 27), (oracle.ALGO_BUCKET, 7)])
+def test_bandwidth_forms_all_rows_equal_and_blocks_are_the_owners_latency_rows(algo, n):
+    E = 4 * n + 3
+    rng = np.random.default_rng(n)
+    x = (rng.standard_normal((n, E)) * 10.0 ** rng.integers(-3, 4, size=(n, E))).astype(np.float32)
+    bw = oracle.allreduce_algo((n,), 1, x, algo)
+    assert all(np.array_equal(bw[0].view(np.uint32), bw[r].view(np.uint32)) for r in range(n))
+    if algo != oracle.ALGO_BUCKET:      # Reduce-Scatter is the latency pattern restricted to the blocks on their way to the owner
+        lat = oracle.allreduce_algo((n,), 0, x, algo)
+        bb = oracle.block_bounds(E, 1, n)
+        for j in range(n):
+            assert np.array_equal(bw[j, bb[j]:bb[j + 1]].view(np.uint32), lat[j, bb[j]:bb[j + 1]].view(np.uint32))
+    xi = rng.integers(-100, 100, size=(n, E)).astype(np.float32)      # small integers: exact, equals the int path
+    assert np.array_equal(oracle.allreduce_algo((n,), 1, xi, algo), oracle.allreduce_algo((n,), 1, xi.astype(np.int32), algo).astype(np.float32))
