@@ -110,8 +110,15 @@ trv_status_t trv_plan_create(const int32_t *dims, int32_t ndims, trv_variant_t v
  * direction reversed, the two sharing the vector half and half (the mirrored sub-collective by
  * which these one-port schedules use both ports, Sec. 2.4); the plan then has two collectives
  * (trv_plan_slices), the second one with negated distances.
- * Comparator plans serve trv_link_loads, trv_cost_model and the schedule queries only;
- * trv_allreduce returns UNSUPPORTED for them. */
+ * Comparator plans serve trv_link_loads, trv_cost_model and the schedule queries, and they are executable:
+ * trv_allreduce / trv_allreduce_ex (TRV_KERNEL_AUTO or TRV_KERNEL_STEP) run them step by step, literally -- at
+ * the start of a step every rank's vector is copied to a wire buffer (scratch of n * round_up(count, 64) * 4
+ * bytes, trv_scratch_bytes), then every rank reduces what its senders put there: the whole slice in the latency
+ * form; in the bandwidth form the blocks the receiver still answers for (Reduce-Scatter) and every finished block
+ * the sender holds (AllGather, steps reversed).  TRV_ALGO_BRUCK is Bruck with joint reductions (Sec. 3.1).  The
+ * paper states no association order; here a rank that gets m0 from the sender whose first peer it is and m1 from
+ * the sender whose second peer it is forms (m1 + own) + m0, with one message own + m0.  They are baselines: no
+ * fused or pipelined kernel family exists for them (UNSUPPORTED), and trv_allreduce_host is Trivance only. */
 trv_status_t trv_plan_create_algo(const int32_t *dims, int32_t ndims, trv_variant_t variant, trv_algo_t algo,
                                   trv_plan_t *out);
 

@@ -166,7 +166,11 @@ trv_status_t trv_plan_message_bytes_side(trv_plan_t plan, size_t count, size_t e
 }
 
 int32_t trv_kernel_supported(trv_plan_t plan, trv_kernel_t kernel) {
-    if (!plan || plan->plan.algo != TRV_ALGO_TRIVANCE) return 0;
+    if (!plan) return 0;
+    if (plan->plan.algo != TRV_ALGO_TRIVANCE) {
+        if (plan->plan.algo == TRV_ALGO_BUCKET && plan->plan.variant != TRV_BANDWIDTH_OPTIMAL) return 0;
+        return (kernel == TRV_KERNEL_AUTO || kernel == TRV_KERNEL_STEP) ? 1 : 0;
+    }
     if (kernel == TRV_KERNEL_FUSED) return fused_supported(plan->plan) ? 1 : 0;
     if (kernel == TRV_KERNEL_PIPELINED) return (pipeline_supported(plan->plan, false) || pipeline_bw_supported(plan->plan)) ? 1 : 0;
     return (kernel == TRV_KERNEL_AUTO || kernel == TRV_KERNEL_STEP) ? 1 : 0;
@@ -175,7 +179,12 @@ int32_t trv_kernel_supported(trv_plan_t plan, trv_kernel_t kernel) {
 trv_status_t trv_scratch_bytes(trv_plan_t plan, size_t count, trv_kernel_t kernel, int32_t in_place, size_t* bytes) {
     if (!plan || !bytes) return TRV_ERR_INVALID_ARG;
     const Plan& p = plan->plan;
-    if (p.algo != TRV_ALGO_TRIVANCE) return TRV_ERR_UNSUPPORTED;
+    if (p.algo != TRV_ALGO_TRIVANCE) {      // comparator schedules: the step-by-step executor and its wire buffer
+        if (kernel != TRV_KERNEL_AUTO && kernel != TRV_KERNEL_STEP) return TRV_ERR_UNSUPPORTED;
+        if (p.algo == TRV_ALGO_BUCKET && p.variant != TRV_BANDWIDTH_OPTIMAL) return TRV_ERR_UNSUPPORTED;
+        *bytes = comparator_scratch_bytes(p, count);
+        return TRV_OK;
+    }
     bool fused = false;
     if (kernel == TRV_KERNEL_PIPELINED) {
         if (pipeline_bw_supported(p)) { *bytes = pipeline_bw_scratch_bytes(p, count); return TRV_OK; }
@@ -200,7 +209,8 @@ trv_status_t trv_allreduce_ex(trv_plan_t plan, const void* const* in_buffers, vo
                               trv_kernel_t kernel, void* scratch, size_t scratch_bytes, void* cuda_stream) {
     if (!plan) return TRV_ERR_INVALID_ARG;
     const Plan& p = plan->plan;
-    if (p.algo != TRV_ALGO_TRIVANCE) return TRV_ERR_UNSUPPORTED;
+    if (p.algo != TRV_ALGO_TRIVANCE && kernel != TRV_KERNEL_AUTO && kernel != TRV_KERNEL_STEP) return TRV_ERR_UNSUPPORTED;
+    if (p.algo == TRV_ALGO_BUCKET && p.variant != TRV_BANDWIDTH_OPTIMAL) return TRV_ERR_UNSUPPORTED;
     if (dtype != TRV_INT32 && dtype != TRV_FLOAT32) return TRV_ERR_INVALID_ARG;
     if (op != TRV_SUM) return TRV_ERR_UNSUPPORTED;
     if (kernel != TRV_KERNEL_AUTO && kernel != TRV_KERNEL_STEP && kernel != TRV_KERNEL_FUSED && kernel != TRV_KERNEL_PIPELINED)
@@ -214,6 +224,7 @@ trv_status_t trv_allreduce_ex(trv_plan_t plan, const void* const* in_buffers, vo
     if (count == 0) return TRV_OK;
     Call c{&p, in_buffers, out_buffers, count, global_count, global_offset, (int)dtype, in_place,
            scratch, scratch_bytes, (cudaStream_t)cuda_stream};
+    if (p.algo != TRV_ALGO_TRIVANCE) return run_comparator(c);
     return dispatch(c, kernel);
 }
 

@@ -245,6 +245,12 @@ bool pipeline_bw_supported(const Plan& p);
 size_t pipeline_bw_scratch_bytes(const Plan& p, size_t gcount);
 trv_status_t run_pipeline_bandwidth(const Call& c);
 
+// joint reduction on host-described segments (trv_joint.cu); the comparator schedules run through it (trv_comparator.cu)
+trv_status_t joint_run(const void* const* left, const void* const* own, const void* const* right, void* const* out,
+                       const size_t* counts, size_t nsegments, int dtype, cudaStream_t st);
+size_t comparator_scratch_bytes(const Plan& p, size_t count);
+trv_status_t run_comparator(const Call& c);
+
 // link-load tally (trv_linkloads.cu)
 trv_status_t run_link_loads(const Plan& p, size_t count, size_t elem_size, int32_t* msgs, int64_t* bytes,
                             int32_t* max_msgs, int64_t* max_bytes);

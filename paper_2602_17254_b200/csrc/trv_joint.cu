@@ -66,21 +66,10 @@ __global__ void __launch_bounds__(kJointThreads) k_joint_reduce(const __grid_con
 
 }  // namespace trv
 
-using namespace trv;
-
-extern "C" trv_status_t trv_joint_reduce(const void* const* left, const void* const* own, const void* const* right, void* const* out,
-                                         const size_t* counts, size_t nsegments, trv_dtype_t dtype, void* cuda_stream) {
-    if (!own || !out || !counts) return TRV_ERR_INVALID_ARG;
-    if (dtype != TRV_INT32 && dtype != TRV_FLOAT32) return TRV_ERR_INVALID_ARG;
-    for (size_t s = 0; s < nsegments; ++s) {
-        if (counts[s] == 0) continue;
-        if (!own[s] || !out[s]) return TRV_ERR_INVALID_ARG;
-        if (((uintptr_t)own[s] | (uintptr_t)out[s] | (uintptr_t)(left ? left[s] : nullptr) | (uintptr_t)(right ? right[s] : nullptr)) & 3)
-            return TRV_ERR_INVALID_ARG;
-        if (counts[s] >= ((size_t)1 << 40)) return TRV_ERR_UNSUPPORTED;
-    }
+namespace trv {
+trv_status_t joint_run(const void* const* left, const void* const* own, const void* const* right, void* const* out,
+                       const size_t* counts, size_t nsegments, int dtype, cudaStream_t st) {
     static thread_local JointBatch b;        // 20 KB: kept off the stack
-    cudaStream_t st = (cudaStream_t)cuda_stream;
     size_t s = 0;
     while (s < nsegments) {
         int k = 0;
@@ -100,6 +89,24 @@ extern "C" trv_status_t trv_joint_reduce(const void* const* left, const void* co
         else TRV_LAUNCH(k_joint_reduce<uint32_t>, dim3((unsigned)gx, k, 1), kJointThreads, 0, st, b);
         if (cudaGetLastError() != cudaSuccess) return TRV_ERR_CUDA;
     }
-    g_last_kernel = "joint_reduce";
     return TRV_OK;
+}
+}  // namespace trv
+
+using namespace trv;
+
+extern "C" trv_status_t trv_joint_reduce(const void* const* left, const void* const* own, const void* const* right, void* const* out,
+                                         const size_t* counts, size_t nsegments, trv_dtype_t dtype, void* cuda_stream) {
+    if (!own || !out || !counts) return TRV_ERR_INVALID_ARG;
+    if (dtype != TRV_INT32 && dtype != TRV_FLOAT32) return TRV_ERR_INVALID_ARG;
+    for (size_t s = 0; s < nsegments; ++s) {
+        if (counts[s] == 0) continue;
+        if (!own[s] || !out[s]) return TRV_ERR_INVALID_ARG;
+        if (((uintptr_t)own[s] | (uintptr_t)out[s] | (uintptr_t)(left ? left[s] : nullptr) | (uintptr_t)(right ? right[s] : nullptr)) & 3)
+            return TRV_ERR_INVALID_ARG;
+        if (counts[s] >= ((size_t)1 << 40)) return TRV_ERR_UNSUPPORTED;
+    }
+    const trv_status_t st = joint_run(left, own, right, out, counts, nsegments, (int)dtype, (cudaStream_t)cuda_stream);
+    g_last_kernel = "joint_reduce";
+    return st;
 }

@@ -87,10 +87,13 @@ def test_allreduce_argument_errors_are_found_before_any_launch(library):
     with pytest.raises(binding.TrivanceError) as e:
         p.allreduce_ex(good, [g + 16 for g in good], 16, binding.FLOAT32)
     assert e.value.status == binding.ERR_INVALID_ARG
-    # comparator plans are for link loads only
+    # comparator plans run step by step through a wire buffer: without one the call is refused before any launch
     b = binding.Plan([9], binding.LATENCY_OPTIMAL, binding.ALGO_BRUCK)
     with pytest.raises(binding.TrivanceError) as e:
         b.allreduce_ex(good, None, 16, binding.FLOAT32)
+    assert e.value.status == binding.ERR_SCRATCH
+    with pytest.raises(binding.TrivanceError) as e:
+        b.allreduce_ex(good, None, 16, binding.FLOAT32, kernel=binding.KERNEL_FUSED)
     assert e.value.status == binding.ERR_UNSUPPORTED
     # count == 0 is fine and launches nothing
     p.allreduce_ex(good, None, 0, binding.FLOAT32)
