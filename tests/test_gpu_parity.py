@@ -281,6 +281,6 @@ def test_calls_can_be_captured_in_a_cuda_graph():
 def test_tma_fed_kernels_never_gave_up():
     """The bounded wait of the TMA-fed 9x9x9 kernel did not run out in any call of this process."""
     check_case((9, 9, 9), LAT, 2051, "normal", 91, FUSED)
-    assert binding.last_kernel_name() == "lat_t999_tma"
+    assert binding.last_kernel_name() == "lat_t999_planes"
     check_case((9, 9, 9), LAT, 1031, "int32", 92, FUSED, in_place=False)
     assert binding.tma_giveups() == 0
