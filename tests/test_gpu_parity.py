@@ -221,6 +221,39 @@ def test_plan_owned_scratch_is_bound_to_its_device_and_can_be_reserved():
     fused.reserve_scratch(10 ** 6)
 
 
+def test_plan_scratch_grows_safely_under_concurrent_host_threads():
+    """Two host threads call trv_allreduce on ONE plan whose shape needs the plan-owned scratch, with growing vector
+    lengths, on one stream (so the calls do not overlap on the device, as the header asks).  The grow path is
+    serialised inside the plan: no double free, no dangling scratch, every result equals the oracle's."""
+    import threading
+    dims = (243, 3)
+    plan = binding.Plan(dims, LAT)
+    stream = torch.cuda.current_stream().cuda_stream
+    counts = [64, 700, 260, 1500, 128, 3000]
+    xs = {c: synth.rank_matrix("int32", 90 + c, plan.n, c) for c in counts}
+    bufs = {(t, c): torch.from_numpy(xs[c]).to(DEV) for t in range(2) for c in counts}
+    errors = []
+
+    def worker(t):
+        try:
+            for c in (counts if t == 0 else counts[::-1]):
+                xd = bufs[(t, c)]
+                plan.allreduce([xd[r].data_ptr() for r in range(plan.n)], c, binding.INT32, stream)
+        except Exception as e:      # pragma: no cover
+            errors.append(e)
+
+    threads = [threading.Thread(target=worker, args=(t,)) for t in range(2)]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    torch.cuda.synchronize()
+    assert not errors
+    for (t, c), xd in bufs.items():
+        compare(dims, LAT, xs[c], xd.cpu().numpy())
+    plan.destroy()
+
+
 def test_fp32_tolerance_against_naive_and_exact_sums():
     """|err| <= 2e-6 * sum|x| against the naive sequential binary32 sum (and the fp64 sum)."""
     for dims, variant, dist in [((27,), LAT, "normal"), ((81,), BW, "normal"), ((9, 9, 9), LAT, "uniform"),
