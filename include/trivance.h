@@ -39,7 +39,7 @@ typedef enum {
 
 typedef enum { TRV_LATENCY_OPTIMAL = 0, TRV_BANDWIDTH_OPTIMAL = 1 } trv_variant_t;
 typedef enum { TRV_ALGO_TRIVANCE = 0, TRV_ALGO_BRUCK = 1, TRV_ALGO_RECDOUB = 2, TRV_ALGO_SWING = 3, TRV_ALGO_BUCKET = 4,
-               TRV_ALGO_MIRRORED = 16 /* flag, see trv_plan_create_algo */ } trv_algo_t;
+               TRV_ALGO_MIRRORED = 16, TRV_ALGO_SINGLE = 32 /* flags, see trv_plan_create_algo */ } trv_algo_t;
 typedef enum { TRV_INT32 = 0, TRV_FLOAT32 = 1 } trv_dtype_t;
 typedef enum { TRV_SUM = 0 } trv_op_t;
 
@@ -106,10 +106,15 @@ trv_status_t trv_plan_create(const int32_t *dims, int32_t ndims, trv_variant_t v
  * message the short way round; block sets by Algorithm 1.  TRV_ALGO_BUCKET: the ring algorithm,
  * n - 1 steps per phase on a ring of any n >= 2, every step one block to the next node (bandwidth
  * form only; rows 0..n-2 Reduce-Scatter, n-1..2n-3 AllGather, both counted forwards).
- * `algo | TRV_ALGO_MIRRORED` (rings, not Trivance): the collective runs a second time with every
+ * `algo | TRV_ALGO_MIRRORED` (not Trivance): the collective runs a second time with every
  * direction reversed, the two sharing the vector half and half (the mirrored sub-collective by
- * which these one-port schedules use both ports, Sec. 2.4); the plan then has two collectives
- * (trv_plan_slices), the second one with negated distances.
+ * which these one-port schedules use both ports, Sec. 2.4); the plan then has twice the collectives
+ * (trv_plan_slices), the second half with negated distances.
+ * Recursive Doubling and Swing also take tori with power-of-two sides (Sec. 2.4; Table 2, App. B): one
+ * collective per dimension, visiting the dimensions in round-robin order like Trivance, 2 D collectives when
+ * mirrored.  `algo | TRV_ALGO_SINGLE` (these two, not mirrored): ONE collective on the whole vector that walks
+ * through the dimensions in turn, which is how their latency-optimal forms use a torus (App. B: "only a
+ * single port per node").  Bruck takes power-of-three tori, Bucket rings only.
  * Comparator plans serve trv_link_loads, trv_cost_model and the schedule queries, and they are executable:
  * trv_allreduce / trv_allreduce_ex (TRV_KERNEL_AUTO or TRV_KERNEL_STEP) run them step by step, literally -- at
  * the start of a step every rank's vector is copied to a wire buffer (scratch of n * round_up(count, 64) * 4

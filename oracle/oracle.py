@@ -18,7 +18,8 @@ _lock = threading.Lock()
 _lib = None
 
 ALGO_TRIVANCE, ALGO_BRUCK, ALGO_RECDOUB, ALGO_SWING, ALGO_BUCKET = 0, 1, 2, 3, 4
-ALGO_MIRROR = 16     # flag: add the mirrored sub-collective on the other half of the vector (rings, comparators)
+ALGO_MIRROR = 16     # flag: add the mirrored sub-collective on the other half of the vector (comparators)
+ALGO_SINGLE = 32     # flag: Recursive Doubling / Swing on a torus as ONE collective walking through the dimensions
 VARIANT_LATENCY, VARIANT_BANDWIDTH = 0, 1
 _DTYPES = {np.dtype(np.int32): 0, np.dtype(np.uint32): 0, np.dtype(np.float32): 1, np.dtype(np.float64): 2}
 _ERR = {1: "bad argument", 2: "schedule undefined for these dimensions", 3: "out of memory", 4: "internal check failed"}

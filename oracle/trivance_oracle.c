@@ -63,7 +63,7 @@
 #define ORC_MAX_DIMS 8
 
 enum { ORC_OK = 0, ORC_BAD_ARG = 1, ORC_UNDEFINED = 2, ORC_NOMEM = 3, ORC_INTERNAL = 4 };
-enum { ORC_TRIVANCE = 0, ORC_BRUCK = 1, ORC_RECDOUB = 2, ORC_SWING = 3, ORC_BUCKET = 4, ORC_MIRROR = 16 };
+enum { ORC_TRIVANCE = 0, ORC_BRUCK = 1, ORC_RECDOUB = 2, ORC_SWING = 3, ORC_BUCKET = 4, ORC_MIRROR = 16, ORC_SINGLE = 32 };
 enum { ORC_LATENCY = 0, ORC_BANDWIDTH = 1 };
 enum { ORC_I32 = 0, ORC_F32 = 1, ORC_F64 = 2 };
 
@@ -88,13 +88,19 @@ static int ilog_exact(int a, int base) {       /* log_base a, or -1 if a is no p
  * "mirrored sub-collective" by which the one-port comparators use both ports (Sec. 2.4). */
 static int topo_init(orc_topo *tp, const int32_t *dims, int ndims, int algo) {
     if (!dims || ndims < 1 || ndims > ORC_MAX_DIMS) return ORC_BAD_ARG;
-    int mirror = (algo & ORC_MIRROR) ? 1 : 0;
-    algo &= ~ORC_MIRROR;
+    int mirror = (algo & ORC_MIRROR) ? 1 : 0, single = (algo & ORC_SINGLE) ? 1 : 0;
+    algo &= ~(ORC_MIRROR | ORC_SINGLE);
     if (algo < ORC_TRIVANCE || algo > ORC_BUCKET) return ORC_BAD_ARG;
-    if (mirror && (algo == ORC_TRIVANCE || ndims != 1)) return ORC_BAD_ARG;
-    tp->algo = algo; tp->ndims = ndims; tp->nsl = ndims * (mirror ? 2 : 1);
+    if (mirror && algo == ORC_TRIVANCE) return ORC_BAD_ARG;
+    if (mirror && ndims != 1 && algo != ORC_RECDOUB && algo != ORC_SWING) return ORC_BAD_ARG;
+    /* ORC_SINGLE: ONE collective on the whole vector that walks through the dimensions in turn -- how the
+     * latency-optimal Recursive Doubling and Swing use a torus ("only a single port per node", App. B) */
+    if (single && (mirror || (algo != ORC_RECDOUB && algo != ORC_SWING))) return ORC_BAD_ARG;
+    tp->algo = algo; tp->ndims = ndims; tp->nsl = single ? 1 : ndims * (mirror ? 2 : 1);
     tp->base = (algo == ORC_RECDOUB || algo == ORC_SWING) ? 2 : 3;
-    if ((algo == ORC_RECDOUB || algo == ORC_SWING || algo == ORC_BUCKET) && ndims != 1) return ORC_UNDEFINED;
+    /* Recursive Doubling and Swing on tori (Sec. 2.4): one collective per dimension, each with its mirrored
+     * sub-collective when asked for (2D collectives on 1/(2D) of the vector each); Bucket: rings only here. */
+    if (algo == ORC_BUCKET && ndims != 1) return ORC_UNDEFINED;
     if (algo == ORC_BUCKET) {           /* ring algorithm: any n >= 2, n - 1 steps per phase (Sec. 2.4) */
         if (dims[0] < 2 || dims[0] > 4096) return ORC_BAD_ARG;
         tp->dims[0] = dims[0]; tp->stride[0] = 1; tp->sdim[0] = dims[0] - 1;

@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libtrivance.so")
 LATENCY_OPTIMAL, BANDWIDTH_OPTIMAL = 0, 1
 ALGO_TRIVANCE, ALGO_BRUCK, ALGO_RECDOUB, ALGO_SWING, ALGO_BUCKET = 0, 1, 2, 3, 4
 ALGO_MIRRORED = 16
+ALGO_SINGLE = 32
 INT32, FLOAT32 = 0, 1
 SUM = 0
 KERNEL_AUTO, KERNEL_STEP, KERNEL_FUSED, KERNEL_PIPELINED = 0, 1, 2, 3

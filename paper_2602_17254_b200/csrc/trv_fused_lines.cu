@@ -182,16 +182,26 @@ static trv_status_t launch_lines_cg(const Call& c, const Addr& in, const Addr& o
 // ------------------------------------------------------------------ host side
 
 #if TRV_LN_PART == 0
+static bool build_program(const Plan& p, LnProgram* prog);
+
 bool fused_lines_supported(const Plan& p) {
-    if (p.algo != TRV_ALGO_TRIVANCE || p.variant != TRV_LATENCY_OPTIMAL) return false;
+    if (p.general || p.algo != TRV_ALGO_TRIVANCE || p.variant != TRV_LATENCY_OPTIMAL) return false;
     if (p.n > 729 || p.ndims > kLnMaxD) return false;
     for (int d = 0; d < p.ndims; ++d)
         if (p.dims[d] > 81) return false;
-    return true;
+    static thread_local LnProgram probe;        // every group of the plan must be one the kernel carries
+    return build_program(p, &probe);
 }
 
+// The (kind, shape) pairs the kernel's dispatch switches carry; build_program refuses anything else, so a shape that
+// a raised limit would let through can never fall through a switch unnoticed.
 static bool plane_ok(int la, int lb) {
     return (la == 3 && (lb == 3 || lb == 9 || lb == 27)) || (la == 9 && (lb == 3 || lb == 9)) || (la == 27 && lb == 3);
+}
+static bool line_ok(int la, int nsteps) {
+    int s = 0;
+    for (int v = la; v > 1; v /= 3) { if (v % 3) return false; ++s; }
+    return (la == 3 || la == 9 || la == 27 || la == 81) && nsteps >= 1 && nsteps <= s;
 }
 
 // base ranks of the sets {r0 + da*sa*i + db*sb*j}: all ranks whose coordinate along the set's
@@ -232,6 +242,7 @@ static bool build_program(const Plan& p, LnProgram* prog) {
                     continue;
                 }
             }
+            if (!line_ok(la, k)) return false;
             g.kind = LN_LINE; g.la = (short)la; g.lb = 1; g.nsteps = (short)k;
             g.stride_a = xa * p.stride[da]; g.stride_b = 0;
             g.base_off = nb;

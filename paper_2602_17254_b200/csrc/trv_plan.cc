@@ -133,22 +133,23 @@ static void build_reach(Plan& p) {
 trv_status_t build_plan(const int32_t* dims, int32_t ndims, int variant, int algo_flags, trv_plan_s** out) {
     if (!dims || !out || ndims < 1 || ndims > TRV_MAX_DIMS) return TRV_ERR_INVALID_ARG;
     if (variant != TRV_LATENCY_OPTIMAL && variant != TRV_BANDWIDTH_OPTIMAL) return TRV_ERR_INVALID_ARG;
-    const bool mirror = (algo_flags & TRV_ALGO_MIRRORED) != 0;
-    const int algo = algo_flags & ~TRV_ALGO_MIRRORED;
+    const bool mirror = (algo_flags & TRV_ALGO_MIRRORED) != 0, single = (algo_flags & TRV_ALGO_SINGLE) != 0;
+    const int algo = algo_flags & ~(TRV_ALGO_MIRRORED | TRV_ALGO_SINGLE);
     if (algo < TRV_ALGO_TRIVANCE || algo > TRV_ALGO_BUCKET) return TRV_ERR_INVALID_ARG;
-    if (mirror && (algo == TRV_ALGO_TRIVANCE || ndims != 1)) return TRV_ERR_INVALID_ARG;
+    const bool binary = algo == TRV_ALGO_RECDOUB || algo == TRV_ALGO_SWING;
+    if (mirror && (algo == TRV_ALGO_TRIVANCE || (ndims != 1 && !binary))) return TRV_ERR_INVALID_ARG;
+    if (single && (mirror || !binary)) return TRV_ERR_INVALID_ARG;
     for (int d = 0; d < ndims; ++d)
         if (dims[d] < 2) return TRV_ERR_INVALID_ARG;
-    const bool binary = algo == TRV_ALGO_RECDOUB || algo == TRV_ALGO_SWING;
     const int base = binary ? 2 : 3;
-    if ((binary || algo == TRV_ALGO_BUCKET) && ndims != 1) return TRV_ERR_UNSUPPORTED;
+    if (algo == TRV_ALGO_BUCKET && ndims != 1) return TRV_ERR_UNSUPPORTED;
     if (algo == TRV_ALGO_BUCKET && (variant != TRV_BANDWIDTH_OPTIMAL || dims[0] > TRV_MAX_RANKS)) return TRV_ERR_UNSUPPORTED;
 
     trv_plan_s* holder = new (std::nothrow) trv_plan_s();
     if (!holder) return TRV_ERR_ALLOC;
     Plan& p = holder->plan;
     p.algo = algo; p.variant = variant; p.ndims = ndims; p.base = base;
-    p.nslices = ndims * (mirror ? 2 : 1);
+    p.nslices = single ? 1 : ndims * (mirror ? 2 : 1);
     if (algo == TRV_ALGO_BUCKET) {
         // ring algorithm (Sec. 2.4): n - 1 steps per phase, every step one block to the next node
         p.dims[0] = dims[0]; p.stride[0] = 1; p.n = dims[0]; p.S = dims[0] - 1;
@@ -219,9 +220,13 @@ bool in_send_set(const Plan& p, int c, int t, int dst, int j) {
         const int sg = p.steps[c][t].dist, src = ((dst - sg) % p.n + p.n) % p.n;
         return j == ((src - sg * (t + 1)) % p.n + p.n) % p.n;
     }
-    if (p.algo == TRV_ALGO_RECDOUB && c >= p.ndims) {     // the mirrored collective is the same pattern on the ring read backwards
-        const int n = p.n;
-        return in_send_set(p, c - p.ndims, t, (n - dst) % n, (n - j) % n);
+    if (p.algo == TRV_ALGO_RECDOUB && c >= p.ndims) {     // the mirrored collective is the same pattern on the rings read backwards
+        int nd = 0, nj = 0;                               // every coordinate x -> (side - x) mod side
+        for (int d = 0; d < p.ndims; ++d) {
+            nd += ((p.dims[d] - p.coord(dst, d)) % p.dims[d]) * p.stride[d];
+            nj += ((p.dims[d] - p.coord(j, d)) % p.dims[d]) * p.stride[d];
+        }
+        return in_send_set(p, c - p.ndims, t, nd, nj);
     }
     for (int d = 0; d < p.ndims; ++d) {
         int m = p.mod[c][t][d];

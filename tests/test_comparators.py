@@ -247,3 +247,74 @@ def test_bandwidth_forms_all_rows_equal_and_blocks_are_the_owners_latency_rows(a
             assert np.array_equal(bw[j, bb[j]:bb[j + 1]].view(np.uint32), lat[j, bb[j]:bb[j + 1]].view(np.uint32))
     xi = rng.integers(-100, 100, size=(n, E)).astype(np.float32)      # small integers: exact, equals the int path
     assert np.array_equal(oracle.allreduce_algo((n,), 1, xi, algo), oracle.allreduce_algo((n,), 1, xi.astype(np.int32), algo).astype(np.float32))
+
+
+# ------------------------------------------------------------------ Table 2 / App. B: Recursive Doubling and Swing on tori
+
+def _rho_abs(k):
+    return abs(sum((-2) ** i for i in range(k + 1)))
+
+
+POW2_TORI = [(4, 4), (8, 8), (16, 16), (4, 4, 4), (8, 8, 8), (4, 4, 4, 4)]
+
+
+@pytest.mark.parametrize("dims", POW2_TORI)
+def test_table2_swing_and_recursive_doubling_bandwidth_forms_on_tori(dims):
+    """App. B: Theta of the bandwidth-optimal forms on a D-dimensional torus, relative to m beta / D, is
+    sum_d sum_k c_k / 2^(1 + d + D k) with c_k = |rho(k)| (Swing, with its mirrored sub-collectives) resp. 2^k
+    (Recursive Doubling).  The tally of Swing's 2 D superposed collectives gives that number exactly.  For Recursive
+    Doubling the appendix counts ONE collective's congestion with the half-size messages of the mirrored set-up (as on
+    rings): that is half the tally of the D unmirrored collectives; the mirrored tally lies between the two."""
+    D, a = len(dims), dims[0]
+    q = a.bit_length() - 1
+    n = a ** D
+    E = n * 2 * D * 4
+    swing = sum(_rho_abs(k) / 2 ** (1 + d + D * k) for d in range(D) for k in range(q))
+    rd = sum(2 ** k / 2 ** (1 + d + D * k) for d in range(D) for k in range(q))
+    c = oracle.cost_model(dims, 1, E, 4, 0.0, 1.0, oracle.ALGO_SWING | oracle.ALGO_MIRROR)
+    assert c["theta"] == pytest.approx(swing, rel=1e-12) and c["steps"] == 2 * D * q and c["delta"] == pytest.approx(1 - 1 / n)
+    c = oracle.cost_model(dims, 1, E, 4, 0.0, 1.0, oracle.ALGO_RECDOUB)
+    assert c["theta"] == pytest.approx(2 * rd, rel=1e-12)
+    m = oracle.cost_model(dims, 1, E, 4, 0.0, 1.0, oracle.ALGO_RECDOUB | oracle.ALGO_MIRROR)
+    assert rd <= m["theta"] <= 2 * rd and m["delta"] == pytest.approx(1 - 1 / n)
+
+
+@pytest.mark.parametrize("dims", POW2_TORI)
+def test_table2_latency_forms_use_a_single_collective(dims):
+    """App. B: the latency-optimal Recursive Doubling and Swing run ONE collective on the whole vector ("only a single port
+    per node"); per dimension the congestions 2^k resp. ceil(|rho(k)| / 2) add up, times D dimensions, times D again
+    relative to m beta / D: D^2 (a - 1) and D^2 sum_k ceil(|rho(k)| / 2) (Table 2: D^2 n^(1/D) and D^2 / 3 n^(1/D))."""
+    D, a = len(dims), dims[0]
+    q = a.bit_length() - 1
+    E = 1024
+    c = oracle.cost_model(dims, 0, E, 4, 0.0, 1.0, oracle.ALGO_RECDOUB | oracle.ALGO_SINGLE)
+    assert c["steps"] == D * q and c["theta"] == pytest.approx(D * D * (a - 1))
+    c = oracle.cost_model(dims, 0, E, 4, 0.0, 1.0, oracle.ALGO_SWING | oracle.ALGO_SINGLE)
+    assert c["theta"] == pytest.approx(D * D * sum(-(-_rho_abs(k) // 2) for k in range(q)))
+    x = np.random.default_rng(a).integers(-1000, 1000, size=(a ** D, 40), dtype=np.int32)
+    for algo in (oracle.ALGO_RECDOUB, oracle.ALGO_SWING):
+        assert (oracle.allreduce_algo(dims, 0, x, algo | oracle.ALGO_SINGLE) == x.sum(0, dtype=np.int32)[None]).all()
+
+
+def test_appendix_b_sums_tend_to_table2_closed_forms():
+    """The sums of App. B converge to Table 2's closed forms: Swing (B) 2^D (2^D - 1) / ((2^D - 2)(2^D + 1)) = 1.2, 1.04, 1.01;
+    Recursive Doubling (B) (2^D - 1) / (2^D - 2) = 1.5, 1.17, 1.07 for D = 2, 3, 4 (arithmetic on the paper's formulas only)."""
+    for D, sw, rd in ((2, 1.2, 1.5), (3, 1.04, 1.17), (4, 1.01, 1.07)):
+        q = 40
+        s = sum(_rho_abs(k) / 2 ** (1 + d + D * k) for d in range(D) for k in range(q))
+        r = sum(2 ** k / 2 ** (1 + d + D * k) for d in range(D) for k in range(q))
+        assert s == pytest.approx(2 ** D * (2 ** D - 1) / ((2 ** D - 2) * (2 ** D + 1)), rel=1e-9) and round(s, 2) == sw
+        assert r == pytest.approx((2 ** D - 1) / (2 ** D - 2), rel=1e-9) and round(r, 2) == rd
+
+
+@pytest.mark.parametrize("algo", [oracle.ALGO_RECDOUB, oracle.ALGO_SWING])
+@pytest.mark.parametrize("dims", [(4, 4), (2, 8), (4, 4, 4)])
+def test_torus_comparator_paths_give_the_column_sums(algo, dims):
+    n = int(np.prod(dims))
+    for variant in (0, 1):
+        for flag in (0, oracle.ALGO_MIRROR):
+            E = 5 * n + 3
+            x = np.random.default_rng(n).integers(-2 ** 31, 2 ** 31 - 1, size=(n, E), dtype=np.int64).astype(np.int32)
+            y, ctr = oracle.allreduce_algo(dims, variant, x, algo | flag, counters=True)
+            assert (y == x.astype(np.int64).sum(0).astype(np.int32)[None]).all()
+            assert np.array_equal(ctr["sent_rs"] + ctr["sent_ag"], oracle.bytes_sent(dims, variant, E, 4, algo | flag))

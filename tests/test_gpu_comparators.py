@@ -85,6 +85,29 @@ def test_windows_short_vectors_and_the_in_place_call(algo, dims):
         _run(algo, dims, variant, 4100, "normal", 75, via_allreduce=True)
 
 
+TORUS_CASES = [(binding.ALGO_RECDOUB, (4, 4)), (binding.ALGO_RECDOUB, (2, 8)), (binding.ALGO_SWING, (8, 8)), (binding.ALGO_SWING, (4, 4, 4)),
+               (binding.ALGO_RECDOUB, (4, 4, 4))]
+
+
+@pytest.mark.parametrize("algo,dims", TORUS_CASES)
+@pytest.mark.parametrize("flag", [0, binding.ALGO_MIRRORED, binding.ALGO_SINGLE])
+def test_recursive_doubling_and_swing_on_tori(algo, dims, flag):
+    """Sec. 2.4, Table 2: one collective per dimension, 2 D when mirrored, or a single one walking through the dimensions:
+    data paths bit-exact against the oracle, link loads and cost model equal to its hop-by-hop tally."""
+    for variant in (LAT, BW):
+        _run(algo | flag, dims, variant, 3001, "normal", 81)
+        _run(algo | flag, dims, variant, 1025, "int32", 82, in_place=False)
+        plan = binding.Plan(dims, variant, algo | flag)
+        got = plan.link_loads(100003, 4)
+        want = oracle.link_loads(dims, variant, 100003, 4, algo=algo | flag)
+        for k in ("msgs", "bytes", "max_msgs", "max_bytes"):
+            assert got[k].dtype == want[k].dtype and np.array_equal(got[k], want[k]), k
+        c, w = plan.cost_model(100003, 4, 1.5e-6, 1e-11), oracle.cost_model(dims, variant, 100003, 4, 1.5e-6, 1e-11, algo | flag)
+        assert c.steps == w["steps"] and c.tx_bytes == w["tx_bytes"] and c.bytes_sent_per_node == w["bytes_sent_per_node"]
+        assert np.isclose(c.theta, w["theta"], rtol=1e-12) and np.isclose(c.delta, w["delta"], rtol=1e-12)
+        plan.destroy()
+
+
 def test_what_the_comparators_do_not_serve():
     plan = binding.Plan((16,), LAT, binding.ALGO_SWING)
     assert plan.kernel_supported(binding.KERNEL_AUTO) and plan.kernel_supported(binding.KERNEL_STEP)
