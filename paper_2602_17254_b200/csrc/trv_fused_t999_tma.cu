@@ -12,6 +12,10 @@
 // no arithmetic at all takes 8.16 ms with two 93 KB tiles per SM: that, not the adds, bounds this design.  Two columns
 // per thread with packed adds and half the instructions: 9.35 ms.  Tiles of 64 columns, one persistent CTA per SM:
 // 9.9 ms.  L2 prefetch of 1 KB-wide boxes ahead of the tiles, clusters of 2 to 8 adjacent tiles: no gain or worse.
+// The plane-wise kernel made persistent, a tenth warp storing each finished phase and refilling its three planes with
+// the NEXT tile at once (so that a CTA's copies in flight never drop to nothing between tiles): 11.6 ms -- the copy
+// thread's wait for the engine to have read a phase before it may refill it serialises what two independent CTAs
+// overlap by themselves.
 // Every wait on a copy's mbarrier is bounded; a waiter that gives up counts it in a device-side counter (trv_tma.cuh)
 // and the CTA leaves without storing.
 #include "trv_dev.cuh"
