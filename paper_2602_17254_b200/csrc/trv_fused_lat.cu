@@ -82,15 +82,16 @@ __device__ __forceinline__ void ring_tail_steps(E (&v)[N]) {     // distances 1,
     }
 }
 
-// 32-column tiles; a thread owns V adjacent columns of one of 9 rank sets: 9 * 32 / V threads.
-template <typename T, int M, int V, bool FULL, typename Addr>
+// Tiles of TILE columns (32, or 64 for long vectors on the ring of 243); a thread owns V adjacent columns of one of 9
+// rank sets: 9 * TILE / V threads.
+template <typename T, int M, int V, int TILE, bool FULL, typename Addr>
 __device__ __forceinline__ void lat_ring_body(const Addr& in, const Addr& out, const LatArgs& a, T* slab, long long t0) {
-    constexpr int NR = 9 * M, LANES = 32 / V;
+    constexpr int NR = 9 * M, LANES = TILE / V;
     using E = Elem<T, V>;
     const int lane = threadIdx.x % LANES, set = threadIdx.x / LANES;
     const long long lo = a.lo[0], hi = a.hi[0];
     const long long e = t0 + lane * V;
-    auto sl = [&](int r) -> E& { return *reinterpret_cast<E*>(slab + r * 32 + lane * V); };
+    auto sl = [&](int r) -> E& { return *reinterpret_cast<E*>(slab + r * TILE + lane * V); };
 
     // group 1: window of M consecutive ranks [set*M, set*M + M) plus a halo of 4 on each side
     E x[M + 8];
@@ -125,15 +126,15 @@ __device__ __forceinline__ void lat_ring_body(const Addr& in, const Addr& out, c
     }
 }
 
-template <typename T, int M, int V, typename Addr>
-__global__ void __launch_bounds__(288 / V) k_lat_ring(Addr in, Addr out, LatArgs a) {
+template <typename T, int M, int V, int TILE, typename Addr>
+__global__ void __launch_bounds__(9 * TILE / V, M == 27 ? (TILE == 64 ? 3 : 4) : 1) k_lat_ring(Addr in, Addr out, LatArgs a) {
     pdl_trigger();
     extern __shared__ uint4 slab_raw[];
-    T* slab = reinterpret_cast<T*>(slab_raw);       // [9 M][32]
-    const long long t0 = (a.lo[0] & ~31LL) + (long long)blockIdx.x * 32;
+    T* slab = reinterpret_cast<T*>(slab_raw);       // [9 M][TILE]
+    const long long t0 = (a.lo[0] & ~(long long)(TILE - 1)) + (long long)blockIdx.x * TILE;
     pdl_wait();
-    if (t0 >= a.lo[0] && t0 + 32 <= a.hi[0]) lat_ring_body<T, M, V, true>(in, out, a, slab, t0);   // CTA-uniform
-    else lat_ring_body<T, M, V, false>(in, out, a, slab, t0);
+    if (t0 >= a.lo[0] && t0 + TILE <= a.hi[0]) lat_ring_body<T, M, V, TILE, true>(in, out, a, slab, t0);   // CTA-uniform
+    else lat_ring_body<T, M, V, TILE, false>(in, out, a, slab, t0);
 }
 
 // ------------------------------------------------------------------ host side
@@ -197,21 +198,35 @@ static trv_status_t lat_fused_launch(const Call& c, const Addr& in, const Addr& 
         else if (A == 3 && D == 4) { g_last_kernel = "lat_reg<3x3x3x3>"; launch_reg<T, 3, 4, 2, 64>(c, in, out, a); }
         else return TRV_ERR_UNSUPPORTED;
     } else if (kind == LatKind::Ring) {
-        const long long tiles = tiles_for(a, 1, 32, 32);
-        if (tiles > 0) {
-            if (p.n == 243) {
-                g_last_kernel = "lat_ring<243>";
-                launch_pdl(k_lat_ring<T, 27, 2, Addr>, dim3((unsigned)tiles), dim3(144), 243 * 32 * 4, c.st, in, out, a);
-            } else {
-                g_last_kernel = "lat_ring<729>";
-                auto kfn = k_lat_ring<T, 81, 1, Addr>;
-                if (!allow_big_smem(kfn, 729 * 32 * 4)) return TRV_ERR_CUDA;
-                launch_pdl(kfn, dim3((unsigned)tiles), dim3(288), 729 * 32 * 4, c.st, in, out, a);
+        // Ring of 243, long vectors: tiles of 64 columns (256 bytes per rank and tile), three CTAs per SM (72 registers).
+        // Every tile touches all 243 input and all 243 output rows, and the 32-column kernel loses bandwidth as the rows
+        // get longer (0.93 of the copy bandwidth at 2 MiB per rank, 0.85 at 8 MiB, 0.83 at 32 MiB) while the 64-column
+        // one holds 0.93 - 0.94 (8 MiB: 730 -> 664 us, 32 MiB: 3013 -> 2648 us).  Up to 2 MiB per rank the two are
+        // within a percent of each other; the 32-column kernel (four CTAs per SM, 96 registers) keeps the short vectors.
+        if (p.n == 243 && a.hi[0] - a.lo[0] >= (1LL << 20)) {
+            const long long tiles = tiles_for(a, 1, 64, 64);
+            g_last_kernel = "lat_ring<243,64>";
+            auto kfn = k_lat_ring<T, 27, 2, 64, Addr>;
+            if (!allow_big_smem(kfn, 243 * 64 * 4)) return TRV_ERR_CUDA;
+            launch_pdl(kfn, dim3((unsigned)tiles), dim3(288), 243 * 64 * 4, c.st, in, out, a);
+        } else {
+            const long long tiles = tiles_for(a, 1, 32, 32);
+            if (tiles > 0) {
+                if (p.n == 243) {
+                    g_last_kernel = "lat_ring<243>";
+                    launch_pdl(k_lat_ring<T, 27, 2, 32, Addr>, dim3((unsigned)tiles), dim3(144), 243 * 32 * 4, c.st, in, out, a);
+                } else {
+                    g_last_kernel = "lat_ring<729>";
+                    auto kfn = k_lat_ring<T, 81, 1, 32, Addr>;
+                    if (!allow_big_smem(kfn, 729 * 32 * 4)) return TRV_ERR_CUDA;
+                    launch_pdl(kfn, dim3((unsigned)tiles), dim3(288), 729 * 32 * 4, c.st, in, out, a);
+                }
             }
         }
     } else if (kind == LatKind::T999) {
         // equally spaced rank buffers: the tile arrives by TMA; else per-thread loads
         trv_status_t st = TRV_OK;
+        if (run_fused_t999_wide(c, a, &st)) return st;
         if (run_fused_t999_tma(c, a, &st)) return st;
         g_last_kernel = "lat_t999";
         return run_fused_t999(c, a);

@@ -1,7 +1,8 @@
 // FUSED latency-optimal kernels for the 9 x 9 x 9 torus (Sec. 4.2, Sec. 5) whose tile moves by TMA.
 //
 // Same three closed groups as k_lat_t999 (trv_fused_t999.cu); both kernels need equally spaced rank buffers (tensor
-// maps describe them as a matrix); other callers keep k_lat_t999.
+// maps describe them as a matrix); other callers keep k_lat_t999.  Vectors from about 3 MiB per rank go to the
+// persistent kernel on 64-column tiles (trv_fused_t999_wide.cu) instead.
 //   k_lat_t999_planes : the 32-column x 729-rank tile arrives as nine bulk tensor copies, one C-plane each, on nine
 //                       mbarriers, so group 1 starts plane by plane; the results leave through bulk tensor stores,
 //                       three planes after each phase of group 3.  729 x 32 MiB: 9.07 ms in a 0.7 s timed region under
@@ -10,8 +11,9 @@
 //                       kept for the case that the four-dimensional tensor maps cannot be encoded.
 // Measured on the way (same workload, 0.7 s regions): the copy engine moving the tile in and straight out again with
 // no arithmetic at all takes 8.16 ms with two 93 KB tiles per SM: that, not the adds, bounds this design.  Two columns
-// per thread with packed adds and half the instructions: 9.35 ms.  Tiles of 64 columns, one persistent CTA per SM:
-// 9.9 ms.  L2 prefetch of 1 KB-wide boxes ahead of the tiles, clusters of 2 to 8 adjacent tiles: no gain or worse.
+// per thread with packed adds and half the instructions: 9.35 ms.  Tiles of 64 columns, one persistent CTA per SM,
+// with no overlap between a tile's arithmetic and the next tile's copies: 9.9 ms (with that overlap: the wide kernel).
+// L2 prefetch of 1 KB-wide boxes ahead of the tiles, clusters of 2 to 8 adjacent tiles: no gain or worse.
 // The plane-wise kernel made persistent, a tenth warp storing each finished phase and refilling its three planes with
 // the NEXT tile at once (so that a CTA's copies in flight never drop to nothing between tiles): 11.6 ms -- the copy
 // thread's wait for the engine to have read a phase before it may refill it serialises what two independent CTAs
@@ -235,10 +237,6 @@ __device__ __forceinline__ void t999_planes_body(const CUtensorMap* omap, const 
     }
 }
 
-struct PlaneMaps {
-    CUtensorMap in[3], out[3];      // one pair per slice: dimensions ordered by increasing rank stride
-};
-
 template <typename T>
 __global__ void __launch_bounds__(288, 2) k_lat_t999_planes(const __grid_constant__ PlaneMaps maps, StrideAddr out, LatArgs a,
                                                             unsigned* giveups) {
@@ -310,9 +308,9 @@ bool tma_encode_ranks(const StrideAddr& in, int n, size_t count, int box_rows, C
 }
 
 // Tensor map of one slice of the 9 x 9 x 9 torus over equally spaced rank buffers: dimensions (column, then the three
-// torus dimensions ordered by increasing rank stride), boxes of 32 columns x one C-plane.  strides[k] = rank stride of
-// the slice's k-th dimension (A, B, C).
-static bool encode_planes(const StrideAddr& base, size_t count, const int strides[3], CUtensorMap* out) {
+// torus dimensions ordered by increasing rank stride), boxes of box_cols columns x one C-plane.  strides[k] = rank
+// stride of the slice's k-th dimension (A, B, C).
+bool encode_planes(const StrideAddr& base, size_t count, const int strides[3], int box_cols, CUtensorMap* out) {
     if ((base.stride & 15) || ((uintptr_t)base.base & 15) || count == 0 || count >= ((size_t)1 << 31)) return false;
     if ((size_t)base.stride < count * 4) return false;
     EncodeTiledFn enc = encode_tiled_fn();
@@ -323,14 +321,15 @@ static bool encode_planes(const StrideAddr& base, size_t count, const int stride
             if (strides[order[j]] < strides[order[i]]) { const int t = order[i]; order[i] = order[j]; order[j] = t; }
     cuuint64_t gdim[4] = {(cuuint64_t)count, 9, 9, 9};
     cuuint64_t gstride[3];
-    cuuint32_t box[4] = {32, 9, 9, 9};
+    cuuint32_t box[4] = {(cuuint32_t)box_cols, 9, 9, 9};
     const cuuint32_t estride[4] = {1, 1, 1, 1};
     for (int i = 0; i < 3; ++i) {
         gstride[i] = (cuuint64_t)strides[order[i]] * base.stride;
         if (order[i] == 2) box[1 + i] = 1;          // one C-plane per box
     }
     return enc(out, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, base.base, gdim, gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
-               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+               CU_TENSOR_MAP_SWIZZLE_NONE, box_cols >= 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // false: this call cannot use the TMA kernels (the caller falls back to k_lat_t999)
@@ -349,7 +348,7 @@ bool run_fused_t999_tma(const Call& c, const LatArgs& a, trv_status_t* status) {
     PlaneMaps maps;
     bool planes = true;             // needs six four-dimensional tensor maps; else the whole-tile kernel below
     for (int sl = 0; sl < 3 && planes; ++sl)
-        planes = encode_planes(sin, c.count, a.rs[sl], &maps.in[sl]) && encode_planes(sout, c.count, a.rs[sl], &maps.out[sl]);
+        planes = encode_planes(sin, c.count, a.rs[sl], 32, &maps.in[sl]) && encode_planes(sout, c.count, a.rs[sl], 32, &maps.out[sl]);
     if (planes) {
         *status = TRV_OK;
         if (tiles_x == 0) return true;

@@ -1,0 +1,239 @@
+// FUSED latency-optimal kernel for the 9 x 9 x 9 torus (Sec. 4.2, Sec. 5) on tiles of 64 element columns.
+//
+// Why 64 columns: every tile touches all 729 input rows and all 729 output rows.  A plain copy that moves 128 bytes
+// per row visit (32 columns) stops at 0.89 - 0.90 of the copy bandwidth on this part however many CTAs are resident,
+// one that moves 256 bytes per visit reaches all of it; the 32-column kernels (trv_fused_t999_tma.cu) sit at that
+// lower ceiling.  A 64-column tile of 729 ranks is 182 KB, so only one fits an SM, and the overlap that two resident
+// CTAs gave for free has to come from inside one persistent CTA:
+//   * a thread owns two adjacent columns (packed adds), a warp one row of 256 bytes;
+//   * the tile arrives as nine plane copies of the copy engine on nine mbarriers (group 1 starts plane by plane);
+//   * group 3 runs in three phases; a phase first pulls its three planes into registers, and as soon as every thread
+//     has done so the copy engine refills those planes with the NEXT tile -- the slab never waits for the stores;
+//   * the results go to HBM from registers (one 256-byte run per warp and rank) and drain while the next tile's
+//     group 1 and 2 run.
+// So loads are in flight during group 3 and the wait for the first planes, stores during groups 1 and 2.
+// 729 x 32 MiB: 8.5 ms in a 0.6 s timed region under the power cap (1.7 GHz), against 9.05 ms for the 32-column kernel.
+// Measured on the way and dropped: all of group 3's 81 values in registers before a single refill of nine planes
+// (spills at 168 registers, 8.56 ms); eleven plane slots with the planes 2 and 5 of the tile after the next loading
+// early (8.75 ms: the run-time slot arithmetic costs more than the two planes' head start gains).
+// The same three closed groups as the other 9 x 9 x 9 kernels: (A,1)(B,1) per C-plane, (C,1)(A,3), (B,3)(C,3).
+// Every wait on a copy's mbarrier is bounded; a CTA that gives up counts it (trv_tma.cuh) and leaves without
+// storing the tile it waited for.
+#include "trv_dev.cuh"
+#include "trv_fused_lat.cuh"
+#include "trv_tma.cuh"
+
+namespace trv {
+
+constexpr int kWideCols = 64;
+constexpr unsigned kWidePlaneBytes = 81 * kWideCols * 4;
+constexpr unsigned kWideTileBytes = 9 * kWidePlaneBytes;
+
+struct WideTiles {
+    long long nx[3];        // tiles of each slice
+    long long total;
+};
+
+__device__ __forceinline__ void wide_locate(const WideTiles& w, const LatArgs& a, long long t, int* c, long long* t0) {
+    int s = 0;
+    while (s < 2 && t >= w.nx[s]) { t -= w.nx[s]; ++s; }
+    *c = s;
+    *t0 = (a.lo[s] & ~(long long)(kWideCols - 1)) + t * kWideCols;
+}
+
+__device__ __forceinline__ int wide_cpos(int c) { return c == 0 ? 3 : (c == 1 ? 1 : 2); }   // where C sits in the slice's maps
+
+// one thread: plane k of the tile (c, t0) into its place in the slab, completing on bars[k]
+__device__ __forceinline__ void wide_fetch_plane(const PlaneMaps& maps, int c, long long t0, int k, unsigned slab_s,
+                                                 unsigned long long* bars) {
+    const unsigned bar_s = smem_u32(bars + k);
+    const int cpos = wide_cpos(c);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s), "r"(kWidePlaneBytes) : "memory");
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(
+            slab_s + k * kWidePlaneBytes),
+        "l"(&maps.in[c]), "r"((int)t0), "r"(cpos == 1 ? k : 0), "r"(cpos == 2 ? k : 0), "r"(cpos == 3 ? k : 0), "r"(bar_s)
+        : "memory");
+}
+
+// One tile.  PA = 1: inside a plane the A coordinate runs fastest, PA = 9: B does (see encode_planes).
+// Returns false when a wait ran out (CTA-uniform).
+template <typename T, int PA, bool FULL>
+__device__ __forceinline__ bool wide_tile(const PlaneMaps& maps, const StrideAddr& out, const LatArgs& a, int c, long long t0,
+                                          unsigned parity, bool has_next, int nc, long long nt0, T* slab, unsigned long long* bars,
+                                          int* gave_up) {
+    constexpr int PB = PA == 1 ? 9 : 1, PC = 81;
+    using E = Elem<T, 2>;
+    const int lane = threadIdx.x % 32, set = threadIdx.x / 32;
+    const long long lo = a.lo[c], hi = a.hi[c];
+    const long long e = t0 + 2 * lane;
+    E* const mine = reinterpret_cast<E*>(slab) + lane;
+    auto sl = [&](int r) -> E& { return mine[r * (kWideCols / 2)]; };
+    {   // ---- group 1: (A,1) (B,1) on the plane C = set, as soon as it has arrived
+        unsigned done = 0;
+        const unsigned bar_s = smem_u32(bars + set);
+        for (unsigned spins = 0; spins < kTmaWaitLimit; ++spins) {
+            asm volatile(
+                "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                : "=r"(done)
+                : "r"(bar_s), "r"(parity)
+                : "memory");
+            if (done) break;
+        }
+        if (!done) *gave_up = 1;
+        const int r0 = set * PC;
+        auto load_row = [&](int j, E (&row)[9]) {
+#pragma unroll
+            for (int i = 0; i < 9; ++i) row[i] = sl(r0 + i * PA + j * PB);
+            reg_step<9, 1, 9, 1>(row);                                      // (A,1)
+        };
+        auto emit = [&](int j, const E (&p)[9], const E (&q)[9], const E (&r)[9]) {     // (B,1) for row j
+#pragma unroll
+            for (int i = 0; i < 9; ++i) sl(r0 + i * PA + j * PB) = add3(p[i], q[i], r[i]);
+        };
+        E first[9], second[9], prev[9], cur[9], next[9];
+        load_row(0, first);
+        load_row(1, second);
+#pragma unroll
+        for (int i = 0; i < 9; ++i) { prev[i] = first[i]; cur[i] = second[i]; }
+#pragma unroll
+        for (int j = 1; j < 8; ++j) {
+            load_row(j + 1, next);          // row j + 1 is read before row j is overwritten
+            emit(j, prev, cur, next);
+#pragma unroll
+            for (int i = 0; i < 9; ++i) { prev[i] = cur[i]; cur[i] = next[i]; }
+        }
+        emit(8, prev, cur, first);
+        emit(0, cur, first, second);
+    }
+    __syncthreads();
+    if (*gave_up) return false;
+    // ---- group 2: (C,1) (A,3) on the sets {A in a0 + 3 i, B = j, all C}; flat index k + 9 i
+#pragma unroll
+    for (int m = 0; m < 3; ++m) {
+        const int q = set + 9 * m, r0 = (q % 3) * PA + (q / 3) * PB;
+        E v[27];
+#pragma unroll
+        for (int idx = 0; idx < 27; ++idx) v[idx] = sl(r0 + 3 * (idx / 9) * PA + (idx % 9) * PC);
+        reg_step<27, 1, 9, 1>(v);       // (C,1)
+        reg_step<27, 9, 3, 1>(v);       // (A,3)
+#pragma unroll
+        for (int idx = 0; idx < 27; ++idx) sl(r0 + 3 * (idx / 9) * PA + (idx % 9) * PC) = v[idx];
+    }
+    __syncthreads();
+    // ---- group 3: (B,3) (C,3) on the sets {A = i, B in b0 + 3 jj, C in c0 + 3 kk}, phase by phase in c0
+    const int sA = a.rs[c][0], sB = a.rs[c][1], sC = a.rs[c][2];
+    const unsigned slab_s = smem_u32(slab);
+#pragma unroll 1
+    for (int c0 = 0; c0 < 3; ++c0) {
+        E v[3][9];
+#pragma unroll
+        for (int m = 0; m < 3; ++m) {
+            const int q = set + 9 * m, r0 = (q % 9) * PA + (q / 9) * PB + c0 * PC;
+#pragma unroll
+            for (int idx = 0; idx < 9; ++idx) v[m][idx] = sl(r0 + 3 * (idx % 3) * PB + 3 * (idx / 3) * PC);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // this thread's slab accesses before the engine's writes
+        __syncthreads();                    // everybody holds its part of the planes c0, c0 + 3, c0 + 6: they may be refilled
+        if (threadIdx.x == 0 && has_next) {
+            for (int kk = 0; kk < 3; ++kk) wide_fetch_plane(maps, nc, nt0, c0 + 3 * kk, slab_s, bars);
+        }
+#pragma unroll
+        for (int m = 0; m < 3; ++m) {
+            const int q = set + 9 * m, g0 = (q % 9) * sA + (q / 9) * sB + c0 * sC;
+            reg_step<9, 1, 3, 1>(v[m]);     // (B,3)
+            reg_step<9, 3, 3, 1>(v[m]);     // (C,3)
+            if (FULL || (e < hi && e + 2 > lo)) {
+#pragma unroll
+                for (int idx = 0; idx < 9; ++idx)
+                    store_elem<T, 2, FULL>(out.ptr(g0 + 3 * (idx % 3) * sB + 3 * (idx / 3) * sC), e, lo, hi, v[m][idx]);
+            }
+        }
+    }
+    return true;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(288, 1) k_lat_t999_wide(const __grid_constant__ PlaneMaps maps, StrideAddr out, LatArgs a,
+                                                          WideTiles w, unsigned* giveups) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    T* slab = reinterpret_cast<T*>(smem_raw);                           // [9 planes][81][64]
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_raw + kWideTileBytes);
+    int* gave_up = reinterpret_cast<int*>(bars + 9);
+    long long t = blockIdx.x;                                           // everything below is CTA-uniform
+    if (t >= w.total) return;
+    int c;
+    long long t0;
+    wide_locate(w, a, t, &c, &t0);
+    if (threadIdx.x == 0) {
+        *gave_up = 0;
+        for (int k = 0; k < 9; ++k) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bars + k)), "r"(1) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        for (int k = 0; k < 9; ++k) wide_fetch_plane(maps, c, t0, k, smem_u32(slab), bars);
+    }
+    __syncthreads();                    // the barriers are initialised before anybody polls them
+    for (unsigned parity = 0;; parity ^= 1) {
+        const long long tn = t + gridDim.x;
+        const bool has_next = tn < w.total;
+        int nc = 0;
+        long long nt0 = 0;
+        if (has_next) wide_locate(w, a, tn, &nc, &nt0);
+        const bool full = t0 >= a.lo[c] && t0 + kWideCols <= a.hi[c];
+        bool ok;
+        if (c == 2) {
+            ok = full ? wide_tile<T, 9, true>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up)
+                      : wide_tile<T, 9, false>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up);
+        } else {
+            ok = full ? wide_tile<T, 1, true>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up)
+                      : wide_tile<T, 1, false>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up);
+        }
+        if (!ok) {                      // a wait ran out: counted once, this tile is not stored
+            if (threadIdx.x == 0) atomicAdd(giveups, 1u);
+            return;
+        }
+        if (!has_next) return;
+        t = tn; c = nc; t0 = nt0;
+    }
+}
+
+// false: this call cannot use the wide kernel (the caller goes on to the 32-column kernels)
+bool run_fused_t999_wide(const Call& c, const LatArgs& a, trv_status_t* status) {
+    StrideAddr sin, sout;
+    if (!uniform_stride(c.in, 729, &sin) || !uniform_stride((const void* const*)c.out, 729, &sout)) return false;
+    if ((sout.stride & 7) || ((uintptr_t)sout.base & 7)) return false;      // two-column stores
+    WideTiles w;
+    w.total = 0;
+    long long local = 0;            // elements of this call's window, all slices
+    for (int sl = 0; sl < 3; ++sl) {
+        if (a.hi[sl] > a.lo[sl]) local += a.hi[sl] - a.lo[sl];
+        w.nx[sl] = a.hi[sl] > a.lo[sl] ? (a.hi[sl] - (a.lo[sl] & ~(long long)(kWideCols - 1)) + kWideCols - 1) / kWideCols : 0;
+        w.total += w.nx[sl];
+    }
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+        return false;
+    // From about 3 MiB per rank on: 4 MiB per rank 1155 -> 1084 us, 8 MiB 2314 -> 2156 us, 32 MiB 9.05 -> 8.5 ms; at 2 MiB the
+    // two kernels tie, below it the 32-column kernels win (more, smaller tiles to spread over the SMs).
+    if (local < (3LL << 18) || w.total < 2LL * sms || w.total > (1LL << 30)) return false;     // short vectors: the 32-column kernels have more tiles to spread
+    unsigned* giveups = tma_giveup_counter();
+    if (!giveups) return false;
+    PlaneMaps maps;
+    for (int sl = 0; sl < 3; ++sl)
+        if (!encode_planes(sin, c.count, a.rs[sl], kWideCols, &maps.in[sl])) return false;
+    *status = TRV_OK;
+    constexpr int smem = (int)kWideTileBytes + 9 * 8 + 16;
+    g_last_kernel = "lat_t999_wide";
+    const unsigned grid = (unsigned)(w.total < sms ? w.total : sms);
+    if (c.dtype == TRV_FLOAT32) {
+        if (!allow_big_smem(k_lat_t999_wide<float>, smem)) { *status = TRV_ERR_CUDA; return true; }
+        TRV_LAUNCH((k_lat_t999_wide<float>), dim3(grid), 288, smem, c.st, maps, sout, a, w, giveups);
+    } else {
+        if (!allow_big_smem(k_lat_t999_wide<uint32_t>, smem)) { *status = TRV_ERR_CUDA; return true; }
+        TRV_LAUNCH((k_lat_t999_wide<uint32_t>), dim3(grid), 288, smem, c.st, maps, sout, a, w, giveups);
+    }
+    if (cudaGetLastError() != cudaSuccess) *status = TRV_ERR_CUDA;
+    return true;
+}
+
+}  // namespace trv

@@ -56,6 +56,11 @@ __device__ __forceinline__ bool tma_fetch_tile(const CUtensorMap* tmap, void* sl
 // Host: the tensor map of n equally spaced rank buffers of `count` words, boxes of 32 x box_rows.
 // false: not expressible (spacing no multiple of 16 bytes, buffers overlapping, driver entry missing).
 bool tma_encode_ranks(const StrideAddr& in, int n, size_t count, int box_rows, CUtensorMap* out);
+// Tensor maps of the three slices of a 9 x 9 x 9 torus, one C-plane of box_cols columns per box (trv_fused_t999_tma.cu)
+struct PlaneMaps {
+    CUtensorMap in[3], out[3];      // one pair per slice: dimensions ordered by increasing rank stride
+};
+bool encode_planes(const StrideAddr& base, size_t count, const int strides[3], int box_cols, CUtensorMap* out);
 unsigned* tma_giveup_counter();     // device address of the counter on the current device (NULL on failure)
 unsigned tma_giveups();             // its value (synchronous copy); ~0u on failure
 

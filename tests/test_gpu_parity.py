@@ -74,6 +74,17 @@ def test_fused_latency_9x9x9_many_tiles_per_cta():
     check_scattered((9, 9, 9), LAT, 20011, "normal", 6, FUSED)
 
 
+def test_fused_latency_9x9x9_tiles_of_64_columns():
+    """Long vectors on the 9x9x9 torus take the persistent kernel on 64-column tiles (one CTA per SM, the next tile
+    loading while group 3 of the current one runs from registers): ragged slice edges that share a tile between two
+    slices, several tiles per CTA with both mbarrier parities, both dtypes, in place and not."""
+    check_case((9, 9, 9), LAT, 800003, "normal", 41, FUSED)
+    assert binding.last_kernel_name() == "lat_t999_wide"
+    check_case((9, 9, 9), LAT, 786754, "int32", 42, FUSED, in_place=False)
+    assert binding.last_kernel_name() == "lat_t999_wide"
+    assert binding.tma_giveups() == 0
+
+
 def test_fused_bandwidth_wide_path_on_729_ranks_sampled():
     """9x9x9 with blocks of >= 256 elements: the oracle checks windows around slice and block
     boundaries and in block interiors."""
