@@ -173,7 +173,8 @@ trv_status_t trv_plan_block_bounds(trv_plan_t plan, size_t count, int32_t c, int
  *   cuda_stream : a cudaStream_t (NULL = the legacy default stream)
  * Asynchronous.  For every shape the FUSED family serves (trv_kernel_supported) the call is a pure launch:
  * it allocates nothing, never synchronises and writes nothing into the plan, so any number of threads and
- * streams may use one plan at once.
+ * streams may use one plan at once.  (Host-side, the library remembers which streams it has seen: the 9 x 9 x 9
+ * kernel for long vectors hands out its tiles from a per-stream counter in a fixed device array.)
  * Shapes that fall to the STEP family of the latency form (e.g. a 243 x 3 torus) need ping-pong scratch.  The
  * plan then allocates it with cudaMalloc on first need -- on the device that is current in that call -- keeps it,
  * grows it when a later call needs more (cudaFree + cudaMalloc: this WAITS FOR THE DEVICE) and frees it in

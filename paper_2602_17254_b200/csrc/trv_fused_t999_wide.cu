@@ -19,11 +19,26 @@
 // The same three closed groups as the other 9 x 9 x 9 kernels: (A,1)(B,1) per C-plane, (C,1)(A,3), (B,3)(C,3).
 // Every wait on a copy's mbarrier is bounded; a CTA that gives up counts it (trv_tma.cuh) and leaves without
 // storing the tile it waited for.
+#include <map>
+#include <mutex>
+
 #include "trv_dev.cuh"
 #include "trv_fused_lat.cuh"
 #include "trv_tma.cuh"
 
 namespace trv {
+
+// Tile scheduling.  With a fixed assignment (tile t, t + grid, ...) the slowest SM ends the kernel; handing out tiles from a
+// counter instead is worth half a percent (three alternating runs each: 8.53 - 8.57 -> 8.50 - 8.51 ms).  The counter must belong to one launch at a time, and the call may
+// allocate nothing, so the library keeps a small pool of counters per device and gives every (device, stream) pair its own:
+// launches of one stream run one after the other, and the last CTA of a launch puts the counter back to zero.  Calls
+// on the per-thread default stream (one handle, many streams), calls being captured into a graph (the graph may later
+// run on any stream) and streams beyond the pool take the fixed assignment.
+struct WideSched {
+    unsigned next, done;
+};
+constexpr int kWideSchedSlots = 256;
+__device__ WideSched g_wide_sched[kWideSchedSlots];
 
 constexpr int kWideCols = 64;
 constexpr unsigned kWidePlaneBytes = 81 * kWideCols * 4;
@@ -155,11 +170,12 @@ __device__ __forceinline__ bool wide_tile(const PlaneMaps& maps, const StrideAdd
 
 template <typename T>
 __global__ void __launch_bounds__(288, 1) k_lat_t999_wide(const __grid_constant__ PlaneMaps maps, StrideAddr out, LatArgs a,
-                                                          WideTiles w, unsigned* giveups) {
+                                                          WideTiles w, unsigned* giveups, WideSched* sched) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     T* slab = reinterpret_cast<T*>(smem_raw);                           // [9 planes][81][64]
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_raw + kWideTileBytes);
     int* gave_up = reinterpret_cast<int*>(bars + 9);
+    long long* next_tile = reinterpret_cast<long long*>(bars + 10);
     long long t = blockIdx.x;                                           // everything below is CTA-uniform
     if (t >= w.total) return;
     int c;
@@ -173,8 +189,20 @@ __global__ void __launch_bounds__(288, 1) k_lat_t999_wide(const __grid_constant_
         for (int k = 0; k < 9; ++k) wide_fetch_plane(maps, c, t0, k, smem_u32(slab), bars);
     }
     __syncthreads();                    // the barriers are initialised before anybody polls them
+    // the first tile is the CTA's own number; further ones are drawn from the counter (or t + grid without one), always one
+    // tile ahead: what thread 0 draws at the top of an iteration is read at the top of the next, many barriers later
+    auto draw = [&]() { return (long long)gridDim.x + atomicAdd(&sched->next, 1u); };
+    auto leave = [&]() {                // the last CTA of the launch hands the counter back as it found it
+        if (sched && threadIdx.x == 0 && atomicAdd(&sched->done, 1u) == gridDim.x - 1) {
+            sched->next = 0;
+            sched->done = 0;
+        }
+    };
+    if (sched && threadIdx.x == 0) next_tile[0] = draw();
+    __syncthreads();
     for (unsigned parity = 0;; parity ^= 1) {
-        const long long tn = t + gridDim.x;
+        const long long tn = sched ? next_tile[parity] : t + gridDim.x;
+        if (sched && threadIdx.x == 0) next_tile[parity ^ 1] = draw();
         const bool has_next = tn < w.total;
         int nc = 0;
         long long nt0 = 0;
@@ -190,11 +218,43 @@ __global__ void __launch_bounds__(288, 1) k_lat_t999_wide(const __grid_constant_
         }
         if (!ok) {                      // a wait ran out: counted once, this tile is not stored
             if (threadIdx.x == 0) atomicAdd(giveups, 1u);
+            leave();
             return;
         }
-        if (!has_next) return;
+        if (!has_next) {
+            leave();
+            return;
+        }
         t = tn; c = nc; t0 = nt0;
     }
+}
+
+// The counter of (current device, stream), or NULL (fixed assignment).  Host-side bookkeeping only.
+static WideSched* wide_sched_for(int dev, cudaStream_t st) {
+    if (st == cudaStreamPerThread) return nullptr;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    if (cap != cudaStreamCaptureStatusNone) return nullptr;
+    if (st == cudaStreamLegacy) st = nullptr;                   // both name the legacy default stream
+    struct PerDevice {
+        WideSched* base = nullptr;
+        std::map<cudaStream_t, int> slot;
+    };
+    static std::mutex mu;
+    static std::map<int, PerDevice> devices;
+    std::lock_guard<std::mutex> lock(mu);
+    PerDevice& d = devices[dev];
+    if (!d.base) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_wide_sched) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+        d.base = (WideSched*)p;
+    }
+    auto it = d.slot.find(st);
+    if (it == d.slot.end()) {
+        if ((int)d.slot.size() >= kWideSchedSlots) return nullptr;
+        it = d.slot.emplace(st, (int)d.slot.size()).first;
+    }
+    return d.base + it->second;
 }
 
 // false: this call cannot use the wide kernel (the caller goes on to the 32-column kernels)
@@ -222,15 +282,16 @@ bool run_fused_t999_wide(const Call& c, const LatArgs& a, trv_status_t* status) 
     for (int sl = 0; sl < 3; ++sl)
         if (!encode_planes(sin, c.count, a.rs[sl], kWideCols, &maps.in[sl])) return false;
     *status = TRV_OK;
-    constexpr int smem = (int)kWideTileBytes + 9 * 8 + 16;
+    constexpr int smem = (int)kWideTileBytes + 9 * 8 + 16 + 24;
     g_last_kernel = "lat_t999_wide";
     const unsigned grid = (unsigned)(w.total < sms ? w.total : sms);
+    WideSched* sched = wide_sched_for(dev, c.st);
     if (c.dtype == TRV_FLOAT32) {
         if (!allow_big_smem(k_lat_t999_wide<float>, smem)) { *status = TRV_ERR_CUDA; return true; }
-        TRV_LAUNCH((k_lat_t999_wide<float>), dim3(grid), 288, smem, c.st, maps, sout, a, w, giveups);
+        TRV_LAUNCH((k_lat_t999_wide<float>), dim3(grid), 288, smem, c.st, maps, sout, a, w, giveups, sched);
     } else {
         if (!allow_big_smem(k_lat_t999_wide<uint32_t>, smem)) { *status = TRV_ERR_CUDA; return true; }
-        TRV_LAUNCH((k_lat_t999_wide<uint32_t>), dim3(grid), 288, smem, c.st, maps, sout, a, w, giveups);
+        TRV_LAUNCH((k_lat_t999_wide<uint32_t>), dim3(grid), 288, smem, c.st, maps, sout, a, w, giveups, sched);
     }
     if (cudaGetLastError() != cudaSuccess) *status = TRV_ERR_CUDA;
     return true;

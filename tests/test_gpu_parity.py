@@ -77,9 +77,38 @@ def test_fused_latency_9x9x9_many_tiles_per_cta():
 def test_fused_latency_9x9x9_tiles_of_64_columns():
     """Long vectors on the 9x9x9 torus take the persistent kernel on 64-column tiles (one CTA per SM, the next tile
     loading while group 3 of the current one runs from registers): ragged slice edges that share a tile between two
-    slices, several tiles per CTA with both mbarrier parities, both dtypes, in place and not."""
-    check_case((9, 9, 9), LAT, 800003, "normal", 41, FUSED)
+    slices, many tiles per CTA with both mbarrier parities, both dtypes, in place and not.  Tiles are handed out from a
+    per-stream counter; a second stream gets its own; a call captured into a CUDA graph takes the fixed assignment
+    instead -- all must give the same bits."""
+    x, want = check_case((9, 9, 9), LAT, 800003, "normal", 41, FUSED)
     assert binding.last_kernel_name() == "lat_t999_wide"
+    plan = binding.Plan((9, 9, 9), LAT)
+    n, count = x.shape
+    pad = (count + 3) // 4 * 4
+    xin = torch.zeros((n, pad), dtype=torch.float32, device=DEV)
+    xin[:, :count].copy_(torch.from_numpy(x))
+    xout = torch.zeros_like(xin)
+    ip = binding.ptr_array([xin[r].data_ptr() for r in range(n)])
+    op = binding.ptr_array([xout[r].data_ptr() for r in range(n)])
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):       # twice on a stream of its own: the counter is back at zero after the first call
+        for _ in range(2):
+            xout.zero_()
+            plan.allreduce_ex(ip, op, count, binding.FLOAT32, kernel=FUSED, stream=side.cuda_stream)
+    side.synchronize()
+    assert binding.last_kernel_name() == "lat_t999_wide"
+    assert np.array_equal(xout[:, :count].cpu().numpy().view(np.uint32), want.view(np.uint32))
+    g = torch.cuda.CUDAGraph()
+    torch.cuda.synchronize()
+    with torch.cuda.graph(g):
+        plan.allreduce_ex(ip, op, count, binding.FLOAT32, kernel=FUSED, stream=torch.cuda.current_stream().cuda_stream)
+    xout.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert np.array_equal(xout[:, :count].cpu().numpy().view(np.uint32), want.view(np.uint32))
+    plan.destroy()
+    del xin, xout
     check_case((9, 9, 9), LAT, 786754, "int32", 42, FUSED, in_place=False)
     assert binding.last_kernel_name() == "lat_t999_wide"
     assert binding.tma_giveups() == 0
