@@ -21,7 +21,7 @@ OBJ = os.path.join(HERE, "build")
 # (source, extra flags, object name); the line-group kernel is compiled in parts (see its header comment)
 UNITS = [(s, [], os.path.splitext(s)[0] + ".o") for s in (
     "trv_plan.cc", "trv_api.cu", "trv_host.cu", "trv_step.cu", "trv_step_gen.cu", "trv_fused_lat.cu", "trv_fused_t999.cu",
-    "trv_fused_t999_tma.cu", "trv_fused_t999_wide.cu", "trv_fused_bw.cu", "trv_fused_tree.cu", "trv_pipe.cu", "trv_pipe_bw.cu", "trv_linkloads.cu", "trv_noalloc.cu", "trv_joint.cu", "trv_comparator.cu")]
+    "trv_fused_t999_tma.cu", "trv_fused_wide.cu", "trv_fused_bw.cu", "trv_fused_tree.cu", "trv_pipe.cu", "trv_pipe_bw.cu", "trv_linkloads.cu", "trv_noalloc.cu", "trv_joint.cu", "trv_comparator.cu")]
 UNITS += [("trv_fused_lines.cu", ["-DTRV_LN_PART=%d" % k], "trv_fused_lines_p%d.o" % k) for k in range(5)]
 SOURCES = sorted({u[0] for u in UNITS})
 NVCC_FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",

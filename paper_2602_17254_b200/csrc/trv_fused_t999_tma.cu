@@ -2,7 +2,7 @@
 //
 // Same three closed groups as k_lat_t999 (trv_fused_t999.cu); both kernels need equally spaced rank buffers (tensor
 // maps describe them as a matrix); other callers keep k_lat_t999.  Vectors from about 3 MiB per rank go to the
-// persistent kernel on 64-column tiles (trv_fused_t999_wide.cu) instead.
+// persistent kernel on 64-column tiles (trv_fused_wide.cu) instead.
 //   k_lat_t999_planes : the 32-column x 729-rank tile arrives as nine bulk tensor copies, one C-plane each, on nine
 //                       mbarriers, so group 1 starts plane by plane; the results leave through bulk tensor stores,
 //                       three planes after each phase of group 3.  729 x 32 MiB: 9.07 ms in a 0.7 s timed region under
@@ -291,6 +291,15 @@ static EncodeTiledFn encode_tiled_fn() {
         return (EncodeTiledFn)p;
     }();
     return fn;
+}
+
+// A tiled map of 4-byte words, no swizzle, 256-byte L2 promotion; gstride has rank - 1 entries (bytes).
+bool tma_encode_raw(CUtensorMap* out, int rank, void* base, const cuuint64_t* gdim, const cuuint64_t* gstride, const cuuint32_t* box) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint32_t estride[5] = {1, 1, 1, 1, 1};
+    return enc(out, CU_TENSOR_MAP_DATA_TYPE_UINT32, (cuuint32_t)rank, base, gdim, gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 bool tma_encode_ranks(const StrideAddr& in, int n, size_t count, int box_rows, CUtensorMap* out) {

@@ -1,4 +1,5 @@
-// FUSED latency-optimal kernel for the 9 x 9 x 9 torus (Sec. 4.2, Sec. 5) on tiles of 64 element columns.
+// FUSED latency-optimal kernels for the 729-rank tori 9 x 9 x 9 and 27 x 27 (Sec. 4.2, Sec. 5) on tiles of 64 element
+// columns, for long vectors.
 //
 // Why 64 columns: every tile touches all 729 input rows and all 729 output rows.  A plain copy that moves 128 bytes
 // per row visit (32 columns) stops at 0.89 - 0.90 of the copy bandwidth on this part however many CTAs are resident,
@@ -16,7 +17,11 @@
 // Measured on the way and dropped: all of group 3's 81 values in registers before a single refill of nine planes
 // (spills at 168 registers, 8.56 ms); eleven plane slots with the planes 2 and 5 of the tile after the next loading
 // early (8.75 ms: the run-time slot arithmetic costs more than the two planes' head start gains).
-// The same three closed groups as the other 9 x 9 x 9 kernels: (A,1)(B,1) per C-plane, (C,1)(A,3), (B,3)(C,3).
+// 9 x 9 x 9: the same three closed groups as the other 9 x 9 x 9 kernels: (A,1)(B,1) per C-plane, (C,1)(A,3), (B,3)(C,3).
+// 27 x 27 (steps A1 B1 A3 B3 A9 B9): a plane is three A-lines (81 ranks); four groups: (A,1) on the 27-rank A-lines of a
+// plane, (B,1) on the B-lines, (A,3)(B,3) on the nine 9 x 9 sets {A = a0 + 3 i, B = b0 + 3 j} streamed row by row, and
+// (A,9)(B,9) on 3 x 3 sets in three phases whose planes are k0, k0 + 3, k0 + 6 -- the phase structure the refill needs.
+// 27 x 27, 729 x 8 MiB: 3132 us with the line-group kernel -> 2400 us.
 // Every wait on a copy's mbarrier is bounded; a CTA that gives up counts it (trv_tma.cuh) and leaves without
 // storing the tile it waited for.
 #include <map>
@@ -51,7 +56,7 @@ struct WideTiles {
 
 __device__ __forceinline__ void wide_locate(const WideTiles& w, const LatArgs& a, long long t, int* c, long long* t0) {
     int s = 0;
-    while (s < 2 && t >= w.nx[s]) { t -= w.nx[s]; ++s; }
+    while (s < 2 && t >= w.nx[s]) { t -= w.nx[s]; ++s; }        // nx[s] = 0 for slices the shape does not have
     *c = s;
     *t0 = (a.lo[s] & ~(long long)(kWideCols - 1)) + t * kWideCols;
 }
@@ -168,9 +173,174 @@ __device__ __forceinline__ bool wide_tile(const PlaneMaps& maps, const StrideAdd
     return true;
 }
 
-template <typename T>
-__global__ void __launch_bounds__(288, 1) k_lat_t999_wide(const __grid_constant__ PlaneMaps maps, StrideAddr out, LatArgs a,
-                                                          WideTiles w, unsigned* giveups, WideSched* sched) {
+
+// bounded wait of a warp for its plane of the current tile
+__device__ __forceinline__ void wide_wait_plane(unsigned long long* bars, int k, unsigned parity, int* gave_up) {
+    unsigned done = 0;
+    const unsigned bar_s = smem_u32(bars + k);
+    for (unsigned spins = 0; spins < kTmaWaitLimit; ++spins) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar_s), "r"(parity)
+            : "memory");
+        if (done) break;
+    }
+    if (!done) *gave_up = 1;
+}
+
+struct ShapeT999 {
+    static constexpr int kSlices = 3;
+    __device__ static __forceinline__ void fetch(const PlaneMaps& maps, int c, long long t0, int k, unsigned slab_s,
+                                                 unsigned long long* bars) {
+        wide_fetch_plane(maps, c, t0, k, slab_s, bars);
+    }
+    template <typename T>
+    __device__ static __forceinline__ bool tile(const PlaneMaps& maps, const StrideAddr& out, const LatArgs& a, int c, long long t0,
+                                                bool full, unsigned parity, bool has_next, int nc, long long nt0, T* slab,
+                                                unsigned long long* bars, int* gave_up) {
+        if (c == 2)
+            return full ? wide_tile<T, 9, true>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up)
+                        : wide_tile<T, 9, false>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up);
+        return full ? wide_tile<T, 1, true>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up)
+                    : wide_tile<T, 1, false>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up);
+    }
+};
+
+// ------------------------------------------------------------------ 27 x 27
+//
+// Slice c runs the steps (A,1) (B,1) (A,3) (B,3) (A,9) (B,9) with A = dimension c, B = the other one (Sec. 5).  Plane
+// k = the three A-lines with B in 3k .. 3k + 2.  The slice's tensor map has the dimension with the smaller rank stride
+// first, so a plane lands as [B - 3k][A] for slice 0 (PA = 1, PB = 27) and as [A][B - 3k] for slice 1 (PA = 3, PB = 1).
+__device__ __forceinline__ void wide_fetch_plane_2727(const PlaneMaps& maps, int c, long long t0, int k, unsigned slab_s,
+                                                      unsigned long long* bars) {
+    const unsigned bar_s = smem_u32(bars + k);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s), "r"(kWidePlaneBytes) : "memory");
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+            slab_s + k * kWidePlaneBytes),
+        "l"(&maps.in[c]), "r"((int)t0), "r"(c == 1 ? 3 * k : 0), "r"(c == 0 ? 3 * k : 0), "r"(bar_s)
+        : "memory");
+}
+
+template <typename T, int PA, bool FULL>
+__device__ __forceinline__ bool wide_tile_2727(const PlaneMaps& maps, const StrideAddr& out, const LatArgs& a, int c, long long t0,
+                                               unsigned parity, bool has_next, int nc, long long nt0, T* slab,
+                                               unsigned long long* bars, int* gave_up) {
+    constexpr int PB = PA == 1 ? 27 : 1, PK = 81;       // row of (A, B) in the slab: (B / 3) * PK + A * PA + (B % 3) * PB
+    using E = Elem<T, 2>;
+    const int lane = threadIdx.x % 32, set = threadIdx.x / 32;
+    const long long lo = a.lo[c], hi = a.hi[c];
+    const long long e = t0 + 2 * lane;
+    E* const mine = reinterpret_cast<E*>(slab) + lane;
+    auto sl = [&](int r) -> E& { return mine[r * (kWideCols / 2)]; };
+    // ---- group 1: (A,1) on the three A-lines of the plane `set`, as soon as it has arrived
+    wide_wait_plane(bars, set, parity, gave_up);
+#pragma unroll 1
+    for (int b = 0; b < 3; ++b) {
+        const int r0 = set * PK + b * PB;
+        E v[27];
+#pragma unroll
+        for (int i = 0; i < 27; ++i) v[i] = sl(r0 + i * PA);
+        reg_step<27, 1, 27, 1>(v);
+#pragma unroll
+        for (int i = 0; i < 27; ++i) sl(r0 + i * PA) = v[i];
+    }
+    __syncthreads();
+    if (*gave_up) return false;
+    // ---- group 2: (B,1) on the B-lines A = set + 9 m
+#pragma unroll 1
+    for (int m = 0; m < 3; ++m) {
+        const int r0 = (set + 9 * m) * PA;
+        E v[27];
+#pragma unroll
+        for (int j = 0; j < 27; ++j) v[j] = sl(r0 + (j / 3) * PK + (j % 3) * PB);
+        reg_step<27, 1, 27, 1>(v);
+#pragma unroll
+        for (int j = 0; j < 27; ++j) sl(r0 + (j / 3) * PK + (j % 3) * PB) = v[j];
+    }
+    __syncthreads();
+    {   // ---- group 3: (A,3) (B,3) on the set {A = a0 + 3 i, B = b0 + 3 j}: a 9 x 9 torus, row j = plane j, streamed
+        const int r0 = (set % 3) * PA + (set / 3) * PB;
+        auto load_row = [&](int j, E (&row)[9]) {
+#pragma unroll
+            for (int i = 0; i < 9; ++i) row[i] = sl(r0 + 3 * i * PA + j * PK);
+            reg_step<9, 1, 9, 1>(row);                                      // (A,3)
+        };
+        auto emit = [&](int j, const E (&p)[9], const E (&q)[9], const E (&r)[9]) {     // (B,3) for row j
+#pragma unroll
+            for (int i = 0; i < 9; ++i) sl(r0 + 3 * i * PA + j * PK) = add3(p[i], q[i], r[i]);
+        };
+        E first[9], second[9], prev[9], cur[9], next[9];
+        load_row(0, first);
+        load_row(1, second);
+#pragma unroll
+        for (int i = 0; i < 9; ++i) { prev[i] = first[i]; cur[i] = second[i]; }
+#pragma unroll
+        for (int j = 1; j < 8; ++j) {
+            load_row(j + 1, next);          // row j + 1 is read before row j is overwritten
+            emit(j, prev, cur, next);
+#pragma unroll
+            for (int i = 0; i < 9; ++i) { prev[i] = cur[i]; cur[i] = next[i]; }
+        }
+        emit(8, prev, cur, first);
+        emit(0, cur, first, second);
+    }
+    __syncthreads();
+    // ---- group 4: (A,9) (B,9) on the sets {A = a + 9 i, B = b + 9 j}; phase k0 takes the b with b / 3 = k0, whose planes are
+    // k0, k0 + 3, k0 + 6; flat index i + 3 j
+    const int sA = a.rs[c][0], sB = a.rs[c][1];
+    const unsigned slab_s = smem_u32(slab);
+#pragma unroll 1
+    for (int k0 = 0; k0 < 3; ++k0) {
+        E v[3][9];
+#pragma unroll
+        for (int m = 0; m < 3; ++m) {
+            const int q = set + 9 * m, r0 = (q % 9) * PA + (q / 9) * PB + k0 * PK;      // a = q % 9, b = 3 k0 + q / 9
+#pragma unroll
+            for (int idx = 0; idx < 9; ++idx) v[m][idx] = sl(r0 + 9 * (idx % 3) * PA + 3 * (idx / 3) * PK);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // this thread's slab accesses before the engine's writes
+        __syncthreads();                    // everybody holds its part of the planes k0, k0 + 3, k0 + 6: they may be refilled
+        if (threadIdx.x == 0 && has_next) {
+            for (int kk = 0; kk < 3; ++kk) wide_fetch_plane_2727(maps, nc, nt0, k0 + 3 * kk, slab_s, bars);
+        }
+#pragma unroll
+        for (int m = 0; m < 3; ++m) {
+            const int q = set + 9 * m, g0 = (q % 9) * sA + (3 * k0 + q / 9) * sB;
+            reg_step<9, 1, 3, 1>(v[m]);     // (A,9)
+            reg_step<9, 3, 3, 1>(v[m]);     // (B,9)
+            if (FULL || (e < hi && e + 2 > lo)) {
+#pragma unroll
+                for (int idx = 0; idx < 9; ++idx)
+                    store_elem<T, 2, FULL>(out.ptr(g0 + 9 * (idx % 3) * sA + 9 * (idx / 3) * sB), e, lo, hi, v[m][idx]);
+            }
+        }
+    }
+    return true;
+}
+
+struct Shape2727 {
+    static constexpr int kSlices = 2;
+    __device__ static __forceinline__ void fetch(const PlaneMaps& maps, int c, long long t0, int k, unsigned slab_s,
+                                                 unsigned long long* bars) {
+        wide_fetch_plane_2727(maps, c, t0, k, slab_s, bars);
+    }
+    template <typename T>
+    __device__ static __forceinline__ bool tile(const PlaneMaps& maps, const StrideAddr& out, const LatArgs& a, int c, long long t0,
+                                                bool full, unsigned parity, bool has_next, int nc, long long nt0, T* slab,
+                                                unsigned long long* bars, int* gave_up) {
+        if (c == 1)
+            return full ? wide_tile_2727<T, 3, true>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up)
+                        : wide_tile_2727<T, 3, false>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up);
+        return full ? wide_tile_2727<T, 1, true>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up)
+                    : wide_tile_2727<T, 1, false>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up);
+    }
+};
+
+template <typename T, typename Shape>
+__global__ void __launch_bounds__(288, 1) k_lat_wide(const __grid_constant__ PlaneMaps maps, StrideAddr out, LatArgs a,
+                                                     WideTiles w, unsigned* giveups, WideSched* sched) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     T* slab = reinterpret_cast<T*>(smem_raw);                           // [9 planes][81][64]
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_raw + kWideTileBytes);
@@ -186,7 +356,7 @@ __global__ void __launch_bounds__(288, 1) k_lat_t999_wide(const __grid_constant_
         for (int k = 0; k < 9; ++k) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bars + k)), "r"(1) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        for (int k = 0; k < 9; ++k) wide_fetch_plane(maps, c, t0, k, smem_u32(slab), bars);
+        for (int k = 0; k < 9; ++k) Shape::fetch(maps, c, t0, k, smem_u32(slab), bars);
     }
     __syncthreads();                    // the barriers are initialised before anybody polls them
     // the first tile is the CTA's own number; further ones are drawn from the counter (or t + grid without one), always one
@@ -208,14 +378,7 @@ __global__ void __launch_bounds__(288, 1) k_lat_t999_wide(const __grid_constant_
         long long nt0 = 0;
         if (has_next) wide_locate(w, a, tn, &nc, &nt0);
         const bool full = t0 >= a.lo[c] && t0 + kWideCols <= a.hi[c];
-        bool ok;
-        if (c == 2) {
-            ok = full ? wide_tile<T, 9, true>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up)
-                      : wide_tile<T, 9, false>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up);
-        } else {
-            ok = full ? wide_tile<T, 1, true>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up)
-                      : wide_tile<T, 1, false>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up);
-        }
+        const bool ok = Shape::template tile<T>(maps, out, a, c, t0, full, parity, has_next, nc, nt0, slab, bars, gave_up);
         if (!ok) {                      // a wait ran out: counted once, this tile is not stored
             if (threadIdx.x == 0) atomicAdd(giveups, 1u);
             leave();
@@ -257,8 +420,14 @@ static WideSched* wide_sched_for(int dev, cudaStream_t st) {
     return d.base + it->second;
 }
 
+// Tensor map of one slice of the 27 x 27 torus over equally spaced rank buffers: dimensions (column, then the two torus
+// dimensions by increasing rank stride), boxes of 64 columns x 27 along the slice's own dimension x 3 along the other.
+static bool encode_planes_2727(const StrideAddr& base, size_t count, int slice, CUtensorMap* out);
+
 // false: this call cannot use the wide kernel (the caller goes on to the 32-column kernels)
-bool run_fused_t999_wide(const Call& c, const LatArgs& a, trv_status_t* status) {
+template <typename Shape>
+static bool run_wide(const Call& c, const LatArgs& a, const char* name, trv_status_t* status) {
+    constexpr int NS = Shape::kSlices;
     StrideAddr sin, sout;
     if (!uniform_stride(c.in, 729, &sin) || !uniform_stride((const void* const*)c.out, 729, &sout)) return false;
     if ((sout.stride & 7) || ((uintptr_t)sout.base & 7)) return false;      // two-column stores
@@ -266,35 +435,59 @@ bool run_fused_t999_wide(const Call& c, const LatArgs& a, trv_status_t* status) 
     w.total = 0;
     long long local = 0;            // elements of this call's window, all slices
     for (int sl = 0; sl < 3; ++sl) {
-        if (a.hi[sl] > a.lo[sl]) local += a.hi[sl] - a.lo[sl];
-        w.nx[sl] = a.hi[sl] > a.lo[sl] ? (a.hi[sl] - (a.lo[sl] & ~(long long)(kWideCols - 1)) + kWideCols - 1) / kWideCols : 0;
+        w.nx[sl] = 0;
+        if (sl >= NS || a.hi[sl] <= a.lo[sl]) continue;
+        local += a.hi[sl] - a.lo[sl];
+        w.nx[sl] = (a.hi[sl] - (a.lo[sl] & ~(long long)(kWideCols - 1)) + kWideCols - 1) / kWideCols;
         w.total += w.nx[sl];
     }
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
         return false;
-    // From about 3 MiB per rank on: 4 MiB per rank 1155 -> 1084 us, 8 MiB 2314 -> 2156 us, 32 MiB 9.05 -> 8.5 ms; at 2 MiB the
-    // two kernels tie, below it the 32-column kernels win (more, smaller tiles to spread over the SMs).
-    if (local < (3LL << 18) || w.total < 2LL * sms || w.total > (1LL << 30)) return false;     // short vectors: the 32-column kernels have more tiles to spread
+    // From about 3 MiB per rank on (9 x 9 x 9: 4 MiB per rank 1155 -> 1084 us, 8 MiB 2314 -> 2156 us, 32 MiB 9.05 -> 8.5 ms; at
+    // 2 MiB the two kernels tie, below it the 32-column kernels win: more, smaller tiles to spread over the SMs).
+    // 27 x 27 has no 32-column TMA kernel to fall back to, only the line-group kernel, and wins from 256 KiB per rank on
+    // (64 Ki elements: 114 -> 91 us; 512 Ki: 811 -> 611 us; 2 Mi: 3132 -> 2400 us; 8 Mi: 9.44 ms, 0.79 of the copy bandwidth).
+    if (local < (NS == 2 ? (1LL << 16) : (3LL << 18)) || w.total < 2LL * sms || w.total > (1LL << 30)) return false;
     unsigned* giveups = tma_giveup_counter();
     if (!giveups) return false;
     PlaneMaps maps;
-    for (int sl = 0; sl < 3; ++sl)
-        if (!encode_planes(sin, c.count, a.rs[sl], kWideCols, &maps.in[sl])) return false;
+    for (int sl = 0; sl < NS; ++sl) {
+        const bool ok = NS == 3 ? encode_planes(sin, c.count, a.rs[sl], kWideCols, &maps.in[sl]) : encode_planes_2727(sin, c.count, sl, &maps.in[sl]);
+        if (!ok) return false;
+    }
     *status = TRV_OK;
     constexpr int smem = (int)kWideTileBytes + 9 * 8 + 16 + 24;
-    g_last_kernel = "lat_t999_wide";
+    g_last_kernel = name;
     const unsigned grid = (unsigned)(w.total < sms ? w.total : sms);
     WideSched* sched = wide_sched_for(dev, c.st);
     if (c.dtype == TRV_FLOAT32) {
-        if (!allow_big_smem(k_lat_t999_wide<float>, smem)) { *status = TRV_ERR_CUDA; return true; }
-        TRV_LAUNCH((k_lat_t999_wide<float>), dim3(grid), 288, smem, c.st, maps, sout, a, w, giveups, sched);
+        if (!allow_big_smem(k_lat_wide<float, Shape>, smem)) { *status = TRV_ERR_CUDA; return true; }
+        TRV_LAUNCH((k_lat_wide<float, Shape>), dim3(grid), 288, smem, c.st, maps, sout, a, w, giveups, sched);
     } else {
-        if (!allow_big_smem(k_lat_t999_wide<uint32_t>, smem)) { *status = TRV_ERR_CUDA; return true; }
-        TRV_LAUNCH((k_lat_t999_wide<uint32_t>), dim3(grid), 288, smem, c.st, maps, sout, a, w, giveups, sched);
+        if (!allow_big_smem(k_lat_wide<uint32_t, Shape>, smem)) { *status = TRV_ERR_CUDA; return true; }
+        TRV_LAUNCH((k_lat_wide<uint32_t, Shape>), dim3(grid), 288, smem, c.st, maps, sout, a, w, giveups, sched);
     }
     if (cudaGetLastError() != cudaSuccess) *status = TRV_ERR_CUDA;
     return true;
+}
+
+bool run_fused_t999_wide(const Call& c, const LatArgs& a, trv_status_t* status) { return run_wide<ShapeT999>(c, a, "lat_t999_wide", status); }
+
+// 27 x 27 with rank = x0 + 27 x1 (the plan's layout); false: not this shape or not this call
+bool run_fused_t2727_wide(const Call& c, const LatArgs& a, trv_status_t* status) {
+    const Plan& p = *c.plan;
+    if (p.ndims != 2 || p.dims[0] != 27 || p.dims[1] != 27 || p.stride[0] != 1 || p.stride[1] != 27) return false;
+    return run_wide<Shape2727>(c, a, "lat_t27x27_wide", status);
+}
+
+static bool encode_planes_2727(const StrideAddr& base, size_t count, int slice, CUtensorMap* out) {
+    if ((base.stride & 15) || ((uintptr_t)base.base & 15) || count == 0 || count >= ((size_t)1 << 31)) return false;
+    if ((size_t)base.stride < count * 4) return false;
+    const cuuint64_t gdim[3] = {(cuuint64_t)count, 27, 27};
+    const cuuint64_t gstride[2] = {(cuuint64_t)base.stride, (cuuint64_t)27 * base.stride};
+    const cuuint32_t box[3] = {(cuuint32_t)kWideCols, slice == 0 ? 27u : 3u, slice == 0 ? 3u : 27u};
+    return tma_encode_raw(out, 3, base.base, gdim, gstride, box);
 }
 
 }  // namespace trv

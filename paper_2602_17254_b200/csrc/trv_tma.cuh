@@ -61,6 +61,7 @@ struct PlaneMaps {
     CUtensorMap in[3], out[3];      // one pair per slice: dimensions ordered by increasing rank stride
 };
 bool encode_planes(const StrideAddr& base, size_t count, const int strides[3], int box_cols, CUtensorMap* out);
+bool tma_encode_raw(CUtensorMap* out, int rank, void* base, const cuuint64_t* gdim, const cuuint64_t* gstride, const cuuint32_t* box);
 unsigned* tma_giveup_counter();     // device address of the counter on the current device (NULL on failure)
 unsigned tma_giveups();             // its value (synchronous copy); ~0u on failure
 

@@ -114,6 +114,16 @@ def test_fused_latency_9x9x9_tiles_of_64_columns():
     assert binding.tma_giveups() == 0
 
 
+def test_fused_latency_27x27_tiles_of_64_columns():
+    """Long vectors on the 27 x 27 torus take the same persistent 64-column kernel with the 27 x 27 groups: both slices
+    (dimension orders), ragged slice edges, both dtypes, in place and not."""
+    check_case((27, 27), LAT, 70001, "normal", 51, FUSED)
+    assert binding.last_kernel_name() == "lat_t27x27_wide"
+    check_case((27, 27), LAT, 300034, "int32", 52, FUSED, in_place=False)
+    assert binding.last_kernel_name() == "lat_t27x27_wide"
+    assert binding.tma_giveups() == 0
+
+
 def test_fused_bandwidth_wide_path_on_729_ranks_sampled():
     """9x9x9 with blocks of >= 256 elements: the oracle checks windows around slice and block
     boundaries and in block interiors."""
