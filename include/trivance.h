@@ -114,7 +114,10 @@ trv_status_t trv_plan_create(const int32_t *dims, int32_t ndims, trv_variant_t v
  * collective per dimension, visiting the dimensions in round-robin order like Trivance, 2 D collectives when
  * mirrored.  `algo | TRV_ALGO_SINGLE` (these two, not mirrored): ONE collective on the whole vector that walks
  * through the dimensions in turn, which is how their latency-optimal forms use a torus (App. B: "only a
- * single port per node").  Bruck takes power-of-three tori, Bucket rings only.
+ * single port per node").  Bruck takes power-of-three tori.  Bucket takes tori of any sides >= 2 (Sec. 2.4):
+ * collective c runs the ring algorithm along dimension c, then c + 1, ... on the blocks a node still answers for (those
+ * that agree with its coordinates in the earlier dimensions), sum of (a_d - 1) steps per phase; the AllGather rows take
+ * the dimensions in reverse order; D collectives, 2 D when mirrored.
  * Comparator plans serve trv_link_loads, trv_cost_model and the schedule queries, and they are executable:
  * trv_allreduce / trv_allreduce_ex (TRV_KERNEL_AUTO or TRV_KERNEL_STEP) run them step by step, literally -- at
  * the start of a step every rank's vector is copied to a wire buffer (scratch of n * round_up(count, 64) * 4

@@ -47,6 +47,10 @@
  *   - the ring (Bucket) algorithm sends block (r - t - 1) mod n in Reduce-Scatter step t and block
  *     (r - t) mod n in AllGather step t, always to r + 1: block j ends at node j.  Any such
  *     numbering gives the same loads when the blocks have equal length.
+ *     On a torus (Sec. 2.4's two sentences on it) the ring algorithm runs dimension after dimension, collective c
+ *     starting with dimension c, each phase on the blocks that agree with the node in the earlier dimensions; the
+ *     AllGather takes the phases in reverse order.  PARITY UNPINNED by the paper beyond Table 2's Theta = 1 and the
+ *     step count, which the tests check; the sums themselves are pinned by the plain column sums.
  *
  * Floating point: binary32 (or binary64 for the error-bound checks), one add
  * at a time, no contraction, no reassociation.  Compile with
@@ -92,19 +96,26 @@ static int topo_init(orc_topo *tp, const int32_t *dims, int ndims, int algo) {
     algo &= ~(ORC_MIRROR | ORC_SINGLE);
     if (algo < ORC_TRIVANCE || algo > ORC_BUCKET) return ORC_BAD_ARG;
     if (mirror && algo == ORC_TRIVANCE) return ORC_BAD_ARG;
-    if (mirror && ndims != 1 && algo != ORC_RECDOUB && algo != ORC_SWING) return ORC_BAD_ARG;
+    if (mirror && ndims != 1 && algo != ORC_RECDOUB && algo != ORC_SWING && algo != ORC_BUCKET) return ORC_BAD_ARG;
     /* ORC_SINGLE: ONE collective on the whole vector that walks through the dimensions in turn -- how the
      * latency-optimal Recursive Doubling and Swing use a torus ("only a single port per node", App. B) */
     if (single && (mirror || (algo != ORC_RECDOUB && algo != ORC_SWING))) return ORC_BAD_ARG;
     tp->algo = algo; tp->ndims = ndims; tp->nsl = single ? 1 : ndims * (mirror ? 2 : 1);
     tp->base = (algo == ORC_RECDOUB || algo == ORC_SWING) ? 2 : 3;
-    /* Recursive Doubling and Swing on tori (Sec. 2.4): one collective per dimension, each with its mirrored
-     * sub-collective when asked for (2D collectives on 1/(2D) of the vector each); Bucket: rings only here. */
-    if (algo == ORC_BUCKET && ndims != 1) return ORC_UNDEFINED;
-    if (algo == ORC_BUCKET) {           /* ring algorithm: any n >= 2, n - 1 steps per phase (Sec. 2.4) */
-        if (dims[0] < 2 || dims[0] > 4096) return ORC_BAD_ARG;
-        tp->dims[0] = dims[0]; tp->stride[0] = 1; tp->sdim[0] = dims[0] - 1;
-        tp->n = dims[0]; tp->S = dims[0] - 1;
+    /* Recursive Doubling, Swing and Bucket on tori (Sec. 2.4): one collective per dimension, each with its mirrored
+     * sub-collective when asked for (2D collectives on 1/(2D) of the vector each). */
+    if (algo == ORC_BUCKET) {
+        /* The ring algorithm, any sides >= 2 (Sec. 2.4): a ring Reduce-Scatter of a_d - 1 steps along one dimension
+         * after the other on the partially reduced data, then the AllGather phases in reverse order.  Collective c
+         * starts with dimension c; see bucket_where. */
+        long long nn = 1; tp->S = 0;
+        for (int d = 0; d < ndims; ++d) {
+            if (dims[d] < 2 || dims[d] > 4096) return ORC_BAD_ARG;
+            tp->dims[d] = dims[d]; tp->stride[d] = (int)nn; tp->sdim[d] = dims[d] - 1;
+            nn *= dims[d]; tp->S += dims[d] - 1;
+            if (nn > 4096) return ORC_BAD_ARG;
+        }
+        tp->n = (int)nn;
         return ORC_OK;
     }
     long long n = 1; tp->S = 0;
@@ -148,6 +159,41 @@ static int shift_rank(const orc_topo *tp, int r, int d, int delta) {
     int x = (r / st) % a;
     int y = ((x + delta) % a + a) % a;
     return r + (y - x) * st;
+}
+
+/* Bucket on a torus (Sec. 2.4).  Collective c walks the dimensions c, c + 1, ... (mod D); in the phase of dimension d
+ * the a_d nodes of every line along d run the ring algorithm on the blocks they still answer for: those that agree
+ * with the node's own coordinates in the dimensions of the earlier phases (block j ends at node j).  Row numbering:
+ * Reduce-Scatter rows 0 .. S-1 take the phases in order, AllGather rows S .. 2S-1 take them in reverse order; inside
+ * a phase the steps s = 0 .. a_d - 2 run forwards in both.  Returns the dimension, the step inside the phase and the
+ * bit mask of the dimensions of the earlier phases. */
+static void bucket_where(const orc_topo *tp, int c, int row, int *d, int *s, int *earlier) {
+    int D = tp->ndims, d0 = c % D, ag = row >= tp->S, i = ag ? row - tp->S : row;
+    for (int k = 0; k < D; ++k) {
+        int ph = ag ? D - 1 - k : k, dd = (d0 + ph) % D, len = tp->dims[dd] - 1;
+        if (i < len) {
+            int mask = 0;
+            for (int q = 0; q < ph; ++q) mask |= 1 << ((d0 + q) % D);
+            *d = dd; *s = i; *earlier = mask;
+            return;
+        }
+        i -= len;
+    }
+    *d = 0; *s = 0; *earlier = 0;
+}
+
+/* The blocks of the message node r passes to its neighbour r + sg e_d in that row: Reduce-Scatter step s carries the
+ * blocks whose d-coordinate is r_d - sg (s + 1), AllGather step s those with r_d - sg s (the ring rule "block
+ * r - t - 1, then block r - t", Sec. 2.4), both restricted to the blocks that agree with r in the earlier dimensions. */
+static void bucket_message(const orc_topo *tp, int r, int row, int d, int s, int earlier, int sg, uint8_t *set) {
+    int a = tp->dims[d], ag = row >= tp->S;
+    int want = (((r / tp->stride[d]) % a - sg * (s + (ag ? 0 : 1))) % a + a) % a;
+    for (int j = 0; j < tp->n; ++j) {
+        int ok = ((j / tp->stride[d]) % a) == want;
+        for (int q = 0; q < tp->ndims && ok; ++q)
+            if (((earlier >> q) & 1) && (j / tp->stride[q]) % tp->dims[q] != (r / tp->stride[q]) % tp->dims[q]) ok = 0;
+        set[j] = (uint8_t)ok;
+    }
 }
 
 /* Peers a rank SENDS to in a step of (dim, dist).  Returns their number;
@@ -502,17 +548,23 @@ int orc_bytes_sent(const int32_t *dims, int ndims, int variant, int algo, int64_
         /* Reduce-Scatter step t: node r sends block (r - t - 1) mod n on; AllGather step t: block (r - t) mod n
          * (block j ends at node j); a mirrored collective runs the ring the other way round (Sec. 2.4). */
         if (variant != ORC_BANDWIDTH) return ORC_UNDEFINED;
+        uint8_t *msg = (uint8_t *)malloc((size_t)n);
+        if (!msg) return ORC_NOMEM;
         memset(sent, 0, sizeof(int64_t) * (size_t)n);
         for (int c = 0; c < D; ++c) {
             int64_t slo, shi; int sg = c >= tp.ndims ? -1 : 1;
             slice_bounds(E, D, c, &slo, &shi);
-            for (int row = 0; row < T; ++row)
+            for (int row = 0; row < T; ++row) {
+                int d, s, earlier;
+                bucket_where(&tp, c, row, &d, &s, &earlier);
                 for (int r = 0; r < n; ++r) {
-                    int t = row < S ? row : row - S;
-                    int j = (((r - sg * (t + (row < S ? 1 : 0))) % n) + n) % n;
-                    sent[r] += (block_bound(slo, shi, n, j + 1) - block_bound(slo, shi, n, j)) * elem_size;
+                    bucket_message(&tp, r, row, d, s, earlier, sg, msg);
+                    for (int j = 0; j < n; ++j)
+                        if (msg[j]) sent[r] += (block_bound(slo, shi, n, j + 1) - block_bound(slo, shi, n, j)) * elem_size;
                 }
+            }
         }
+        free(msg);
         return ORC_OK;
     }
     uint8_t *set = (uint8_t *)malloc((size_t)n);
@@ -588,14 +640,17 @@ int orc_link_loads(const int32_t *dims, int ndims, int variant, int algo, int64_
         for (int c = 0; c < NSL; ++c) {
             int64_t slo, shi; int sg = c >= tp.ndims ? -1 : 1;
             slice_bounds(E, NSL, c, &slo, &shi);
-            for (int row = 0; row < T; ++row)
-                for (int r = 0; r < n; ++r) {
-                    int t = row < S ? row : row - S;
-                    int j = (((r - sg * (t + (row < S ? 1 : 0))) % n) + n) % n;
-                    size_t li = (((size_t)row * n + r) * D + 0) * 2 + (sg > 0 ? 0 : 1);
+            for (int row = 0; row < T; ++row) {
+                int d, s, earlier;
+                bucket_where(&tp, c, row, &d, &s, &earlier);
+                for (int r = 0; r < n; ++r) {       /* one message over the one link from r to its neighbour along d */
+                    size_t li = (((size_t)row * n + r) * D + d) * 2 + (sg > 0 ? 0 : 1);
+                    bucket_message(&tp, r, row, d, s, earlier, sg, set);
                     lm[li] += 1;
-                    lb[li] += (block_bound(slo, shi, n, j + 1) - block_bound(slo, shi, n, j)) * elem_size;
+                    for (int j = 0; j < n; ++j)
+                        if (set[j]) lb[li] += (block_bound(slo, shi, n, j + 1) - block_bound(slo, shi, n, j)) * elem_size;
                 }
+            }
         }
     } else
     for (int c = 0; c < NSL; ++c) {
@@ -1145,7 +1200,8 @@ done:
  *   bandwidth form : Reduce-Scatter: the message to peer p carries the blocks p still answers for after the step
  *                    (p's own and all it forwards later: the same sets the link-load tally uses); AllGather: the
  *                    steps in reverse order, a rank sends every finished block it holds to the step's peers.
- *                    Bucket: step t passes block r - t - 1 (Reduce-Scatter) resp. r - t (AllGather) to r + 1.
+ *                    Bucket: step t passes block r - t - 1 (Reduce-Scatter) resp. r - t (AllGather) to r + 1; on a torus
+ *                    dimension after dimension on the blocks still answered for (bucket_where, bucket_message).
  * Reading (PARITY UNPINNED by the paper, which never states an association order): a rank that receives m0 from the
  * sender whose FIRST peer it is and m1 from the sender whose SECOND peer it is forms (m1 + own) + m0; with one
  * message own + m0.  For Trivance's peers (first = left, second = right) this is (from_left + own) + from_right.
@@ -1157,7 +1213,7 @@ static int algo_slice_##SUFFIX(const orc_topo *tp, int c, int variant, int64_t s
     int64_t c0 = clampi(slo, e0, e1) - e0, c1 = clampi(shi, e0, e1) - e0, wc = c1 - c0;                         \
     if (wc <= 0) return ORC_OK;                                                                                 \
     int sd[64], sx[64];                                                                                         \
-    int sg = c >= tp->ndims ? -1 : 1;                                                                           \
+    int sg = c >= tp->ndims ? -1 : 1, bd = 0, bstep = 0, bearlier = 0;   /* Bucket: direction; dimension, step, earlier dimensions of the row */ \
     if (tp->algo != ORC_BUCKET) step_list(tp, c, sd, sx);                                                       \
     int64_t *bs = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n + 1));                                         \
     T *wire = (T *)malloc(sizeof(T) * (size_t)n * (size_t)wc);       /* what every rank puts on the wire */       \
@@ -1172,7 +1228,7 @@ static int algo_slice_##SUFFIX(const orc_topo *tp, int c, int variant, int64_t s
         for (int r = 0; r < n; ++r) {                                                                           \
             int peer[2] = {-1, -1}, dir[2], hops[2];                                                            \
             int np = tp->algo == ORC_BUCKET ? 1 : send_peers(tp, r, sd[t], sx[t], peer, dir, hops);             \
-            if (tp->algo == ORC_BUCKET) peer[0] = ((r + sg) % n + n) % n;                                       \
+            if (tp->algo == ORC_BUCKET) { bucket_where(tp, c, t, &bd, &bstep, &bearlier); peer[0] = shift_rank(tp, r, bd, sg); } \
             for (int k = 0; k < np; ++k) {                                                                      \
                 if (from[2 * peer[k] + k] >= 0) { rc = ORC_INTERNAL; goto done; }                               \
                 from[2 * peer[k] + k] = r;                                                                      \
@@ -1181,7 +1237,7 @@ static int algo_slice_##SUFFIX(const orc_topo *tp, int c, int variant, int64_t s
         for (int p = 0; p < n; ++p) {                                                                           \
             int r0 = from[2 * p], r1 = from[2 * p + 1];                                                         \
             if (variant == ORC_LATENCY) memset(set, 1, (size_t)n);                                              \
-            else if (tp->algo == ORC_BUCKET) { memset(set, 0, (size_t)n); set[(((p - sg * (t + 2)) % n) + n) % n] = 1; } \
+            else if (tp->algo == ORC_BUCKET) bucket_message(tp, r0, t, bd, bstep, bearlier, sg, set);  /* what its upstream neighbour passes on */ \
             else send_set(tp, sd, sx, p, t, set);                                                               \
             for (int j = 0; j < n; ++j) if (set[j]) {                                                           \
                 T *own = data + (size_t)p * w + bs[j];                                                          \
@@ -1211,10 +1267,14 @@ static int algo_slice_##SUFFIX(const orc_topo *tp, int c, int variant, int64_t s
             for (int r = 0; r < n; ++r) {                                                                       \
                 int peer[2] = {-1, -1}, dir[2], hops[2];                                                        \
                 int np = tp->algo == ORC_BUCKET ? 1 : send_peers(tp, r, sd[t], sx[t], peer, dir, hops);         \
-                if (tp->algo == ORC_BUCKET) peer[0] = ((r + sg) % n + n) % n;                                   \
+                if (tp->algo == ORC_BUCKET) {                                                                   \
+                    bucket_where(tp, c, S + row, &bd, &bstep, &bearlier);                                       \
+                    peer[0] = shift_rank(tp, r, bd, sg);                                                        \
+                    bucket_message(tp, r, S + row, bd, bstep, bearlier, sg, set);                               \
+                }                                                                                               \
                 for (int k = 0; k < np; ++k)                                                                    \
                     for (int j = 0; j < n; ++j) {                                                               \
-                        int sends = tp->algo == ORC_BUCKET ? (j == (((r - sg * row) % n) + n) % n) : snap[(size_t)r * n + j]; \
+                        int sends = tp->algo == ORC_BUCKET ? set[j] : snap[(size_t)r * n + j];                  \
                         if (!sends) continue;                                                                   \
                         if (have[(size_t)peer[k] * n + j]) { rc = ORC_INTERNAL; goto done; }     /* never twice */ \
                         memcpy(data + (size_t)peer[k] * w + bs[j], wire + (size_t)r * wc + (bs[j] - c0),        \

@@ -108,7 +108,7 @@ trv_status_t trv_plan_step(trv_plan_t plan, int32_t c, int32_t row, int32_t* dim
     if (!plan) return TRV_ERR_INVALID_ARG;
     const Plan& p = plan->plan;
     if (c < 0 || c >= p.nslices || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
-    const Step& s = p.steps[c][p.algo == TRV_ALGO_BUCKET ? 0 : p.step_of_row(row)];
+    const Step& s = p.steps[c][p.row_step(c, row)];
     if (dim) *dim = s.dim;
     if (dist) *dist = s.dist;
     return TRV_OK;
@@ -118,7 +118,7 @@ trv_status_t trv_plan_peers(trv_plan_t plan, int32_t c, int32_t row, int32_t* pe
     if (!plan || !peers) return TRV_ERR_INVALID_ARG;
     const Plan& p = plan->plan;
     if (c < 0 || c >= p.nslices || row < 0 || row >= p.rows()) return TRV_ERR_INVALID_ARG;
-    const Step& s = p.steps[c][p.algo == TRV_ALGO_BUCKET ? 0 : p.step_of_row(row)];
+    const Step& s = p.steps[c][p.row_step(c, row)];
     for (int r = 0; r < p.n; ++r) {
         int peer[2], dir[2], hops[2];
         send_peers(p, r, s.dim, s.dist, peer, dir, hops);

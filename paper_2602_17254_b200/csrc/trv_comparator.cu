@@ -67,10 +67,9 @@ trv_status_t run_comparator(const Call& c) {
         if (lhi <= llo) continue;
         std::vector<long long> bs((size_t)n + 1);
         for (int j = 0; j <= n; ++j) bs[j] = clip(block_lo(slo, shi, n, j));
-        const int sg = p.steps[sl][0].dist < 0 ? -1 : 1;        // Bucket: direction of this collective
         for (int t = 0; t < S; ++t) {                           // ---- latency form, or Reduce-Scatter
             if ((st = snapshot(llo, lhi)) != TRV_OK) return st;
-            const Step& step = p.steps[sl][p.algo == TRV_ALGO_BUCKET ? 0 : t];
+            const Step& step = p.steps[sl][t];
             std::fill(from.begin(), from.end(), -1);
             for (int r = 0; r < n; ++r) {
                 int peer[2], dir[2], hops[2];
@@ -105,13 +104,13 @@ trv_status_t run_comparator(const Call& c) {
             const int t = S - 1 - rw;
             if ((st = snapshot(llo, lhi)) != TRV_OK) return st;
             snap = have;
-            const Step& step = p.steps[sl][p.algo == TRV_ALGO_BUCKET ? 0 : t];
+            const Step& step = p.steps[sl][p.algo == TRV_ALGO_BUCKET ? p.bucket_step(sl, S + rw) : t];
             for (int r = 0; r < n; ++r) {
                 int peer[2], dir[2], hops[2];
                 const int np = send_peers(p, r, step.dim, step.dist, peer, dir, hops);
                 for (int k = 0; k < np; ++k)
                     for (int j = 0; j < n; ++j) {
-                        const bool sends = p.algo == TRV_ALGO_BUCKET ? j == ((r - sg * rw) % n + n) % n : snap[(size_t)r * n + j] != 0;
+                        const bool sends = p.algo == TRV_ALGO_BUCKET ? bucket_sends(p, sl, S + rw, r, j) : snap[(size_t)r * n + j] != 0;
                         if (!sends) continue;
                         have[(size_t)peer[k] * n + j] = 1;
                         segs.add(nullptr, wire_of(r, bs[j]), nullptr, out_of(peer[k], bs[j]), (size_t)(bs[j + 1] - bs[j]));

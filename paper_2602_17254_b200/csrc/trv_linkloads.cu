@@ -139,7 +139,7 @@ trv_status_t run_link_loads(const Plan& p, size_t count, size_t elem_size, int32
     int max_rings = 1;
     for (int row = 0; row < T; ++row) {
         for (int c = 0; c < NS; ++c) {
-            const Step& st = p.steps[c][p.algo == TRV_ALGO_BUCKET ? 0 : p.step_of_row(row)];
+            const Step& st = p.steps[c][p.row_step(c, row)];
             RowSlice& rs = desc[(size_t)row * NS + c];
             rs.dim = st.dim; rs.stride = p.stride[st.dim]; rs.size = p.dims[st.dim];
             if (rs.size > kMaxRing) return TRV_ERR_UNSUPPORTED;

@@ -137,13 +137,16 @@ trv_status_t build_plan(const int32_t* dims, int32_t ndims, int variant, int alg
     const int algo = algo_flags & ~(TRV_ALGO_MIRRORED | TRV_ALGO_SINGLE);
     if (algo < TRV_ALGO_TRIVANCE || algo > TRV_ALGO_BUCKET) return TRV_ERR_INVALID_ARG;
     const bool binary = algo == TRV_ALGO_RECDOUB || algo == TRV_ALGO_SWING;
-    if (mirror && (algo == TRV_ALGO_TRIVANCE || (ndims != 1 && !binary))) return TRV_ERR_INVALID_ARG;
+    if (mirror && (algo == TRV_ALGO_TRIVANCE || (ndims != 1 && !binary && algo != TRV_ALGO_BUCKET))) return TRV_ERR_INVALID_ARG;
     if (single && (mirror || !binary)) return TRV_ERR_INVALID_ARG;
     for (int d = 0; d < ndims; ++d)
         if (dims[d] < 2) return TRV_ERR_INVALID_ARG;
     const int base = binary ? 2 : 3;
-    if (algo == TRV_ALGO_BUCKET && ndims != 1) return TRV_ERR_UNSUPPORTED;
-    if (algo == TRV_ALGO_BUCKET && (variant != TRV_BANDWIDTH_OPTIMAL || dims[0] > TRV_MAX_RANKS)) return TRV_ERR_UNSUPPORTED;
+    if (algo == TRV_ALGO_BUCKET) {
+        long long nn = 1;
+        for (int d = 0; d < ndims; ++d) nn *= dims[d];
+        if (variant != TRV_BANDWIDTH_OPTIMAL || nn > TRV_MAX_RANKS) return TRV_ERR_UNSUPPORTED;
+    }
 
     trv_plan_s* holder = new (std::nothrow) trv_plan_s();
     if (!holder) return TRV_ERR_ALLOC;
@@ -151,10 +154,29 @@ trv_status_t build_plan(const int32_t* dims, int32_t ndims, int variant, int alg
     p.algo = algo; p.variant = variant; p.ndims = ndims; p.base = base;
     p.nslices = single ? 1 : ndims * (mirror ? 2 : 1);
     if (algo == TRV_ALGO_BUCKET) {
-        // ring algorithm (Sec. 2.4): n - 1 steps per phase, every step one block to the next node
-        p.dims[0] = dims[0]; p.stride[0] = 1; p.n = dims[0]; p.S = dims[0] - 1;
+        // ring algorithm (Sec. 2.4), dimension after dimension: a_d - 1 steps per phase, every step one message to the
+        // next node of the ring along the phase's dimension
+        int nn = 1;
+        for (int d = 0; d < ndims; ++d) {
+            p.dims[d] = dims[d]; p.stride[d] = nn; nn *= dims[d]; p.S += dims[d] - 1;
+            if (dims[d] != dims[0]) p.equal_dims = false;
+        }
+        p.n = nn;
         p.steps.assign(p.nslices, {});
-        for (int c = 0; c < p.nslices; ++c) p.steps[c].assign(p.S, Step{0, c >= ndims ? -1 : 1});
+        p.bk_step.assign(p.nslices, {}); p.bk_earlier.assign(p.nslices, {}); p.bk_start.assign(p.nslices, {});
+        for (int c = 0; c < p.nslices; ++c) {
+            int earlier = 0;
+            for (int ph = 0; ph < ndims; ++ph) {
+                const int d = (c + ph) % ndims;
+                p.bk_start[c].push_back((int)p.steps[c].size());
+                for (int s = 0; s < dims[d] - 1; ++s) {
+                    p.steps[c].push_back(Step{d, c >= ndims ? -1 : 1});
+                    p.bk_step[c].push_back(s);
+                    p.bk_earlier[c].push_back(earlier);
+                }
+                earlier |= 1 << d;
+            }
+        }
         *out = holder;
         return TRV_OK;
     }
@@ -214,12 +236,22 @@ trv_status_t build_plan(const int32_t* dims, int32_t ndims, int variant, int alg
     return TRV_OK;
 }
 
+// Bucket: is block j in the message node src passes on in `row`?  Reduce-Scatter step s of a phase carries the blocks whose
+// coordinate in the phase's dimension is src's minus (s + 1) (mirrored: plus), AllGather step s those with src's minus s
+// -- the ring rule "block r - t - 1, then block r - t" -- among the blocks that agree with src in the earlier dimensions.
+bool bucket_sends(const Plan& p, int c, int row, int src, int j) {
+    const int t = p.bucket_step(c, row), d = p.steps[c][t].dim, sg = p.steps[c][t].dist, a = p.dims[d];
+    const int off = p.bk_step[c][t] + (row < p.S ? 1 : 0);
+    if (p.coord(j, d) != ((p.coord(src, d) - sg * off) % a + a) % a) return false;
+    for (int q = 0; q < p.ndims; ++q)
+        if (((p.bk_earlier[c][t] >> q) & 1) && p.coord(j, q) != p.coord(src, q)) return false;
+    return true;
+}
+
 bool in_send_set(const Plan& p, int c, int t, int dst, int j) {
     if (p.algo == TRV_ALGO_SWING) return (p.reach[c][t + 1][(size_t)dst * p.words + j / 64] >> (j % 64)) & 1;
-    if (p.algo == TRV_ALGO_BUCKET) {    // step t: node r sends block r - t - 1 on (mirrored: r + t + 1)
-        const int sg = p.steps[c][t].dist, src = ((dst - sg) % p.n + p.n) % p.n;
-        return j == ((src - sg * (t + 1)) % p.n + p.n) % p.n;
-    }
+    if (p.algo == TRV_ALGO_BUCKET)      // what dst's upstream neighbour passes on in Reduce-Scatter step t
+        return bucket_sends(p, c, t, p.shift(dst, p.steps[c][t].dim, -p.steps[c][t].dist), j);
     if (p.algo == TRV_ALGO_RECDOUB && c >= p.ndims) {     // the mirrored collective is the same pattern on the rings read backwards
         int nd = 0, nj = 0;                               // every coordinate x -> (side - x) mod side
         for (int d = 0; d < p.ndims; ++d) {
@@ -301,7 +333,7 @@ void message_bytes_side(const Plan& p, int64_t E, int64_t elem_size, int c, int 
     }
     std::vector<int64_t> tmp((size_t)n);
     message_bytes(p, E, elem_size, c, row, tmp.data());
-    const Step& st = p.steps[c][p.algo == TRV_ALGO_BUCKET ? 0 : p.step_of_row(row)];
+    const Step& st = p.steps[c][p.row_step(c, row)];
     const bool by_source = p.variant == TRV_BANDWIDTH_OPTIMAL && row >= p.S;
     for (int r = 0; r < n; ++r) {
         int peer[2], dir[2], hops[2];
@@ -319,12 +351,14 @@ void message_bytes(const Plan& p, int64_t E, int64_t elem_size, int c, int row, 
     }
     auto blen = [&](int j) { return (block_lo(lo, hi, n, j + 1) - block_lo(lo, hi, n, j)) * elem_size; };
     if (p.algo == TRV_ALGO_BUCKET) {
-        // Reduce-Scatter row t, by destination: the block its upstream neighbour passes on; AllGather row t
-        // (rows run forwards in both phases), by source: block r - t (mirrored: r + t)
-        const int sg = p.steps[c][0].dist;
+        // Reduce-Scatter rows by destination (what its upstream neighbour passes on), AllGather rows by source
+        const Step& st = p.steps[c][p.bucket_step(c, row)];
         for (int r = 0; r < n; ++r) {
-            const int off = row < p.S ? sg * (row + 2) : sg * (row - p.S);
-            out[r] = blen(((r - off) % n + n) % n);
+            const int src = row < p.S ? p.shift(r, st.dim, -st.dist) : r;
+            int64_t sum = 0;
+            for (int j = 0; j < n; ++j)
+                if (bucket_sends(p, c, row, src, j)) sum += blen(j);
+            out[r] = sum;
         }
         return;
     }

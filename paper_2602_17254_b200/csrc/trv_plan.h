@@ -35,6 +35,13 @@ struct Plan {
     std::vector<std::vector<std::vector<uint64_t>>> reach;
     int words = 0;      // 64-bit words per bitset
 
+    // The ring (Bucket) algorithm on a torus (Sec. 2.4): collective c runs a ring Reduce-Scatter of a_d - 1 steps along
+    // dimension c, then along c + 1, ... on the blocks a node still answers for (those that agree with its own coordinates
+    // in the dimensions of the earlier phases); the AllGather takes the phases in reverse order.  steps[c][t] = (dimension,
+    // +1 or -1 for a mirrored collective) of Reduce-Scatter step t; bk_step[c][t] = the step's number inside its phase,
+    // bk_earlier[c][t] = bit mask of the dimensions of the earlier phases, bk_start[c][ph] = first step of phase ph.
+    std::vector<std::vector<int>> bk_step, bk_earlier, bk_start;
+
     // Rings and tori with a side that is no power of three (Sec. 4.4, per dimension as in Sec. 5), bandwidth-optimal
     // form only.  The tree a block follows is the same for every block up to translation, so it is stored once per
     // collective, by the OFFSET o = node - block (coordinate by coordinate, modulo the sides; o is the linear index
@@ -53,6 +60,20 @@ struct Plan {
     int rows() const { return variant == TRV_BANDWIDTH_OPTIMAL ? 2 * S : S; }
     // schedule step behind a row: AllGather rows mirror the Reduce-Scatter steps
     int step_of_row(int row) const { return row < S ? row : 2 * S - 1 - row; }
+    // Bucket: the Reduce-Scatter step with the same dimension, step inside the phase and earlier dimensions as `row`
+    // (AllGather rows walk the phases backwards, the steps of a phase forwards)
+    int bucket_step(int c, int row) const {
+        if (row < S) return row;
+        int i = row - S;
+        for (int ph = ndims - 1; ph >= 0; --ph) {
+            const int len = (ph + 1 < ndims ? bk_start[c][ph + 1] : S) - bk_start[c][ph];
+            if (i < len) return bk_start[c][ph] + i;
+            i -= len;
+        }
+        return 0;
+    }
+    // the schedule step whose (dimension, distance) a row uses
+    int row_step(int c, int row) const { return algo == TRV_ALGO_BUCKET ? bucket_step(c, row) : step_of_row(row); }
     int coord(int r, int d) const { return (r / stride[d]) % dims[d]; }
     int shift(int r, int d, int delta) const {
         int a = dims[d], x = coord(r, d);
@@ -81,6 +102,8 @@ inline int64_t block_lo(int64_t lo, int64_t hi, int n, int j) {
 }
 
 bool in_send_set(const Plan& p, int c, int t, int dst, int j);
+// Bucket: is block j in the message node src passes to its neighbour in `row` (Reduce-Scatter or AllGather)?
+bool bucket_sends(const Plan& p, int c, int row, int src, int j);
 // peers a rank sends to in step (dim, dist); returns how many; dir = +1 / -1, hops = links crossed
 int send_peers(const Plan& p, int r, int dim, int dist, int peer[2], int dir[2], int hops[2]);
 // message bytes of one row, indexed by destination (row < S) or by source (AllGather rows)

@@ -100,6 +100,51 @@ def test_bucket_ring_matches_table_1(n):
         oracle.link_loads([n], LAT, E, 4, algo=oracle.ALGO_BUCKET)
 
 
+@pytest.mark.parametrize("dims", [(3, 3), (4, 4), (8, 8), (5, 5, 5), (4, 4, 4, 4)])
+def test_bucket_on_tori_matches_table_2(dims):
+    """Bucket on an a^D torus with all 2D ports (Sec. 2.4, Table 2): 2D concurrent collectives on 1/(2D) of the vector
+    each, every one in a different direction in every step, so no link ever carries two messages; 2 D (a - 1) steps;
+    phase p of a collective moves messages of m / (2D a^(p+1)) bytes; Theta = Delta = (n - 1)/n -> Table 2's 1
+    against the ideal m beta / D, Lambda = 2 D (a - 1) / log3 n (the table's 2 D n^(1/D) / log3 n counts a for a - 1)."""
+    D, a = len(dims), dims[0]
+    n = a ** D
+    E = 2 * D * n * 3                   # every collective's slice splits into n blocks of 3 elements
+    ll = oracle.link_loads(dims, BW, E, 4, algo=oracle.ALGO_BUCKET | M)
+    S = D * (a - 1)
+    assert ll["msgs"].shape == (2 * S, n, D, 2)
+    assert (ll["msgs"] == 1).all()                              # every link, both directions, exactly one message
+    per_row = [3 * 4 * n // a ** (p + 1) for p in range(D) for _ in range(a - 1)]
+    assert ll["max_bytes"].tolist() == per_row + per_row[::-1]  # the AllGather takes the phases in reverse order
+    assert (ll["bytes"].max(axis=(1, 2, 3)) == ll["bytes"].min(axis=(1, 2, 3))).all()      # all links alike in a row
+    cm = oracle.cost_model(dims, BW, E, 4, 0.0, 1.0, algo=oracle.ALGO_BUCKET | M)
+    assert cm["steps"] == 2 * S
+    assert np.isclose(cm["theta"], (n - 1) / n) and np.isclose(cm["delta"], (n - 1) / n)
+    assert np.isclose(cm["lambda"], 2 * S / (math.log(n) / math.log(3)))
+    # one port per collective only (no mirrored sub-collectives): the + links carry everything
+    one = oracle.link_loads(dims, BW, E, 4, algo=oracle.ALGO_BUCKET)
+    assert (one["msgs"][..., 0] == 1).all() and (one["msgs"][..., 1] == 0).all()
+
+
+def test_bucket_on_a_torus_worked_by_hand():
+    """3 x 2 torus (rank = x0 + 3 x1), collective 0 (dimension 0 first): rows 0, 1 ring Reduce-Scatter along
+    dimension 0 on super-blocks {j : j0 = x0 - s - 1}, row 2 along dimension 1 on the one block with j0 = x0,
+    j1 = x1 - 1; then the AllGather: dimension 1 first, dimension 0 last.  Node 0 = (0, 0)."""
+    E = 2 * 6 * 5
+    ll = oracle.link_loads((3, 2), BW, E, 4, algo=oracle.ALGO_BUCKET)
+    b = ll["bytes"]                     # [row][node][dimension][direction]
+    # collective 0 uses, in row order, dimensions 0 0 1 | 1 0 0 with 2, 2, 1 | 1, 2, 2 blocks of 20 bytes per message;
+    # collective 1 dimensions 1 0 0 | 0 0 1 with 3, 1, 1 | 1, 1, 3 blocks: with unequal sides they meet on a link (rows 1, 4)
+    assert b[:, 0, 0, 0].tolist() == [40, 60, 20, 20, 60, 40] and b[:, 0, 1, 0].tolist() == [60, 0, 20, 20, 0, 60]
+    assert ll["msgs"][:, 0, 0, 0].tolist() == [1, 2, 1, 1, 2, 1] and (ll["msgs"][..., 1] == 0).all()
+    x = np.zeros((6, E), np.int32)
+    for r in range(6):
+        x[r] = 10 ** r
+    y, ctr = oracle.allreduce_algo((3, 2), BW, x, oracle.ALGO_BUCKET, counters=True)
+    assert (y == 111111).all()
+    # per collective a node sends 2 x (2 blocks) + 1 block in the Reduce-Scatter: 5 of 6 blocks
+    assert (ctr["sent_rs"] == 2 * 5 * 20).all() and (ctr["sent_ag"] == 2 * 5 * 20).all()
+
+
 @pytest.mark.parametrize("n", [8, 64, 256])
 def test_recursive_doubling_mirrored(n):
     """Both ports through a mirrored collective (Sec. 2.4): the bytes per node halve per collective
@@ -121,7 +166,8 @@ def test_recursive_doubling_mirrored(n):
 # ------------------------------------------------------------------ the library's host-side tables
 
 CASES = [((8,), oracle.ALGO_SWING), ((64,), oracle.ALGO_SWING), ((64,), oracle.ALGO_SWING | M), ((16,), oracle.ALGO_RECDOUB | M),
-         ((27,), oracle.ALGO_BRUCK | M), ((9,), oracle.ALGO_BUCKET), ((10,), oracle.ALGO_BUCKET | M)]
+         ((27,), oracle.ALGO_BRUCK | M), ((9,), oracle.ALGO_BUCKET), ((10,), oracle.ALGO_BUCKET | M),
+         ((4, 4), oracle.ALGO_BUCKET | M), ((3, 5), oracle.ALGO_BUCKET), ((2, 3, 4), oracle.ALGO_BUCKET | M)]
 
 
 @pytest.mark.parametrize("dims,algo", CASES)
@@ -135,7 +181,7 @@ def test_plan_tables_match_oracle(dims, algo, variant):
         return
     plan = binding.Plan(dims, variant, algo)
     n = plan.n
-    assert plan.nslices == (2 if algo & M else 1)
+    assert plan.nslices == len(dims) * (2 if algo & M else 1)
     E = 37 * n + 5
     sent = np.zeros(n, np.int64)
     for c in range(plan.nslices):
@@ -190,6 +236,28 @@ def test_comparator_paths_give_the_column_sums_and_the_modelled_bytes(algo, size
             assert np.array_equal(ctr["sent_rs"] + ctr["sent_ag"], oracle.bytes_sent((n,), variant, E, 4, algo | mirror))
             part = oracle.allreduce_algo((n,), variant, np.ascontiguousarray(x[:, 2:E - 3]), algo | mirror, E=E, e0=2)
             assert np.array_equal(part, y[:, 2:E - 3])          # a window gives the full run's columns
+
+
+@pytest.mark.parametrize("dims", [(3, 3), (4, 4), (3, 5), (2, 3, 4), (5, 5, 5)])
+@pytest.mark.parametrize("mirror", [0, oracle.ALGO_MIRROR])
+def test_bucket_path_on_tori(dims, mirror):
+    """Bucket dimension after dimension (Sec. 2.4): every rank ends with the column sums, the bytes on the wire are the
+    modelled ones -- (n - 1)/n of a collective's slice per node and phase direction -- and a window of the vector gives
+    the full run's columns."""
+    n = int(np.prod(dims))
+    E = 7 * n + 3
+    x = np.random.default_rng(n).integers(-2 ** 31, 2 ** 31 - 1, size=(n, E), dtype=np.int64).astype(np.int32)
+    y, ctr = oracle.allreduce_algo(dims, 1, x, oracle.ALGO_BUCKET | mirror, counters=True)
+    assert (y == x.astype(np.int64).sum(0).astype(np.int32)[None]).all()
+    assert np.array_equal(ctr["sent_rs"] + ctr["sent_ag"], oracle.bytes_sent(dims, 1, E, 4, oracle.ALGO_BUCKET | mirror))
+    if E % (n * len(dims) * (2 if mirror else 1)) == 0:
+        assert (ctr["sent_rs"] == 4 * E * (n - 1) // n).all()
+    part = oracle.allreduce_algo(dims, 1, np.ascontiguousarray(x[:, 2:E - 3]), oracle.ALGO_BUCKET | mirror, E=E, e0=2)
+    assert np.array_equal(part, y[:, 2:E - 3])
+    xf = np.random.default_rng(n + 1).standard_normal((n, E)).astype(np.float32)
+    yf = oracle.allreduce_algo(dims, 1, xf, oracle.ALGO_BUCKET | mirror)
+    assert (yf == yf[0][None]).all()                            # one reduction order per block: every rank gets the same bits
+    assert np.abs(yf[0].astype(np.float64) - xf.astype(np.float64).sum(0)).max() <= 2e-6 * np.abs(xf).sum(0).max()
 
 
 @pytest.mark.parametrize("dims", [(9,), (27,), (3, 3), (9, 9), (3, 9), (3, 3, 3)])

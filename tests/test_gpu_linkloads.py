@@ -94,7 +94,8 @@ M = binding.ALGO_MIRRORED
 NEW = [((8,), binding.ALGO_SWING), ((64,), binding.ALGO_SWING), ((1024,), binding.ALGO_SWING), ((64,), binding.ALGO_SWING | M),
        ((256,), binding.ALGO_SWING | M), ((16,), binding.ALGO_RECDOUB | M), ((512,), binding.ALGO_RECDOUB | M),
        ((27,), binding.ALGO_BRUCK | M), ((9,), binding.ALGO_BUCKET), ((10,), binding.ALGO_BUCKET | M),
-       ((100,), binding.ALGO_BUCKET | M), ((2,), binding.ALGO_BUCKET | M)]
+       ((100,), binding.ALGO_BUCKET | M), ((2,), binding.ALGO_BUCKET | M),
+       ((4, 4), binding.ALGO_BUCKET | M), ((3, 5), binding.ALGO_BUCKET), ((2, 3, 4), binding.ALGO_BUCKET | M), ((8, 8, 8), binding.ALGO_BUCKET | M)]
 
 
 @pytest.mark.parametrize("dims,algo", NEW)
