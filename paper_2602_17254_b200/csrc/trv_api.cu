@@ -16,6 +16,12 @@ static bool fused_supported(const Plan& p) {
     return p.variant == TRV_LATENCY_OPTIMAL ? fused_latency_supported(p) : fused_bandwidth_supported(p);
 }
 
+void prepare_launch_data(Plan& p) {
+    if (p.algo != TRV_ALGO_TRIVANCE) return;
+    if (p.general) tree_prepare(p);
+    else if (p.variant == TRV_LATENCY_OPTIMAL) latency_prepare(p);
+}
+
 static trv_status_t check_buffers(const Plan& p, const void* const* in, void* const* out, size_t count, bool* in_place) {
     if (!in || !out) return TRV_ERR_INVALID_ARG;
     const int n = p.n;
@@ -27,6 +33,21 @@ static trv_status_t check_buffers(const Plan& p, const void* const* in, void* co
     }
     // pairwise disjoint outputs; inputs either identical to the outputs or disjoint from all of them
     const size_t bytes = count * 4;
+    {   // the usual case needs no sorting: equally spaced rows (of one tensor) are disjoint as soon as the spacing holds a
+        // row, and two such families either are the same or must not touch (243 ranks: 3 us of a 9 us call otherwise)
+        StrideAddr so, si;
+        if (n > 1 && uniform_stride((const void* const*)out, n, &so) && so.stride >= bytes &&
+            (same || (uniform_stride(in, n, &si) && si.stride >= bytes))) {
+            if (!same) {
+                const uintptr_t o0 = (uintptr_t)so.base, o1 = o0 + (uintptr_t)so.stride * (n - 1) + bytes;
+                const uintptr_t i0 = (uintptr_t)si.base, i1 = i0 + (uintptr_t)si.stride * (n - 1) + bytes;
+                if (i0 < o1 && o0 < i1) goto sorted_check;      // the two spans meet: let the general check decide
+            }
+            *in_place = same;
+            return TRV_OK;
+        }
+    }
+sorted_check:
     std::vector<std::pair<uintptr_t, int>> iv;
     iv.reserve(2 * (size_t)n);
     for (int r = 0; r < n; ++r) iv.emplace_back((uintptr_t)out[r], 1);
@@ -79,7 +100,9 @@ trv_status_t trv_plan_create_algo(const int32_t* dims, int32_t ndims, trv_varian
                                   trv_plan_t* out) {
     if (!out) return TRV_ERR_INVALID_ARG;
     *out = nullptr;
-    return build_plan(dims, ndims, (int)variant, (int)algo, out);
+    const trv_status_t st = build_plan(dims, ndims, (int)variant, (int)algo, out);
+    if (st == TRV_OK) prepare_launch_data((*out)->plan);
+    return st;
 }
 
 trv_status_t trv_plan_destroy(trv_plan_t plan) {

@@ -232,6 +232,8 @@ trv_status_t run_fused_latency(const Call& c);
 trv_status_t run_fused_bandwidth(const Call& c);
 // rings of any other size (trv_fused_tree.cu)
 bool fused_tree_supported(const Plan& p);
+void tree_prepare(Plan& p);         // once per plan: the stack-machine programs
+void latency_prepare(Plan& p);      // once per plan: which latency kernel, and the line-group program if that is the one
 trv_status_t run_fused_tree(const Call& c);
 
 // chunk-level readiness engine (trv_pipe.cu)

@@ -142,6 +142,7 @@ __global__ void __launch_bounds__(9 * TILE / V, M == 27 ? (TILE == 64 ? 3 : 4) :
 enum class LatKind { None, Reg, Ring, T999, Lines };
 
 static LatKind classify(const Plan& p) {
+    if (p.lat_kind >= 0) return (LatKind)p.lat_kind;        // decided when the plan was created
     if (p.algo != TRV_ALGO_TRIVANCE || p.variant != TRV_LATENCY_OPTIMAL) return LatKind::None;
     if (p.equal_dims) {
         if (p.n <= 81 && p.ndims <= 4) return LatKind::Reg;
@@ -152,6 +153,14 @@ static LatKind classify(const Plan& p) {
 }
 
 bool fused_latency_supported(const Plan& p) { return classify(p) != LatKind::None; }
+
+// once per plan (prepare_launch_data)
+void latency_prepare(Plan& p) {
+    p.lat_kind = -1;
+    const LatKind k = classify(p);
+    if (k == LatKind::Lines) lines_prepare(p);
+    p.lat_kind = (int)k;
+}
 
 static void fill_args(const Call& c, LatArgs* a) {
     const Plan& p = *c.plan;

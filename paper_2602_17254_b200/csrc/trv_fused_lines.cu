@@ -229,6 +229,7 @@ static trv_status_t launch_lines_cg(const Call& c, const Addr& in, const Addr& o
 static bool build_program(const Plan& p, LnProgram* prog);
 
 bool fused_lines_supported(const Plan& p) {
+    if (p.lines_prog) return true;
     if (p.general || p.algo != TRV_ALGO_TRIVANCE || p.variant != TRV_LATENCY_OPTIMAL) return false;
     if (p.n > 729 || p.ndims > kLnMaxD) return false;
     for (int d = 0; d < p.ndims; ++d)
@@ -327,11 +328,18 @@ template trv_status_t launch_lines_part<uint32_t, 1>(const Call&, const LatArgs&
 #endif  // TRV_LN_PART > 0
 
 #if TRV_LN_PART == 0
+// once per plan (prepare_launch_data): the group list and the base ranks of all sets
+void lines_prepare(Plan& p) {
+    p.lines_prog.reset();
+    if (!fused_lines_supported(p)) return;
+    auto prog = std::make_shared<LnProgram>();
+    if (build_program(p, prog.get())) p.lines_prog = prog;
+}
+
 trv_status_t run_fused_lines(const Call& c, const LatArgs& a) {
     const Plan& p = *c.plan;
-    if (!fused_lines_supported(p)) return TRV_ERR_UNSUPPORTED;
-    static thread_local LnProgram prog;       // 13 KB: kept off the stack
-    if (!build_program(p, &prog)) return TRV_ERR_UNSUPPORTED;
+    if (!p.lines_prog) return TRV_ERR_UNSUPPORTED;
+    const LnProgram& prog = *static_cast<const LnProgram*>(p.lines_prog.get());
     trv_status_t st;
     if (c.dtype == TRV_FLOAT32) st = prog.cg == 9 ? launch_lines_part<float, 9>(c, a, prog) : launch_lines_part<float, 1>(c, a, prog);
     else st = prog.cg == 9 ? launch_lines_part<uint32_t, 9>(c, a, prog) : launch_lines_part<uint32_t, 1>(c, a, prog);

@@ -278,18 +278,29 @@ static trv_status_t tree_by_cap(const Call& c, const std::vector<std::vector<uns
 }
 
 bool fused_tree_supported(const Plan& p) {
+    if (p.tree_ready) return true;
     return p.general && p.n <= TRV_MAX_RANKS && p.nslices <= kTreeMaxSlices && p.ndims <= 4 && p.S + 2 <= kTreeDepth;
 }
 
-trv_status_t run_fused_tree(const Call& c) {
-    const Plan& p = *c.plan;
-    if (!fused_tree_supported(p)) return TRV_ERR_UNSUPPORTED;
+// once per plan (prepare_launch_data): the depth-first programs of all collectives
+void tree_prepare(Plan& p) {
+    p.tree_ready = false;
+    p.tree_progs.clear();
+    if (!fused_tree_supported(p)) return;
     std::vector<std::vector<unsigned short>> progs(p.nslices);
     for (int sl = 0; sl < p.nslices; ++sl) {
         progs[sl].reserve(p.n);
         const int depth = build_program(p, sl, progs[sl]);
-        if ((int)progs[sl].size() != p.n || depth > kTreeDepth) return TRV_ERR_UNSUPPORTED;
+        if ((int)progs[sl].size() != p.n || depth > kTreeDepth) return;
     }
+    p.tree_progs.swap(progs);
+    p.tree_ready = true;
+}
+
+trv_status_t run_fused_tree(const Call& c) {
+    const Plan& p = *c.plan;
+    if (!p.tree_ready) return TRV_ERR_UNSUPPORTED;
+    const std::vector<std::vector<unsigned short>>& progs = p.tree_progs;
     // two columns per thread when blocks are long (few threads straddle a block boundary) and the
     // vector is long enough to fill the GPU with such threads.  Measured on B200 at 8 MiB per rank:
     // four columns per thread are slower from 53 ranks up (0.82 against 0.89 of the copy bandwidth

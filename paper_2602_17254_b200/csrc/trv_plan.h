@@ -3,6 +3,7 @@
 #include <cstddef>
 #include <cstdint>
 #include <mutex>
+#include <memory>
 #include <vector>
 
 #include "../../include/trivance.h"
@@ -50,6 +51,15 @@ struct Plan {
     // after it, -1 if to the node `dist` before it.
     bool general = false;
     std::vector<std::vector<int8_t>> gstep, gsgn;
+
+    // Host data that the fused launchers derive from the schedule alone, built ONCE by prepare_launch_data() when the plan
+    // is created and read-only afterwards (a call writes nothing into the plan): which latency kernel serves the shape
+    // (-1: not classified), the line-group kernel's program, the block-tree programs of the stack-machine kernel.
+    // Rebuilding them in every call cost 94 us per call on a 27 x 27 torus and 178 us on 32 x 32.
+    int lat_kind = -1;
+    std::shared_ptr<const void> lines_prog;                     // LnProgram (trv_fused_lines.cu), or empty
+    std::vector<std::vector<unsigned short>> tree_progs;        // one per collective (trv_fused_tree.cu), or empty
+    bool tree_ready = false;
 
     // plan-owned scratch for trv_allreduce (STEP family of the latency form), grown on demand under
     // trv_plan_s::scratch_mu; scratch_device = ordinal of the GPU it was allocated on (-1: none yet)
@@ -125,4 +135,5 @@ struct trv_plan_s {
 
 namespace trv {
 trv_status_t build_plan(const int32_t* dims, int32_t ndims, int variant, int algo, trv_plan_s** out);
+void prepare_launch_data(Plan& p);      // trv_api.cu: fills lat_kind, lines_prog, tree_progs
 }
