@@ -226,7 +226,7 @@ trv_status_t trv_allreduce_ex(trv_plan_t plan, const void *const *in_buffers, vo
  *                 Pinned memory is needed for the copies to overlap; equally spaced rows (rows of one matrix)
  *                 are moved by one 2-D copy per window and direction instead of n copies.
  *   workspace   : DEVICE pointer, 256-byte aligned.  trv_host_workspace_bytes(...) is the size for the preferred
- *                 window (an eighth of the vector, between 64 KiB per rank and 128 MiB over all ranks); a smaller
+ *                 window (an eighth of the vector, between 64 KiB per rank and 512 MiB over all ranks); a smaller
  *                 workspace is accepted and gives shorter windows; SCRATCH if not even windows of 64 elements fit.
  * Uploads and downloads run on two internal streams that the library creates on the first call on a device (make
  * that call outside any stream capture); kernels run on `cuda_stream`.  The internal streams wait for the work
