@@ -242,6 +242,7 @@ static trv_status_t lat_fused_launch(const Call& c, const Addr& in, const Addr& 
     } else if (kind == LatKind::Lines) {
         trv_status_t st = TRV_OK;
         if (run_fused_t2727_wide(c, a, &st)) return st;       // 27 x 27, long vectors, equally spaced rank buffers
+        if (run_fused_t981_wide(c, a, &st)) return st;        // 9 x 81, likewise
         g_last_kernel = "lat_lines";
         return run_fused_lines(c, a);
     } else {

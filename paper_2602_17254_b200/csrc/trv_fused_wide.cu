@@ -191,6 +191,9 @@ __device__ __forceinline__ void wide_wait_plane(unsigned long long* bars, int k,
 
 struct ShapeT999 {
     static constexpr int kSlices = 3;
+    static bool encode(const StrideAddr& base, size_t count, const LatArgs& a, int sl, CUtensorMap* out) {
+        return encode_planes(base, count, a.rs[sl], kWideCols, out);
+    }
     __device__ static __forceinline__ void fetch(const PlaneMaps& maps, int c, long long t0, int k, unsigned slab_s,
                                                  unsigned long long* bars) {
         wide_fetch_plane(maps, c, t0, k, slab_s, bars);
@@ -320,8 +323,10 @@ __device__ __forceinline__ bool wide_tile_2727(const PlaneMaps& maps, const Stri
     return true;
 }
 
+static bool encode_planes_2727(const StrideAddr& base, size_t count, int slice, CUtensorMap* out);
 struct Shape2727 {
     static constexpr int kSlices = 2;
+    static bool encode(const StrideAddr& base, size_t count, const LatArgs&, int sl, CUtensorMap* out) { return encode_planes_2727(base, count, sl, out); }
     __device__ static __forceinline__ void fetch(const PlaneMaps& maps, int c, long long t0, int k, unsigned slab_s,
                                                  unsigned long long* bars) {
         wide_fetch_plane_2727(maps, c, t0, k, slab_s, bars);
@@ -335,6 +340,181 @@ struct Shape2727 {
                         : wide_tile_2727<T, 3, false>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up);
         return full ? wide_tile_2727<T, 1, true>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up)
                     : wide_tile_2727<T, 1, false>(maps, out, a, c, t0, parity, has_next, nc, nt0, slab, bars, gave_up);
+    }
+};
+
+// ------------------------------------------------------------------ 9 x 81 and 81 x 9
+//
+// 9 x 81: rank = A + 9 B with A < 9, B < 81; write B = Bl + 9 Bh: the ranks form a 9 x 9 x 9 index space (A, Bl, Bh) with
+// rank strides 1, 9, 81, and plane k = the ranks with Bl = k lands as [Bh][A] (row Bh * 9 + A: PA = 1).  81 x 9: rank =
+// B + 81 A, strides 81, 1, 9, the plane lands as [A][Bh] (PA = 9).  The slice that starts with the side of 9 runs the steps
+// A1 B1 A3 B3 B9 B27, the other one B1 A1 B3 A3 B9 B27 (Sec. 5).  Steps along B with distance 1 or 3 walk a ring of 81 or 27
+// positions that crosses the planes: they are streamed as three-point stencils, nine positions at a time, in place.
+// Groups: (A,1) on the 9-rank A-lines of a plane; (B,1) on the nine B-lines; (A,3)(B,3) on the nine sets
+// {A = a0 + 3 i, B = b0 + 3 j}, streamed along j; (B,9)(B,27) on the 9-rank sets {A, Bl fixed}, which lie inside ONE plane:
+// three phases of three planes each, as the refill wants them.
+template <bool SWAP>
+__device__ __forceinline__ void wide_fetch_plane_981(const PlaneMaps& maps, long long t0, int k, unsigned slab_s, unsigned long long* bars) {
+    const unsigned bar_s = smem_u32(bars + k);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s), "r"(kWidePlaneBytes) : "memory");
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(
+            slab_s + k * kWidePlaneBytes),
+        "l"(&maps.in[0]), "r"((int)t0), "r"(SWAP ? k : 0), "r"(SWAP ? 0 : k), "r"(0), "r"(bar_s)
+        : "memory");
+}
+
+// One distance-1 step on a ring of L positions (L a multiple of 9), each position a row of W values, in place:
+// out[i] = (row[i - 1] + row[i]) + row[i + 1] where row[i] = what load(i, .) delivers (the stored values BEFORE this step,
+// possibly with a step of their own applied), handed to store(i, .).  Nine positions at a time: position i is stored
+// only after positions up to i + 1 have been loaded, and positions 0 and 1 are kept for the wrap-around.
+template <int L, int W, typename E, typename Load, typename Store>
+__device__ __forceinline__ void wide_ring_stencil(Load load, Store store) {
+    E first[W], second[W], a[W], b[W];
+    load(0, first);
+    load(1, second);
+#pragma unroll
+    for (int w = 0; w < W; ++w) { a[w] = first[w]; b[w] = second[w]; }
+#pragma unroll
+    for (int k = 0; k < L / 9; ++k) {
+        E x[11][W];
+#pragma unroll
+        for (int w = 0; w < W; ++w) { x[0][w] = a[w]; x[1][w] = b[w]; }
+#pragma unroll
+        for (int m = 0; m < 9; ++m) {
+            const int i = 9 * k + 2 + m;
+            if (i < L) load(i, x[2 + m]);
+            else {
+#pragma unroll
+                for (int w = 0; w < W; ++w) x[2 + m][w] = i == L ? first[w] : second[w];
+            }
+        }
+#pragma unroll
+        for (int m = 0; m < 9; ++m) {
+            E o[W];
+#pragma unroll
+            for (int w = 0; w < W; ++w) o[w] = add3(x[m][w], x[m + 1][w], x[m + 2][w]);
+            store((9 * k + 1 + m) % L, o);
+        }
+#pragma unroll
+        for (int w = 0; w < W; ++w) { a[w] = x[9][w]; b[w] = x[10][w]; }
+    }
+}
+
+// BFIRST = false: the slice A1 B1 A3 B3 B9 B27; true: B1 A1 B3 A3 B9 B27.  PA = 1: 9 x 81, PA = 9: 81 x 9.
+template <typename T, int PA, bool BFIRST, bool FULL>
+__device__ __forceinline__ bool wide_tile_981(const PlaneMaps& maps, const StrideAddr& out, const LatArgs& a, int c, long long t0,
+                                              unsigned parity, bool has_next, long long nt0, T* slab, unsigned long long* bars,
+                                              int* gave_up) {
+    constexpr int PK = 81, PH = PA == 1 ? 9 : 1;        // row of (A, B) in the slab: (B % 9) * PK + (B / 9) * PH + A * PA
+    using E = Elem<T, 2>;
+    const int lane = threadIdx.x % 32, set = threadIdx.x / 32;
+    const long long lo = a.lo[c], hi = a.hi[c];
+    const long long e = t0 + 2 * lane;
+    E* const mine = reinterpret_cast<E*>(slab) + lane;
+    auto sl = [&](int r) -> E& { return mine[r * (kWideCols / 2)]; };
+    auto a_lines = [&]() {              // (A,1) on the nine A-lines of the plane `set`
+#pragma unroll 3
+        for (int h = 0; h < 9; ++h) {
+            E v[9];
+#pragma unroll
+            for (int i = 0; i < 9; ++i) v[i] = sl(set * PK + h * PH + i * PA);
+            reg_step<9, 1, 9, 1>(v);
+#pragma unroll
+            for (int i = 0; i < 9; ++i) sl(set * PK + h * PH + i * PA) = v[i];
+        }
+    };
+    auto b_lines = [&]() {              // (B,1) on the B-line A = set: a ring of 81 positions across the planes
+        wide_ring_stencil<81, 1, E>([&](int i, E (&row)[1]) { row[0] = sl((i % 9) * PK + (i / 9) * PH + set * PA); },
+                                    [&](int i, const E (&row)[1]) { sl((i % 9) * PK + (i / 9) * PH + set * PA) = row[0]; });
+    };
+    if (!BFIRST) {
+        wide_wait_plane(bars, set, parity, gave_up);
+        a_lines();
+        __syncthreads();
+        if (*gave_up) return false;
+        b_lines();
+    } else {
+#pragma unroll 1
+        for (int k = 0; k < 9; ++k) wide_wait_plane(bars, k, parity, gave_up);     // a B-line crosses every plane
+        __syncthreads();
+        if (*gave_up) return false;
+        b_lines();
+        __syncthreads();
+        a_lines();
+    }
+    __syncthreads();
+    {   // ---- (A,3) (B,3), or (B,3) (A,3), on the set {A = a0 + 3 i, B = b0 + 3 j}: rows of three values, ring of 27 rows
+        const int a0 = set % 3, b0 = set / 3;
+        auto row_at = [&](int j) { return (b0 + 3 * (j % 3)) * PK + (j / 3) * PH + a0 * PA; };       // B = b0 + 3 j
+        wide_ring_stencil<27, 3, E>(
+            [&](int j, E (&row)[3]) {
+#pragma unroll
+                for (int i = 0; i < 3; ++i) row[i] = sl(row_at(j) + 3 * i * PA);
+                if (!BFIRST) reg_step<3, 1, 3, 1>(row);        // (A,3) comes before (B,3)
+            },
+            [&](int j, const E (&row)[3]) {
+                E o[3];
+#pragma unroll
+                for (int i = 0; i < 3; ++i) o[i] = row[i];
+                if (BFIRST) reg_step<3, 1, 3, 1>(o);           // (A,3) comes after (B,3)
+#pragma unroll
+                for (int i = 0; i < 3; ++i) sl(row_at(j) + 3 * i * PA) = o[i];
+            });
+    }
+    __syncthreads();
+    // ---- (B,9) (B,27) on the sets {A, Bl fixed, Bh = 0 .. 8}: inside the plane Bl; phase k0 takes the planes k0, k0 + 3, k0 + 6
+    const int sA = a.rs[c][BFIRST ? 1 : 0], sB = a.rs[c][BFIRST ? 0 : 1];       // rank strides of the side of 9 and of the side of 81
+    const unsigned slab_s = smem_u32(slab);
+#pragma unroll 1
+    for (int k0 = 0; k0 < 3; ++k0) {
+        E v[3][9];
+#pragma unroll
+        for (int m = 0; m < 3; ++m) {
+            const int q = set + 9 * m, r0 = (k0 + 3 * (q / 9)) * PK + (q % 9) * PA;     // A = q % 9, Bl = k0 + 3 (q / 9)
+#pragma unroll
+            for (int idx = 0; idx < 9; ++idx) v[m][idx] = sl(r0 + PH * idx);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // this thread's slab accesses before the engine's writes
+        __syncthreads();                    // everybody holds its part of the planes k0, k0 + 3, k0 + 6: they may be refilled
+        if (threadIdx.x == 0 && has_next) {
+            for (int kk = 0; kk < 3; ++kk) wide_fetch_plane_981<PA == 9>(maps, nt0, k0 + 3 * kk, slab_s, bars);
+        }
+#pragma unroll
+        for (int m = 0; m < 3; ++m) {
+            const int q = set + 9 * m, g0 = (q % 9) * sA + (k0 + 3 * (q / 9)) * sB;
+            reg_step<9, 1, 9, 1>(v[m]);     // (B,9): distance 1 in Bh
+            reg_step<9, 1, 9, 3>(v[m]);     // (B,27): distance 3 in Bh
+            if (FULL || (e < hi && e + 2 > lo)) {
+#pragma unroll
+                for (int idx = 0; idx < 9; ++idx) store_elem<T, 2, FULL>(out.ptr(g0 + 9 * idx * sB), e, lo, hi, v[m][idx]);
+            }
+        }
+    }
+    return true;
+}
+
+template <bool SWAP>          // false: 9 x 81, true: 81 x 9
+struct Shape981 {
+    static constexpr int kSlices = 2;
+    static bool encode(const StrideAddr& base, size_t count, const LatArgs&, int, CUtensorMap* out) {
+        const int s981[3] = {1, 81, 9}, s819[3] = {81, 9, 1};       // A, Bh, and Bl in the place of the plane coordinate
+        return encode_planes(base, count, SWAP ? s819 : s981, kWideCols, out);
+    }
+    __device__ static __forceinline__ void fetch(const PlaneMaps& maps, int c, long long t0, int k, unsigned slab_s,
+                                                 unsigned long long* bars) {
+        wide_fetch_plane_981<SWAP>(maps, t0, k, slab_s, bars);  // both slices read the same map
+    }
+    template <typename T>
+    __device__ static __forceinline__ bool tile(const PlaneMaps& maps, const StrideAddr& out, const LatArgs& a, int c, long long t0,
+                                                bool full, unsigned parity, bool has_next, int nc, long long nt0, T* slab,
+                                                unsigned long long* bars, int* gave_up) {
+        constexpr int PA = SWAP ? 9 : 1;
+        if ((c == 1) != SWAP)           // the slice that starts with the side of 81
+            return full ? wide_tile_981<T, PA, true, true>(maps, out, a, c, t0, parity, has_next, nt0, slab, bars, gave_up)
+                        : wide_tile_981<T, PA, true, false>(maps, out, a, c, t0, parity, has_next, nt0, slab, bars, gave_up);
+        return full ? wide_tile_981<T, PA, false, true>(maps, out, a, c, t0, parity, has_next, nt0, slab, bars, gave_up)
+                    : wide_tile_981<T, PA, false, false>(maps, out, a, c, t0, parity, has_next, nt0, slab, bars, gave_up);
     }
 };
 
@@ -420,10 +600,6 @@ static WideSched* wide_sched_for(int dev, cudaStream_t st) {
     return d.base + it->second;
 }
 
-// Tensor map of one slice of the 27 x 27 torus over equally spaced rank buffers: dimensions (column, then the two torus
-// dimensions by increasing rank stride), boxes of 64 columns x 27 along the slice's own dimension x 3 along the other.
-static bool encode_planes_2727(const StrideAddr& base, size_t count, int slice, CUtensorMap* out);
-
 // false: this call cannot use the wide kernel (the caller goes on to the 32-column kernels)
 template <typename Shape>
 static bool run_wide(const Call& c, const LatArgs& a, const char* name, trv_status_t* status) {
@@ -453,8 +629,7 @@ static bool run_wide(const Call& c, const LatArgs& a, const char* name, trv_stat
     if (!giveups) return false;
     PlaneMaps maps;
     for (int sl = 0; sl < NS; ++sl) {
-        const bool ok = NS == 3 ? encode_planes(sin, c.count, a.rs[sl], kWideCols, &maps.in[sl]) : encode_planes_2727(sin, c.count, sl, &maps.in[sl]);
-        if (!ok) return false;
+        if (!Shape::encode(sin, c.count, a, sl, &maps.in[sl])) return false;
     }
     *status = TRV_OK;
     constexpr int smem = (int)kWideTileBytes + 9 * 8 + 16 + 24;
@@ -481,6 +656,17 @@ bool run_fused_t2727_wide(const Call& c, const LatArgs& a, trv_status_t* status)
     return run_wide<Shape2727>(c, a, "lat_t27x27_wide", status);
 }
 
+// 9 x 81 (rank = x0 + 9 x1) and 81 x 9 (rank = x0 + 81 x1); false: not these shapes or not this call
+bool run_fused_t981_wide(const Call& c, const LatArgs& a, trv_status_t* status) {
+    const Plan& p = *c.plan;
+    if (p.ndims != 2 || p.stride[0] != 1) return false;
+    if (p.dims[0] == 9 && p.dims[1] == 81 && p.stride[1] == 9) return run_wide<Shape981<false>>(c, a, "lat_t9x81_wide", status);
+    if (p.dims[0] == 81 && p.dims[1] == 9 && p.stride[1] == 81) return run_wide<Shape981<true>>(c, a, "lat_t81x9_wide", status);
+    return false;
+}
+
+// Tensor map of one slice of the 27 x 27 torus over equally spaced rank buffers: dimensions (column, then the two torus
+// dimensions by increasing rank stride), boxes of 64 columns x 27 along the slice's own dimension x 3 along the other.
 static bool encode_planes_2727(const StrideAddr& base, size_t count, int slice, CUtensorMap* out) {
     if ((base.stride & 15) || ((uintptr_t)base.base & 15) || count == 0 || count >= ((size_t)1 << 31)) return false;
     if ((size_t)base.stride < count * 4) return false;

@@ -124,6 +124,20 @@ def test_fused_latency_27x27_tiles_of_64_columns():
     assert binding.tma_giveups() == 0
 
 
+def test_fused_latency_9x81_tiles_of_64_columns():
+    """9 x 81 and 81 x 9: the persistent 64-column kernel with steps along the side of 81 streamed as ring stencils across the
+    planes; both slices (A1 B1 A3 B3 B9 B27 and B1 A1 B3 A3 B9 B27), ragged edges, both dtypes, in place and not."""
+    check_case((9, 81), LAT, 70001, "normal", 61, FUSED)
+    assert binding.last_kernel_name() == "lat_t9x81_wide"
+    check_case((9, 81), LAT, 300034, "int32", 62, FUSED, in_place=False)
+    assert binding.last_kernel_name() == "lat_t9x81_wide"
+    check_case((81, 9), LAT, 70001, "int32", 63, FUSED)
+    assert binding.last_kernel_name() == "lat_t81x9_wide"
+    check_case((81, 9), LAT, 200002, "normal", 64, FUSED, in_place=False)
+    assert binding.last_kernel_name() == "lat_t81x9_wide"
+    assert binding.tma_giveups() == 0
+
+
 def test_fused_bandwidth_wide_path_on_729_ranks_sampled():
     """9x9x9 with blocks of >= 256 elements: the oracle checks windows around slice and block
     boundaries and in block interiors."""
