@@ -318,6 +318,52 @@ def test_plan_scratch_grows_safely_under_concurrent_host_threads():
     plan.destroy()
 
 
+def test_wide_kernels_on_several_streams_and_threads_at_once():
+    """The persistent 64-column kernels draw their tiles from a counter that belongs to the (device, stream) pair.  Three
+    host threads, each with a stream of its own, run ONE plan's AllReduce several times at once (the kernels of
+    different streams overlap on the device); one more thread shares the first thread's stream (its calls are serialised
+    with that thread's).  Every output equals the oracle's bits."""
+    import threading
+    dims, count, reps = (27, 27), 70001, 4
+    plan = binding.Plan(dims, LAT)
+    n = plan.n
+    x = synth.rank_matrix("normal", 77, n, count)
+    want = oracle.allreduce(dims, LAT, x)
+    pad = (count + 3) // 4 * 4
+    xin = torch.zeros((n, pad), dtype=torch.float32, device=DEV)
+    xin[:, :count].copy_(torch.from_numpy(x))
+    ip = binding.ptr_array([xin[r].data_ptr() for r in range(n)])
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    use = [0, 1, 2, 0]
+    outs = [torch.zeros((reps, n, pad), dtype=torch.float32, device=DEV) for _ in use]
+    torch.cuda.synchronize()
+    errors, names = [], []
+
+    def worker(t):
+        try:
+            st = streams[use[t]].cuda_stream
+            for k in range(reps):
+                op = binding.ptr_array([outs[t][k, r].data_ptr() for r in range(n)])
+                plan.allreduce_ex(ip, op, count, binding.FLOAT32, kernel=FUSED, stream=st)
+            names.append(binding.last_kernel_name())
+        except Exception as e:      # pragma: no cover
+            errors.append(e)
+
+    threads = [threading.Thread(target=worker, args=(t,)) for t in range(len(use))]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    torch.cuda.synchronize()
+    assert not errors and names == ["lat_t27x27_wide"] * len(use)
+    for o in outs:
+        got = o[:, :, :count].cpu().numpy()
+        for k in range(reps):
+            assert np.array_equal(got[k].view(np.uint32), want.view(np.uint32))
+    assert binding.tma_giveups() == 0
+    plan.destroy()
+
+
 def test_fp32_tolerance_against_naive_and_exact_sums():
     """|err| <= 2e-6 * sum|x| against the naive sequential binary32 sum (and the fp64 sum)."""
     for dims, variant, dist in [((27,), LAT, "normal"), ((81,), BW, "normal"), ((9, 9, 9), LAT, "uniform"),
