@@ -579,25 +579,18 @@ static WideSched* wide_sched_for(int dev, cudaStream_t st) {
     if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
     if (cap != cudaStreamCaptureStatusNone) return nullptr;
     if (st == cudaStreamLegacy) st = nullptr;                   // both name the legacy default stream
-    struct PerDevice {
-        WideSched* base = nullptr;
-        std::map<cudaStream_t, int> slot;
-    };
+    void* base = nullptr;               // asked for in every call: a pointer kept from before a device reset would dangle
+    if (cudaGetSymbolAddress(&base, g_wide_sched) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
     static std::mutex mu;
-    static std::map<int, PerDevice> devices;
+    static std::map<int, std::map<cudaStream_t, int>> slots;    // per device: stream -> counter number
     std::lock_guard<std::mutex> lock(mu);
-    PerDevice& d = devices[dev];
-    if (!d.base) {
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_wide_sched) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
-        d.base = (WideSched*)p;
+    std::map<cudaStream_t, int>& d = slots[dev];
+    auto it = d.find(st);
+    if (it == d.end()) {
+        if ((int)d.size() >= kWideSchedSlots) return nullptr;
+        it = d.emplace(st, (int)d.size()).first;
     }
-    auto it = d.slot.find(st);
-    if (it == d.slot.end()) {
-        if ((int)d.slot.size() >= kWideSchedSlots) return nullptr;
-        it = d.slot.emplace(st, (int)d.slot.size()).first;
-    }
-    return d.base + it->second;
+    return (WideSched*)base + it->second;
 }
 
 // false: this call cannot use the wide kernel (the caller goes on to the 32-column kernels)
