@@ -207,6 +207,10 @@ static trv_status_t lat_fused_launch(const Call& c, const Addr& in, const Addr& 
         else if (A == 3 && D == 4) { g_last_kernel = "lat_reg<3x3x3x3>"; launch_reg<T, 3, 4, 2, 64>(c, in, out, a); }
         else return TRV_ERR_UNSUPPORTED;
     } else if (kind == LatKind::Ring) {
+        if (p.n == 729) {               // long vectors, equally spaced rank buffers: the persistent 64-column kernel
+            trv_status_t st = TRV_OK;
+            if (run_fused_r729_wide(c, a, &st)) return st;
+        }
         // Ring of 243, long vectors: tiles of 64 columns (256 bytes per rank and tile), three CTAs per SM (72 registers).
         // Every tile touches all 243 input and all 243 output rows, and the 32-column kernel loses bandwidth as the rows
         // get longer (0.93 of the copy bandwidth at 2 MiB per rank, 0.85 at 8 MiB, 0.83 at 32 MiB) while the 64-column

@@ -62,6 +62,7 @@ bool run_fused_t999_tma(const Call& c, const LatArgs& a, trv_status_t* status);
 bool run_fused_t999_wide(const Call& c, const LatArgs& a, trv_status_t* status);
 bool run_fused_t2727_wide(const Call& c, const LatArgs& a, trv_status_t* status);
 bool run_fused_t981_wide(const Call& c, const LatArgs& a, trv_status_t* status);
+bool run_fused_r729_wide(const Call& c, const LatArgs& a, trv_status_t* status);
 bool fused_lines_supported(const Plan& p);
 void lines_prepare(Plan& p);
 void latency_prepare(Plan& p);

@@ -518,6 +518,136 @@ struct Shape981 {
     }
 };
 
+// ------------------------------------------------------------------ ring of 729
+//
+// rank r = a + 9 b + 81 c: the index space and the plane (the ranks with b = k, landing as [c][a]) of the 9 x 81 shape.
+// Steps 1 3 9 27 81 243.  Distance 1 and 3 walk the whole ring: warp w takes the 81 positions with c = w as an open
+// segment whose halo (four positions on either side, the neighbouring warps' values) it reads before anybody stores, and
+// runs both steps in one pass.  Distance 9 and 27 walk the ring of the 81 positions {a + 9 m} of one a (distance 1 and 3
+// in m = b + 9 c): one ring per warp, the same two-step pass with the ring's own other end as the halo.  Distance 81 and 243 stay inside the 9-rank sets {a, b fixed}, which lie inside ONE plane:
+// three phases of three planes.
+//
+// Two steps at once on an open segment of L positions (L a multiple of 9) with four halo positions on either side, in
+// place: t[i] = (old[i - 1] + old[i]) + old[i + 1], then out[i] = (t[i - 3] + t[i]) + t[i + 3] -- a distance-1 step followed
+// by a distance-3 step, both roundings as the two separate steps have them.  Nine outputs at a time; out[i] is stored
+// after old[i + 12] has been loaded, and nothing at or before i is read again.
+template <int L, typename E, typename Load, typename Store>
+__device__ __forceinline__ void wide_seg_stencil13(Load load, Store store, const E (&left)[4], const E (&right)[4]) {
+    auto old_at = [&](int i) { return i < 0 ? left[i + 4] : (i < L ? load(i) : right[i - L]); };     // i known at compile time
+    E t6[6], o2[2];         // t[9k - 3 .. 9k + 2] and old[9k + 2], old[9k + 3]
+    {
+        E o[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[i] = old_at(i - 4);
+#pragma unroll
+        for (int i = 0; i < 6; ++i) t6[i] = add3(o[i], o[i + 1], o[i + 2]);
+        o2[0] = o[6]; o2[1] = o[7];
+    }
+#pragma unroll
+    for (int k = 0; k < L / 9; ++k) {
+        E o[11], t[15];
+        o[0] = o2[0]; o[1] = o2[1];
+#pragma unroll
+        for (int m = 0; m < 9; ++m) o[2 + m] = old_at(9 * k + 4 + m);
+#pragma unroll
+        for (int i = 0; i < 6; ++i) t[i] = t6[i];
+#pragma unroll
+        for (int m = 0; m < 9; ++m) t[6 + m] = add3(o[m], o[m + 1], o[m + 2]);         // t[9k + 3 + m]
+#pragma unroll
+        for (int m = 0; m < 9; ++m) store(9 * k + m, add3(t[m], t[m + 3], t[m + 6]));  // t[9k + m - 3], t[9k + m], t[9k + m + 3]
+#pragma unroll
+        for (int i = 0; i < 6; ++i) t6[i] = t[9 + i];
+        o2[0] = o[9]; o2[1] = o[10];
+    }
+}
+
+template <typename T, bool FULL>
+__device__ __forceinline__ bool wide_tile_729(const PlaneMaps& maps, const StrideAddr& out, const LatArgs& a, long long t0,
+                                              unsigned parity, bool has_next, long long nt0, T* slab, unsigned long long* bars,
+                                              int* gave_up) {
+    constexpr int PK = 81;              // row of rank a + 9 b + 81 c in the slab: b * PK + c * 9 + a
+    using E = Elem<T, 2>;
+    const int lane = threadIdx.x % 32, set = threadIdx.x / 32;
+    const long long lo = a.lo[0], hi = a.hi[0];
+    const long long e = t0 + 2 * lane;
+    E* const mine = reinterpret_cast<E*>(slab) + lane;
+    auto sl = [&](int r) -> E& { return mine[r * (kWideCols / 2)]; };
+    const int prev_c = (set + 8) % 9, next_c = (set + 1) % 9;
+#pragma unroll 1
+    for (int k = 0; k < 9; ++k) wide_wait_plane(bars, k, parity, gave_up);     // the ring crosses every plane
+    {   // ---- distance 1, then 3: segment c = set, positions i = a + 9 b; halo: the last four positions of c - 1, the first four of c + 1
+        E left[4], right[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            left[i] = sl(8 * PK + prev_c * 9 + 5 + i);
+            right[i] = sl(next_c * 9 + i);
+        }
+        __syncthreads();                // every halo is read before any segment is written
+        if (*gave_up) return false;
+        auto at = [&](int i) { return (i / 9) * PK + set * 9 + i % 9; };
+        wide_seg_stencil13<81, E>([&](int i) { return sl(at(i)); }, [&](int i, const E& v) { sl(at(i)) = v; }, left, right);
+    }
+    __syncthreads();
+    {   // ---- distance 9, then 27: the ring of the 81 positions m = b + 9 c with a = set -- a segment whose halo is its own other end
+        auto at = [&](int m) { return (m % 9) * PK + (m / 9) * 9 + set; };
+        E left[4], right[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            left[i] = sl(at(77 + i));
+            right[i] = sl(at(i));
+        }
+        wide_seg_stencil13<81, E>([&](int m) { return sl(at(m)); }, [&](int m, const E& v) { sl(at(m)) = v; }, left, right);
+    }
+    __syncthreads();
+    // ---- distance 81, then 243, on the sets {a, b fixed, c = 0 .. 8}: inside the plane b; phase k0 takes the planes k0, k0 + 3, k0 + 6
+    const unsigned slab_s = smem_u32(slab);
+#pragma unroll 1
+    for (int k0 = 0; k0 < 3; ++k0) {
+        E v[3][9];
+#pragma unroll
+        for (int m = 0; m < 3; ++m) {
+            const int q = set + 9 * m, r0 = (k0 + 3 * (q / 9)) * PK + q % 9;       // a = q % 9, b = k0 + 3 (q / 9)
+#pragma unroll
+            for (int idx = 0; idx < 9; ++idx) v[m][idx] = sl(r0 + 9 * idx);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // this thread's slab accesses before the engine's writes
+        __syncthreads();                    // everybody holds its part of the planes k0, k0 + 3, k0 + 6: they may be refilled
+        if (threadIdx.x == 0 && has_next) {
+            for (int kk = 0; kk < 3; ++kk) wide_fetch_plane_981<false>(maps, nt0, k0 + 3 * kk, slab_s, bars);
+        }
+#pragma unroll
+        for (int m = 0; m < 3; ++m) {
+            const int q = set + 9 * m, g0 = q % 9 + 9 * (k0 + 3 * (q / 9));
+            reg_step<9, 1, 9, 1>(v[m]);     // distance 81
+            reg_step<9, 1, 9, 3>(v[m]);     // distance 243
+            if (FULL || (e < hi && e + 2 > lo)) {
+#pragma unroll
+                for (int idx = 0; idx < 9; ++idx) store_elem<T, 2, FULL>(out.ptr(g0 + 81 * idx), e, lo, hi, v[m][idx]);
+            }
+        }
+    }
+    return true;
+}
+
+struct Shape729 {
+    static constexpr int kSlices = 1;
+    static bool encode(const StrideAddr& base, size_t count, const LatArgs&, int, CUtensorMap* out) {
+        const int strides[3] = {1, 81, 9};      // a, c, and b in the place of the plane coordinate
+        return encode_planes(base, count, strides, kWideCols, out);
+    }
+    __device__ static __forceinline__ void fetch(const PlaneMaps& maps, int c, long long t0, int k, unsigned slab_s,
+                                                 unsigned long long* bars) {
+        wide_fetch_plane_981<false>(maps, t0, k, slab_s, bars);
+    }
+    template <typename T>
+    __device__ static __forceinline__ bool tile(const PlaneMaps& maps, const StrideAddr& out, const LatArgs& a, int c, long long t0,
+                                                bool full, unsigned parity, bool has_next, int nc, long long nt0, T* slab,
+                                                unsigned long long* bars, int* gave_up) {
+        return full ? wide_tile_729<T, true>(maps, out, a, t0, parity, has_next, nt0, slab, bars, gave_up)
+                    : wide_tile_729<T, false>(maps, out, a, t0, parity, has_next, nt0, slab, bars, gave_up);
+    }
+};
+
 template <typename T, typename Shape>
 __global__ void __launch_bounds__(288, 1) k_lat_wide(const __grid_constant__ PlaneMaps maps, StrideAddr out, LatArgs a,
                                                      WideTiles w, unsigned* giveups, WideSched* sched) {
@@ -617,7 +747,7 @@ static bool run_wide(const Call& c, const LatArgs& a, const char* name, trv_stat
     // 2 MiB the two kernels tie, below it the 32-column kernels win: more, smaller tiles to spread over the SMs).
     // 27 x 27 has no 32-column TMA kernel to fall back to, only the line-group kernel, and wins from 256 KiB per rank on
     // (64 Ki elements: 114 -> 91 us; 512 Ki: 811 -> 611 us; 2 Mi: 3132 -> 2400 us; 8 Mi: 9.44 ms, 0.79 of the copy bandwidth).
-    if (local < (NS == 2 ? (1LL << 16) : (3LL << 18)) || w.total < 2LL * sms || w.total > (1LL << 30)) return false;
+    if (local < (NS == 3 ? (3LL << 18) : (1LL << 16)) || w.total < 2LL * sms || w.total > (1LL << 30)) return false;
     unsigned* giveups = tma_giveup_counter();
     if (!giveups) return false;
     PlaneMaps maps;
@@ -647,6 +777,13 @@ bool run_fused_t2727_wide(const Call& c, const LatArgs& a, trv_status_t* status)
     const Plan& p = *c.plan;
     if (p.ndims != 2 || p.dims[0] != 27 || p.dims[1] != 27 || p.stride[0] != 1 || p.stride[1] != 27) return false;
     return run_wide<Shape2727>(c, a, "lat_t27x27_wide", status);
+}
+
+// the ring of 729; false: not this shape or not this call
+bool run_fused_r729_wide(const Call& c, const LatArgs& a, trv_status_t* status) {
+    const Plan& p = *c.plan;
+    if (p.ndims != 1 || p.n != 729) return false;
+    return run_wide<Shape729>(c, a, "lat_ring729_wide", status);
 }
 
 // 9 x 81 (rank = x0 + 9 x1) and 81 x 9 (rank = x0 + 81 x1); false: not these shapes or not this call

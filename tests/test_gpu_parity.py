@@ -138,6 +138,16 @@ def test_fused_latency_9x81_tiles_of_64_columns():
     assert binding.tma_giveups() == 0
 
 
+def test_fused_latency_ring729_tiles_of_64_columns():
+    """Ring of 729: the persistent 64-column kernel with the steps 1 and 3 as open-segment stencils with halos (one
+    segment of 81 ranks per warp) and 9, 27 as ring stencils; ragged edges, both dtypes, in place and not."""
+    check_case((729,), LAT, 70001, "normal", 71, FUSED)
+    assert binding.last_kernel_name() == "lat_ring729_wide"
+    check_case((729,), LAT, 150034, "int32", 72, FUSED, in_place=False)
+    assert binding.last_kernel_name() == "lat_ring729_wide"
+    assert binding.tma_giveups() == 0
+
+
 def test_fused_bandwidth_wide_path_on_729_ranks_sampled():
     """9x9x9 with blocks of >= 256 elements: the oracle checks windows around slice and block
     boundaries and in block interiors."""
