@@ -143,6 +143,7 @@ __device__ __forceinline__ bool wide_tile(const PlaneMaps& maps, const StrideAdd
     __syncthreads();
     // ---- group 3: (B,3) (C,3) on the sets {A = i, B in b0 + 3 jj, C in c0 + 3 kk}, phase by phase in c0
     const int sA = a.rs[c][0], sB = a.rs[c][1], sC = a.rs[c][2];
+    const long long dB = 3LL * sB * out.stride, dC = 3LL * sC * out.stride;       // bytes between the rows of a set
     const unsigned slab_s = smem_u32(slab);
 #pragma unroll 1
     for (int c0 = 0; c0 < 3; ++c0) {
@@ -164,9 +165,18 @@ __device__ __forceinline__ bool wide_tile(const PlaneMaps& maps, const StrideAdd
             reg_step<9, 1, 3, 1>(v[m]);     // (B,3)
             reg_step<9, 3, 3, 1>(v[m]);     // (C,3)
             if (FULL || (e < hi && e + 2 > lo)) {
+                // nine rows at rank offsets 3 jj sB + 3 kk sC: one base pointer per set, the rest by two byte strides
+                char* row = out.ptr(g0);
 #pragma unroll
-                for (int idx = 0; idx < 9; ++idx)
-                    store_elem<T, 2, FULL>(out.ptr(g0 + 3 * (idx % 3) * sB + 3 * (idx / 3) * sC), e, lo, hi, v[m][idx]);
+                for (int kk = 0; kk < 3; ++kk) {
+                    char* r = row;
+#pragma unroll
+                    for (int jj = 0; jj < 3; ++jj) {
+                        store_elem<T, 2, FULL>(r, e, lo, hi, v[m][jj + 3 * kk]);
+                        r += dB;
+                    }
+                    row += dC;
+                }
             }
         }
     }
