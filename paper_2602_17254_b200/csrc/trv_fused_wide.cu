@@ -303,6 +303,7 @@ __device__ __forceinline__ bool wide_tile_2727(const PlaneMaps& maps, const Stri
     // ---- group 4: (A,9) (B,9) on the sets {A = a + 9 i, B = b + 9 j}; phase k0 takes the b with b / 3 = k0, whose planes are
     // k0, k0 + 3, k0 + 6; flat index i + 3 j
     const int sA = a.rs[c][0], sB = a.rs[c][1];
+    const long long dA = 9LL * sA * out.stride, dB = 9LL * sB * out.stride;
     const unsigned slab_s = smem_u32(slab);
 #pragma unroll 1
     for (int k0 = 0; k0 < 3; ++k0) {
@@ -324,9 +325,17 @@ __device__ __forceinline__ bool wide_tile_2727(const PlaneMaps& maps, const Stri
             reg_step<9, 1, 3, 1>(v[m]);     // (A,9)
             reg_step<9, 3, 3, 1>(v[m]);     // (B,9)
             if (FULL || (e < hi && e + 2 > lo)) {
+                char* row = out.ptr(g0);        // nine rows at rank offsets 9 i sA + 9 j sB: two byte strides from one base
 #pragma unroll
-                for (int idx = 0; idx < 9; ++idx)
-                    store_elem<T, 2, FULL>(out.ptr(g0 + 9 * (idx % 3) * sA + 9 * (idx / 3) * sB), e, lo, hi, v[m][idx]);
+                for (int j = 0; j < 3; ++j) {
+                    char* r = row;
+#pragma unroll
+                    for (int i = 0; i < 3; ++i) {
+                        store_elem<T, 2, FULL>(r, e, lo, hi, v[m][i + 3 * j]);
+                        r += dA;
+                    }
+                    row += dB;
+                }
             }
         }
     }
@@ -475,6 +484,7 @@ __device__ __forceinline__ bool wide_tile_981(const PlaneMaps& maps, const Strid
     __syncthreads();
     // ---- (B,9) (B,27) on the sets {A, Bl fixed, Bh = 0 .. 8}: inside the plane Bl; phase k0 takes the planes k0, k0 + 3, k0 + 6
     const int sA = a.rs[c][BFIRST ? 1 : 0], sB = a.rs[c][BFIRST ? 0 : 1];       // rank strides of the side of 9 and of the side of 81
+    const long long d9 = 9LL * sB * out.stride;         // bytes between the rows of a set
     const unsigned slab_s = smem_u32(slab);
 #pragma unroll 1
     for (int k0 = 0; k0 < 3; ++k0) {
@@ -497,7 +507,14 @@ __device__ __forceinline__ bool wide_tile_981(const PlaneMaps& maps, const Strid
             reg_step<9, 1, 9, 3>(v[m]);     // (B,27): distance 3 in Bh
             if (FULL || (e < hi && e + 2 > lo)) {
 #pragma unroll
-                for (int idx = 0; idx < 9; ++idx) store_elem<T, 2, FULL>(out.ptr(g0 + 9 * idx * sB), e, lo, hi, v[m][idx]);
+                {
+                    char* row = out.ptr(g0);
+#pragma unroll
+                    for (int idx = 0; idx < 9; ++idx) {
+                        store_elem<T, 2, FULL>(row, e, lo, hi, v[m][idx]);
+                        row += d9;
+                    }
+                }
             }
         }
     }
@@ -610,6 +627,7 @@ __device__ __forceinline__ bool wide_tile_729(const PlaneMaps& maps, const Strid
     }
     __syncthreads();
     // ---- distance 81, then 243, on the sets {a, b fixed, c = 0 .. 8}: inside the plane b; phase k0 takes the planes k0, k0 + 3, k0 + 6
+    const long long d81 = 81LL * out.stride;            // bytes between the rows of a set
     const unsigned slab_s = smem_u32(slab);
 #pragma unroll 1
     for (int k0 = 0; k0 < 3; ++k0) {
@@ -632,7 +650,14 @@ __device__ __forceinline__ bool wide_tile_729(const PlaneMaps& maps, const Strid
             reg_step<9, 1, 9, 3>(v[m]);     // distance 243
             if (FULL || (e < hi && e + 2 > lo)) {
 #pragma unroll
-                for (int idx = 0; idx < 9; ++idx) store_elem<T, 2, FULL>(out.ptr(g0 + 81 * idx), e, lo, hi, v[m][idx]);
+                {
+                    char* row = out.ptr(g0);
+#pragma unroll
+                    for (int idx = 0; idx < 9; ++idx) {
+                        store_elem<T, 2, FULL>(row, e, lo, hi, v[m][idx]);
+                        row += d81;
+                    }
+                }
             }
         }
     }
