@@ -16,6 +16,9 @@
 // On a torus every collective (slice of the vector) has its own program (grid.y = collective) and block + offset
 // needs one modular addition per dimension: the CTA tabulates it once for the block its first column lies in
 // (shared memory, 2 bytes per node); the threads of the few CTAs that straddle a block boundary compute it.
+// Few ranks leave a thread little to do (n loads, n stores): a ring of 8 reaches 0.77 - 0.82 of the copy bandwidth, 32 ranks
+// 0.95.  Letting a CTA work through 2 - 8 consecutive tiles made that worse (ring of 8: 0.50, 32 ranks: 0.80): what these
+// sizes lack is loads in flight, and a CTA that runs its tiles one after the other has fewer of them than eight CTAs side by side.
 #include <algorithm>
 #include <type_traits>
 #include <vector>
