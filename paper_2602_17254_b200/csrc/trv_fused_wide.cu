@@ -1,5 +1,5 @@
-// FUSED latency-optimal kernels for the 729-rank tori 9 x 9 x 9 and 27 x 27 (Sec. 4.2, Sec. 5) on tiles of 64 element
-// columns, for long vectors.
+// FUSED latency-optimal kernels for the 729-rank shapes 9 x 9 x 9, 27 x 27, 9 x 81 / 81 x 9 and the ring of 729 (Sec. 4.2,
+// Sec. 5) on tiles of 64 element columns, for long vectors: one persistent kernel, a shape policy for each.
 //
 // Why 64 columns: every tile touches all 729 input rows and all 729 output rows.  A plain copy that moves 128 bytes
 // per row visit (32 columns) stops at 0.89 - 0.90 of the copy bandwidth on this part however many CTAs are resident,
@@ -21,7 +21,7 @@
 // 27 x 27 (steps A1 B1 A3 B3 A9 B9): a plane is three A-lines (81 ranks); four groups: (A,1) on the 27-rank A-lines of a
 // plane, (B,1) on the B-lines, (A,3)(B,3) on the nine 9 x 9 sets {A = a0 + 3 i, B = b0 + 3 j} streamed row by row, and
 // (A,9)(B,9) on 3 x 3 sets in three phases whose planes are k0, k0 + 3, k0 + 6 -- the phase structure the refill needs.
-// 27 x 27, 729 x 8 MiB: 3132 us with the line-group kernel -> 2400 us.
+// 27 x 27, 729 x 8 MiB: 3132 us with the line-group kernel -> 2400 us.  9 x 81 and the ring of 729: see their sections below.
 // Every wait on a copy's mbarrier is bounded; a CTA that gives up counts it (trv_tma.cuh) and leaves without
 // storing the tile it waited for.
 #include <map>
@@ -34,8 +34,8 @@
 namespace trv {
 
 // Tile scheduling.  With a fixed assignment (tile t, t + grid, ...) the slowest SM ends the kernel; handing out tiles from a
-// counter instead is worth half a percent (three alternating runs each: 8.53 - 8.57 -> 8.50 - 8.51 ms).  The counter must belong to one launch at a time, and the call may
-// allocate nothing, so the library keeps a small pool of counters per device and gives every (device, stream) pair its own:
+// counter instead is worth half a percent (three alternating runs each: 8.53 - 8.57 -> 8.50 - 8.51 ms).  The counter must
+// belong to one launch at a time, and the call may allocate nothing, so the library keeps a small pool of counters per device and gives every (device, stream) pair its own:
 // launches of one stream run one after the other, and the last CTA of a launch puts the counter back to zero.  Calls
 // on the per-thread default stream (one handle, many streams), calls being captured into a graph (the graph may later
 // run on any stream) and streams beyond the pool take the fixed assignment.
