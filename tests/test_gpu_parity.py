@@ -121,6 +121,12 @@ def test_fused_latency_27x27_tiles_of_64_columns():
     assert binding.last_kernel_name() == "lat_t27x27_wide"
     check_case((27, 27), LAT, 300034, "int32", 52, FUSED, in_place=False)
     assert binding.last_kernel_name() == "lat_t27x27_wide"
+    # an element-range shard: the buffers hold elements [64999, 135000) of vectors of 200003 (the slice boundary at 100001
+    # falls inside the window, at an odd column)
+    check_case((27, 27), LAT, 70001, "normal", 53, FUSED, shard=(200003, 64999))
+    assert binding.last_kernel_name() == "lat_t27x27_wide"
+    check_case((9, 9, 9), LAT, 800003, "int32", 54, FUSED, in_place=False, shard=(2400011, 790001))
+    assert binding.last_kernel_name() == "lat_t999_wide"
     assert binding.tma_giveups() == 0
 
 
