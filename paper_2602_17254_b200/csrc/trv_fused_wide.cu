@@ -506,7 +506,6 @@ __device__ __forceinline__ bool wide_tile_981(const PlaneMaps& maps, const Strid
             reg_step<9, 1, 9, 1>(v[m]);     // (B,9): distance 1 in Bh
             reg_step<9, 1, 9, 3>(v[m]);     // (B,27): distance 3 in Bh
             if (FULL || (e < hi && e + 2 > lo)) {
-#pragma unroll
                 {
                     char* row = out.ptr(g0);
 #pragma unroll
@@ -649,7 +648,6 @@ __device__ __forceinline__ bool wide_tile_729(const PlaneMaps& maps, const Strid
             reg_step<9, 1, 9, 1>(v[m]);     // distance 81
             reg_step<9, 1, 9, 3>(v[m]);     // distance 243
             if (FULL || (e < hi && e + 2 > lo)) {
-#pragma unroll
                 {
                     char* row = out.ptr(g0);
 #pragma unroll
