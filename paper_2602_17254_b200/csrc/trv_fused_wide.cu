@@ -17,6 +17,8 @@
 // Measured on the way and dropped: all of group 3's 81 values in registers before a single refill of nine planes
 // (spills at 168 registers, 8.56 ms); eleven plane slots with the planes 2 and 5 of the tile after the next loading
 // early (8.75 ms: the run-time slot arithmetic costs more than the two planes' head start gains).
+// Asking the copy engine to bring the next tile's planes into L2 while groups 1 and 2 run (bulk tensor prefetch): slower
+// on the same box (8.22 - 8.31 -> 8.62 - 8.64 ms).
 // 9 x 9 x 9: the same three closed groups as the other 9 x 9 x 9 kernels: (A,1)(B,1) per C-plane, (C,1)(A,3), (B,3)(C,3).
 // 27 x 27 (steps A1 B1 A3 B3 A9 B9): a plane is three A-lines (81 ranks); four groups: (A,1) on the 27-rank A-lines of a
 // plane, (B,1) on the B-lines, (A,3)(B,3) on the nine 9 x 9 sets {A = a0 + 3 i, B = b0 + 3 j} streamed row by row, and
