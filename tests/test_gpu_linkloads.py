@@ -116,3 +116,18 @@ def test_swing_bucket_and_mirrored_link_loads(dims, algo, variant):
     assert got.steps == want["steps"] and got.bytes_sent_per_node == want["bytes_sent_per_node"] and got.tx_bytes == want["tx_bytes"]
     for name, key in [("total", "total"), ("lambda_", "lambda"), ("delta", "delta"), ("theta", "theta")]:
         assert np.isclose(getattr(got, name), want[key], rtol=1e-12, atol=0), name
+
+
+def test_table_generator_reproduces_the_papers_entries():
+    """paper_2602_17254_b200.tables: Table 1 on the ring of 27 and Table 2 on 9 x 9 and 4 x 4 x 4, from the GPU tally."""
+    from paper_2602_17254_b200 import tables
+    ring = {r["algorithm"]: r for r in tables.table((27,))}
+    assert ring["Trivance (L)"]["steps"] == 3 and np.isclose(ring["Trivance (L)"]["lambda"], 1.0)
+    assert np.isclose(ring["Trivance (L)"]["theta"], 13.0)                 # sum of 3^k: 1 + 3 + 9
+    assert np.isclose(ring["Trivance (B)"]["delta"], 26 / 27) and np.isclose(ring["Bruck (L)"]["theta"], 39.0)
+    assert np.isclose(ring["Bucket"]["theta"], 26 / 27) and ring["Bucket"]["steps"] == 52
+    t2 = {r["algorithm"]: r for r in tables.table((9, 9))}
+    assert np.isclose(t2["Trivance (L)"]["theta"], t2["Trivance (L)"]["paper_closed_form"])    # (D / 2)(a - 1) -> (D / 2) n^(1/D)
+    assert np.isclose(t2["Bucket"]["theta"], 80 / 81)
+    t3 = {r["algorithm"]: r for r in tables.table((4, 4, 4))}
+    assert np.isclose(t3["Rec.Doub. (L)"]["theta"], 9 * 3) and np.isclose(t3["Bucket"]["theta"], 63 / 64)   # D^2 (a - 1)
