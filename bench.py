@@ -210,7 +210,8 @@ class ClockSampler:
 
 MIN_REGION_S = 0.55     # every timed region lasts at least this long, so that NVML samples fall inside it
 PER_WORKLOAD = ["ring27_lat_2MiB", "ring81_bw_8MiB", "torus9x9x9_lat_32MiB", "torus9x9x9_bw_32MiB", "ring243_lat_8MiB",
-                "ring243_bw_8MiB", "ring243_lat_32MiB", "ring243_bw_32MiB"]      # the configurations with >= 2 MiB per rank
+                "ring243_bw_8MiB", "ring243_lat_32MiB", "ring243_bw_32MiB",      # the configurations with >= 2 MiB per rank
+                "torus27x27_lat_8MiB", "torus9x81_lat_8MiB", "ring729_lat_8MiB"]  # the other 729-rank shapes, latency form
 
 
 class Leg:

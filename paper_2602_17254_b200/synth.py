@@ -99,3 +99,7 @@ for _n in (32, 100):
 for _dims in ((32, 32), (8, 64), (16, 16, 4)):
     _name = "torus%s_bw_8MiB" % "x".join(map(str, _dims))
     CONFIGS[_name] = Workload(_name, _dims, BANDWIDTH, 8 * MiB // 4, "normal", 6)
+# The other 729-rank shapes in the latency form (27 x 27 is a torus the paper evaluates), 8 MiB per rank.
+for _dims in ((27, 27), (9, 81), (729,)):
+    _name = ("torus%s_lat_8MiB" % "x".join(map(str, _dims))) if len(_dims) > 1 else "ring729_lat_8MiB"
+    CONFIGS[_name] = Workload(_name, _dims, LATENCY, 8 * MiB // 4, "normal", 7)

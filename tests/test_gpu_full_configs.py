@@ -88,7 +88,8 @@ def _every_element(w, x_dev, res_dev, chunk_bytes=3 << 29):
 
 @pytest.mark.parametrize("name", ["ring243_lat_8MiB", "ring243_bw_8MiB", "ring243_lat_32MiB", "ring243_bw_32MiB",
                                   "torus9x9x9_lat_32MiB", "torus9x9x9_bw_32MiB", "ring32_bw_8MiB", "ring100_bw_8MiB",
-                                  "torus32x32_bw_8MiB", "torus8x64_bw_8MiB", "torus16x16x4_bw_8MiB"])
+                                  "torus32x32_bw_8MiB", "torus8x64_bw_8MiB", "torus16x16x4_bw_8MiB",
+                                  "torus27x27_lat_8MiB", "torus9x81_lat_8MiB", "ring729_lat_8MiB"])
 def test_config_full_size_every_element(name):
     """The multi-GiB configurations, in the launch configuration bench.py times (AUTO, separate outputs):
     first the boundary-centred windows (fast to fail), then every element against the oracle, then the
