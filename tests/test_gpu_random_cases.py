@@ -62,3 +62,28 @@ def test_random_case(case):
         kernel = AUTO
     plan.destroy()
     check_case(dims, variant, count, dist, seed, kernel, in_place=in_place, shard=shard)
+
+
+def _wide_cases(seed, k):
+    """The persistent 64-column kernels (729-rank shapes, long vectors): sizes just above their thresholds, ragged, sharded."""
+    rng = np.random.default_rng(seed)
+    shapes = [((27, 27), "lat_t27x27_wide"), ((9, 81), "lat_t9x81_wide"), ((81, 9), "lat_t81x9_wide"), ((729,), "lat_ring729_wide")]
+    out = []
+    for i in range(k):
+        dims, name = shapes[i % len(shapes)]
+        count = int(rng.integers(66000, 140000))
+        shard = None
+        if rng.random() < 0.5:
+            gcount = count + int(rng.integers(1, 300000))
+            shard = (gcount, int(rng.integers(0, gcount - count + 1)))
+        out.append((dims, name, count, bool(rng.random() < 0.5), shard, ["int32", "normal", "uniform"][int(rng.integers(0, 3))], 2000 + i))
+    return out
+
+
+@pytest.mark.parametrize("case", _wide_cases(20260218, 12), ids=lambda c: "%s-%d%s%s" % (
+    "x".join(map(str, c[0])), c[2], "-ip" if c[3] else "-oop", "-shard" if c[4] else ""))
+def test_random_case_on_the_wide_kernels(case):
+    dims, name, count, in_place, shard, dist, seed = case
+    check_case(dims, LAT, count, dist, seed, FUSED, in_place=in_place, shard=shard)
+    if shard is None or min(shard[0] - shard[1], count) >= 66000:
+        assert binding.last_kernel_name() == name
